@@ -1,0 +1,335 @@
+"""Pins of the fp64 oracle against things that are not the oracle itself:
+an independent Philox implementation, LAPACK routines, closed forms and the
+identities the paper states (Eq. 4, Eq. 5-6, Eq. 9)."""
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+# --------------------------------------------------------------------------
+# Philox4x32-10: independent library implementation (Triton's, CPU interpreter)
+# --------------------------------------------------------------------------
+
+_TRITON_PHILOX = r"""
+import sys, numpy as np, torch
+import triton, triton.language as tl
+
+@triton.jit
+def k(c_ptr, k_ptr, o_ptr, N: tl.constexpr):
+    i = tl.arange(0, N)
+    c0 = tl.load(c_ptr + 4 * i + 0).to(tl.uint32); c1 = tl.load(c_ptr + 4 * i + 1).to(tl.uint32)
+    c2 = tl.load(c_ptr + 4 * i + 2).to(tl.uint32); c3 = tl.load(c_ptr + 4 * i + 3).to(tl.uint32)
+    k0 = tl.load(k_ptr + 2 * i + 0).to(tl.uint32); k1 = tl.load(k_ptr + 2 * i + 1).to(tl.uint32)
+    a, b, c, d = tl.philox_impl(c0, c1, c2, c3, k0, k1, 10)
+    tl.store(o_ptr + 4 * i + 0, a.to(tl.int32, bitcast=True)); tl.store(o_ptr + 4 * i + 1, b.to(tl.int32, bitcast=True))
+    tl.store(o_ptr + 4 * i + 2, c.to(tl.int32, bitcast=True)); tl.store(o_ptr + 4 * i + 3, d.to(tl.int32, bitcast=True))
+
+N = 64
+rng = np.random.default_rng(12345)
+ctr = rng.integers(0, 2**32, size=(N, 4), dtype=np.uint64).astype(np.uint32)
+key = rng.integers(0, 2**32, size=(N, 2), dtype=np.uint64).astype(np.uint32)
+ctr[0] = 0; key[0] = 0
+ctr[1] = 0xFFFFFFFF; key[1] = 0xFFFFFFFF
+c = torch.from_numpy(ctr.view(np.int32).copy()); kk = torch.from_numpy(key.view(np.int32).copy())
+o = torch.zeros((N, 4), dtype=torch.int32)
+k[(1,)](c, kk, o, N)
+np.save(sys.argv[1], np.concatenate([ctr, key, o.numpy().view(np.uint32)], axis=1))
+"""
+
+
+def test_philox_matches_independent_library(oracle, tmp_path):
+    pytest.importorskip("triton")
+    out = tmp_path / "philox.npy"
+    env = dict(os.environ, TRITON_INTERPRET="1")
+    r = subprocess.run([sys.executable, "-c", _TRITON_PHILOX, str(out)], env=env, capture_output=True, text=True,
+                       timeout=600)
+    if r.returncode != 0:
+        pytest.skip("triton interpreter unavailable: " + r.stderr[-300:])
+    table = np.load(out)
+    for row in table:
+        got = oracle.philox4x32_10(row[0:4], row[4:6])
+        assert np.array_equal(got, row[6:10]), (row, got)
+
+
+def test_philox_is_a_bijection_of_the_counter(oracle):
+    # Each round is invertible (odd multipliers): undo ten rounds and recover the counter.
+    M0, M1, W0, W1 = 0xD2511F53, 0xCD9E8D57, 0x9E3779B9, 0xBB67AE85
+    inv0, inv1 = pow(M0, -1, 2**32), pow(M1, -1, 2**32)
+    rng = np.random.default_rng(7)
+    for _ in range(20):
+        ctr = [int(x) for x in rng.integers(0, 2**32, 4)]
+        key = [int(x) for x in rng.integers(0, 2**32, 2)]
+        x = [int(v) for v in oracle.philox4x32_10(ctr, key)]
+        for r in reversed(range(10)):
+            k0 = (key[0] + r * W0) % 2**32; k1 = (key[1] + r * W1) % 2**32
+            c2 = (x[1] * inv1) % 2**32; c0 = (x[3] * inv0) % 2**32
+            c1 = x[0] ^ ((M1 * c2) >> 32) ^ k0; c3 = x[2] ^ ((M0 * c0) >> 32) ^ k1
+            x = [c0, c1, c2, c3]
+        assert x == ctr
+
+
+def test_word_stream_layout(oracle):
+    seed = (0xABCDEF01 << 32) | 0x12345678
+    w = oracle.philox_words(seed, 3, 2, 0, 64)
+    # element e sits in block e // 4, word e % 4; key = (lo, hi) of the seed; counter = (q, 0, stream, attempt)
+    for e in (0, 1, 5, 18, 63):
+        blk = oracle.philox4x32_10([e // 4, 0, 3, 2], [0x12345678, 0xABCDEF01])
+        assert w[e] == blk[e % 4]
+    # windows of the stream agree with the whole
+    assert np.array_equal(oracle.philox_words(seed, 3, 2, 5, 11), w[5:16])
+    # the high counter word takes over past 2^34 elements
+    far = oracle.philox_words(seed, 3, 2, (1 << 34) + 4, 4)
+    assert np.array_equal(far, oracle.philox4x32_10([1, 1, 3, 2], [0x12345678, 0xABCDEF01]))
+    # stream, attempt and seed all change the words
+    for other in (oracle.philox_words(seed, 2, 2, 0, 64), oracle.philox_words(seed, 3, 1, 0, 64),
+                  oracle.philox_words(seed + 1, 3, 2, 0, 64)):
+        assert (other != w).mean() > 0.9
+
+
+def test_gaussian_box_muller_structure(oracle):
+    seed, stream, attempt = 99, 1, 4
+    z = oracle.gaussian(seed, stream, attempt, 1, 4096).ravel()
+    w = oracle.philox_words(seed, stream, attempt, 0, 4096).astype(np.float64)
+    u = (np.floor(w / 256.0) + 0.5) / 2.0**24
+    r2 = z[0::2] ** 2 + z[1::2] ** 2
+    assert np.allclose(r2, -2.0 * np.log(u[0::2]), rtol=1e-12, atol=1e-14)
+    ang = np.mod(np.arctan2(z[1::2], z[0::2]), 2 * np.pi)
+    d = np.abs(ang - 2 * np.pi * u[1::2])
+    assert np.all(np.minimum(d, 2 * np.pi - d) < 1e-9)
+
+
+def test_gaussian_moments_and_ks(oracle):
+    from scipy import stats
+    z = oracle.gaussian(2024, 0, 0, 1000, 1000).ravel()
+    n = z.size
+    assert abs(z.mean()) < 5 / np.sqrt(n)
+    assert abs(z.var() - 1.0) < 5 * np.sqrt(2.0 / n)
+    assert abs(np.mean(z**4) - 3.0) < 5 * np.sqrt(96.0 / n)
+    assert abs(np.mean(z**3)) < 5 * np.sqrt(15.0 / n)
+    assert stats.kstest(z, "norm").pvalue > 1e-3
+    assert np.max(np.abs(z)) < 5.9  # 24-bit uniforms truncate the tails
+    # rows of a matrix are uncorrelated
+    g = z.reshape(1000, 1000)
+    c = (g[:-1] * g[1:]).mean()
+    assert abs(c) < 5 / np.sqrt(n)
+
+
+def test_gaussian_matrix_indexing(oracle):
+    g = oracle.gaussian(5, 0, 0, 7, 13)
+    flat = oracle.gaussian(5, 0, 0, 1, 91).ravel()
+    assert np.array_equal(g.ravel(), flat)
+
+
+# --------------------------------------------------------------------------
+# Linear algebra building blocks
+# --------------------------------------------------------------------------
+
+def test_matmul_against_blas(oracle):
+    rng = np.random.default_rng(0)
+    A = rng.standard_normal((37, 53)); B = rng.standard_normal((53, 29))
+    assert np.allclose(oracle.matmul(A, B), A @ B, rtol=1e-13, atol=1e-13)
+    # not symmetric in its operands: a transposed operand must change the answer
+    S = rng.standard_normal((9, 9)); T = rng.standard_normal((9, 9))
+    assert not np.allclose(oracle.matmul(S, T), S.T @ T)
+    rows = np.array([0, 36, 5, 5])
+    W = rng.standard_normal((53, 11))
+    assert np.allclose(oracle.rows_times_w(A, W, rows), A[rows] @ W, rtol=1e-13, atol=1e-13)
+
+
+@pytest.mark.parametrize("m", [1, 2, 3, 17, 64, 130])
+def test_householder_qr(oracle, m):
+    rng = np.random.default_rng(m)
+    G = rng.standard_normal((m, m))
+    Q, R = oracle.householder_qr(G)
+    assert np.allclose(Q.T @ Q, np.eye(m), atol=1e-13)
+    assert np.allclose(Q @ R, G, atol=1e-12)
+    assert np.all(np.tril(R, -1) == 0) and np.all(np.diag(R) > 0)
+    # LAPACK's factor, made unique the same way
+    Ql, Rl = np.linalg.qr(G)
+    s = np.sign(np.diag(Rl))
+    assert np.allclose(Q, Ql * s, atol=1e-9) and np.allclose(R, (Rl.T * s).T, atol=1e-9)
+
+
+def test_householder_qr_special_cases(oracle):
+    Q, R = oracle.householder_qr(np.array([[-3.0]]))
+    assert Q[0, 0] == -1.0 and R[0, 0] == 3.0
+    # an upper-triangular matrix with positive diagonal is its own R
+    T = np.triu(np.arange(1.0, 17.0).reshape(4, 4)) + np.eye(4)
+    Q, R = oracle.householder_qr(T)
+    assert np.allclose(Q, np.eye(4), atol=1e-14) and np.allclose(R, T, atol=1e-13)
+    # a rotation is its own Q
+    th = 0.3
+    G = np.array([[np.cos(th), -np.sin(th)], [np.sin(th), np.cos(th)]])
+    Q, R = oracle.householder_qr(G)
+    assert np.allclose(Q, G, atol=1e-14) and np.allclose(R, np.eye(2), atol=1e-14)
+
+
+@pytest.mark.parametrize("m", [1, 2, 5, 33, 100])
+def test_lu_inverse(oracle, m):
+    rng = np.random.default_rng(100 + m)
+    A = rng.standard_normal((m, m)) + 0.1 * np.eye(m)
+    X = oracle.lu_inverse(A)
+    assert np.allclose(X, np.linalg.inv(A), rtol=1e-8, atol=1e-8)
+    assert np.allclose(A @ X, np.eye(m), atol=1e-9)
+
+
+def test_lu_inverse_closed_forms(oracle):
+    rng = np.random.default_rng(3)
+    m = 12
+    P = np.eye(m)[rng.permutation(m)]            # needs pivoting; inverse is the transpose
+    assert np.array_equal(oracle.lu_inverse(P), P.T)
+    D = np.diag(np.arange(1.0, m + 1))
+    assert np.allclose(oracle.lu_inverse(D), np.diag(1.0 / np.arange(1.0, m + 1)), atol=1e-15)
+    u = rng.standard_normal((m, 1)); v = rng.standard_normal((m, 1))
+    B = np.eye(m) + u @ v.T                      # Sherman-Morrison
+    assert np.allclose(oracle.lu_inverse(B), np.eye(m) - (u @ v.T) / (1.0 + (v.T @ u).item()), atol=1e-11)
+    Z = np.array([[0.0, 2.0], [4.0, 1.0]])       # zero leading entry: a pivot swap is mandatory
+    assert np.allclose(oracle.lu_inverse(Z), np.array([[-0.125, 0.25], [0.5, 0.0]]), atol=1e-15)
+    with pytest.raises(ZeroDivisionError):
+        oracle.lu_inverse(np.ones((3, 3)))
+
+
+def test_condition_number(oracle):
+    assert oracle.cond2(np.diag(np.arange(1.0, 41.0))) == pytest.approx(40.0, rel=1e-12)
+    rng = np.random.default_rng(11)
+    Q, _ = np.linalg.qr(rng.standard_normal((30, 30)))
+    assert oracle.cond2(Q) == pytest.approx(1.0, abs=1e-12)
+    A = rng.standard_normal((48, 48))
+    s = np.linalg.svd(A, compute_uv=False)
+    hi, lo = oracle.singular_extremes(A)
+    assert hi == pytest.approx(s[0], rel=1e-10) and lo == pytest.approx(s[-1], rel=1e-8)
+
+
+def test_median_row_norm_and_shields(oracle):
+    rng = np.random.default_rng(5)
+    for n in (1, 2, 7, 10):
+        H = rng.standard_normal((n, 19)) * rng.uniform(0.1, 5.0, size=(n, 1))
+        assert oracle.median_row_norm(H) == pytest.approx(np.median(np.linalg.norm(H, axis=1)), rel=1e-14)
+    H = rng.standard_normal((64, 4096))
+    H /= np.sqrt((H * H).mean(axis=1, keepdims=True))
+    S = oracle.shield_rows(H, 6, 10.0, seed=77)
+    med = np.median(np.linalg.norm(H, axis=1))
+    # one global factor on unit-variance Gaussian rows drawn from stream 2
+    G = oracle.gaussian(77, 2, 0, 6, 4096)
+    assert np.allclose(S, (10.0 * med / 64.0) * G, rtol=1e-14)
+    # "scaled to 10x the median row norm": shield norms concentrate at 10 * med
+    assert np.allclose(np.linalg.norm(S, axis=1), 10.0 * med, rtol=0.06)
+    assert oracle.shield_rows(H, 0, 10.0, seed=77).shape == (0, 4096)
+
+
+# --------------------------------------------------------------------------
+# What the paper fixes (Section 3.2 and its Gram-leak discussion)
+# --------------------------------------------------------------------------
+
+def _inputs(rng, n, d, p):
+    return rng.standard_normal((n, d)), 0.02 * rng.standard_normal((d, p))
+
+
+@pytest.mark.parametrize("kind", [0, 1])
+def test_a_times_inverse_is_identity(oracle, kind):
+    A, X = oracle.sample_mixing(40, kind, seed=8)
+    assert np.allclose(A @ X, np.eye(40), atol=1e-11) and np.allclose(X @ A, np.eye(40), atol=1e-11)
+    if kind == 0:
+        assert np.array_equal(X, A.T)                      # "If A is orthogonal, A^-1 = A^T"
+        assert np.allclose(A.T @ A, np.eye(40), atol=1e-13)
+    else:
+        assert np.linalg.norm(A.T @ A - np.eye(40)) / np.sqrt(40) > 0.3   # Mitigation 1: A^T A != I
+        assert oracle.cond2(A) < 100.0
+
+
+@pytest.mark.parametrize("kind,k", [(0, 0), (1, 0), (0, 3), (1, 5)])
+def test_chain_equals_direct_product(oracle, kind, k):
+    # Eq. 4: A^-1((A H') W) = H' W ; the first n rows are H W and the shield rows are gone
+    rng = np.random.default_rng(21 + k)
+    n, d, p = 24, 16, 12
+    H, W = _inputs(rng, n, d, p)
+    S = oracle.shield_rows(H, k, 10.0, seed=4) if k else None
+    A, X = oracle.sample_mixing(n + k, kind, seed=4)
+    U, Yp, Y = oracle.chain(A, X, H, S, W, want_intermediates=True)
+    assert Y.shape == (n, p)
+    assert np.allclose(Y, H @ W, atol=1e-11)
+    Hf = H if S is None else np.vstack([H, S])
+    assert np.allclose(U, A @ Hf, atol=1e-12) and np.allclose(Yp, (A @ Hf) @ W, atol=1e-11)
+    assert np.allclose(X @ Yp, Hf @ W, atol=1e-10)         # the full un-mixed block, shields included
+    assert not np.allclose(U[:n], H, atol=1e-2)            # mixing does hide H
+
+
+def test_gram_identities(oracle):
+    rng = np.random.default_rng(9)
+    n, d, k = 32, 20, 4
+    H, _ = _inputs(rng, n, d, 6)
+    S = oracle.shield_rows(H, k, 10.0, seed=1)
+    Hf = np.vstack([H, S])
+    A, _ = oracle.sample_mixing(n + k, 0, seed=1)
+    U = oracle.matmul(A, Hf)
+    # Eq. 5 and Eq. 9: U^T U = H'^T H' = H^T H + S^T S
+    assert np.allclose(U.T @ U, H.T @ H + S.T @ S, rtol=1e-11, atol=1e-9)
+    # Eq. 6: U U^T is similar to H' H'^T (same spectrum)
+    assert np.allclose(np.linalg.eigvalsh(U @ U.T), np.linalg.eigvalsh(Hf @ Hf.T), rtol=1e-8, atol=1e-8)
+    # Mitigation 1: a non-orthogonal A masks the Gram matrix
+    B, _ = oracle.sample_mixing(n + k, 1, seed=1)
+    V = oracle.matmul(B, Hf)
+    G0 = Hf.T @ Hf
+    assert np.linalg.norm(V.T @ V - G0) / np.linalg.norm(G0) > 0.1
+
+
+def test_same_seed_same_matrix(oracle):
+    for kind in (0, 1):
+        A1, X1 = oracle.sample_mixing(20, kind, seed=123)
+        A2, X2 = oracle.sample_mixing(20, kind, seed=123)
+        A3, _ = oracle.sample_mixing(20, kind, seed=124)
+        A4, _ = oracle.sample_mixing(20, kind, seed=123, attempt=1)
+        assert np.array_equal(A1, A2) and np.array_equal(X1, X2)
+        assert not np.allclose(A1, A3) and not np.allclose(A1, A4)
+
+
+def test_orthogonal_sample_is_q_of_the_gaussian(oracle):
+    m = 16
+    A, _ = oracle.sample_mixing(m, 0, seed=55)
+    G = oracle.gaussian(55, 0, 0, m, m)
+    Ql, Rl = np.linalg.qr(G)
+    assert np.allclose(A, Ql * np.sign(np.diag(Rl)), atol=1e-10)
+    # non-orthogonal: Q0 + gamma * G1 / sqrt(m), G1 from stream 1
+    B, _ = oracle.sample_mixing(m, 1, seed=55, gamma=0.5)
+    assert np.allclose(B - A, 0.5 * oracle.gaussian(55, 1, 0, m, m) / np.sqrt(m), atol=1e-13)
+
+
+def test_verified_sampling_resamples(oracle):
+    # with a large gamma the Gaussian part dominates and kappa <= 100 is rare at first try;
+    # the verified sampler must return an attempt that really meets the bound
+    m = 48
+    A, X, c, attempt = oracle.sample_mixing_verified(m, 1, seed=3, gamma=0.5)
+    assert attempt == 0 and c < 10.0
+    found = False
+    for seed in range(40):
+        try:
+            A, X, c, attempt = oracle.sample_mixing_verified(m, 1, seed=seed, gamma=40.0, max_attempts=8)
+        except ArithmeticError:
+            continue
+        assert c <= 100.0 and c == pytest.approx(np.linalg.cond(A), rel=1e-6)
+        if attempt > 0:
+            found = True
+            A0, _ = oracle.sample_mixing(m, 1, seed, 0, 40.0)
+            assert np.linalg.cond(A0) > 100.0
+            break
+    assert found
+
+
+def test_golden_fixture(oracle):
+    path = os.path.join(ROOT, "tests", "golden", "oracle_seed0.txt")
+    vals = {}
+    with open(path) as f:
+        for line in f:
+            if line.startswith("#") or not line.strip():
+                continue
+            name, rest = line.split(":", 1)
+            vals[name.strip()] = rest.split()
+    w = oracle.philox_words(0, 0, 0, 0, 8)
+    assert [f"{int(x):08x}" for x in w] == vals["philox_words_seed0_stream0"]
+    A, _ = oracle.sample_mixing(4, 0, seed=0)
+    assert np.allclose(A.ravel(), np.array(vals["orthogonal_A_m4_seed0"], dtype=float), atol=1e-15)
