@@ -69,10 +69,11 @@ void oracle_philox_words(uint64_t seed, uint32_t stream, uint32_t attempt,
     }
 }
 
-/* 24-bit uniform strictly inside (0,1): u = ((w >> 8) + 1/2) * 2^-24. */
+/* 23-bit uniform strictly inside (0,1): u = ((w >> 9) + 1/2) * 2^-23.  Every such u is
+ * exactly representable in binary32, so a single-precision sampler sees the same u. */
 static double uniform_from_word(uint32_t w)
 {
-    return ((double)(w >> 8) + 0.5) * (1.0 / 16777216.0);
+    return ((double)(w >> 9) + 0.5) * (1.0 / 8388608.0);
 }
 
 /*

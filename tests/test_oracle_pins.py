@@ -95,7 +95,7 @@ def test_gaussian_box_muller_structure(oracle):
     seed, stream, attempt = 99, 1, 4
     z = oracle.gaussian(seed, stream, attempt, 1, 4096).ravel()
     w = oracle.philox_words(seed, stream, attempt, 0, 4096).astype(np.float64)
-    u = (np.floor(w / 256.0) + 0.5) / 2.0**24
+    u = (np.floor(w / 512.0) + 0.5) / 2.0**23
     r2 = z[0::2] ** 2 + z[1::2] ** 2
     assert np.allclose(r2, -2.0 * np.log(u[0::2]), rtol=1e-12, atol=1e-14)
     ang = np.mod(np.arctan2(z[1::2], z[0::2]), 2 * np.pi)
@@ -112,7 +112,7 @@ def test_gaussian_moments_and_ks(oracle):
     assert abs(np.mean(z**4) - 3.0) < 5 * np.sqrt(96.0 / n)
     assert abs(np.mean(z**3)) < 5 * np.sqrt(15.0 / n)
     assert stats.kstest(z, "norm").pvalue > 1e-3
-    assert np.max(np.abs(z)) < 5.9  # 24-bit uniforms truncate the tails
+    assert np.max(np.abs(z)) < 5.78  # 23-bit uniforms truncate the tails at sqrt(48 ln 2)
     # rows of a matrix are uncorrelated
     g = z.reshape(1000, 1000)
     c = (g[:-1] * g[1:]).mean()
