@@ -1,0 +1,341 @@
+#!/usr/bin/env python
+"""Benchmark of the GELO obfuscated Q/K/V offload on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+One step = one prefill sweep over the 32 layers of a Llama-2-7B-shaped model: 32 calls of
+the whole path (sample a fresh A, shield rows, mix, project, unmix) on n = 4096 token rows
+with d = 4096, p = 12288, 204 shield rows, bf16 storage, mixing kind alternating between
+orthogonal and non-orthogonal.  Inputs are seeded synthetic tensors (see
+paper_2603_05035_b200/inputs.py).  Rank 0 prints ONE JSON line.
+
+With N > 1 every rank runs an independent replica of the same sweep (the path has no
+exchange step), and the value is the total number of token rows all ranks pushed through
+the obfuscated projection divided by the slowest rank's time.
+
+--impl reference times the fp64 CPU oracle on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "obfuscated-QKV tokens/s at Llama-2-7B shapes"
+UNIT = "tokens/s"
+WORKLOAD = "prefill_bf16"
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            d = json.load(f)
+        return {"hbm_gbs": float(d["hbm_gbs"]), "bf16_tflops": float(d["bf16_tflops"]),
+                "bf16_tflops_sustained": float(d.get("bf16_tflops_sustained", d["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "200",
+                 "-i", str(self.gpu)], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._pump, daemon=True)
+        self.thread.start()
+
+    def _pump(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in self.lines:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 9:
+                continue
+            try:
+                sm.append(float(parts[1])); mx.append(float(parts[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, parts[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ---------------------------------------------------------------------------------------------
+# reference arm and CPU baseline: the oracle on the host cores
+# ---------------------------------------------------------------------------------------------
+
+def oracle_sample_step(w, n_s, k_s, call):
+    """One oracle pass of the whole path on a reduced row count (same d, p, dtype, kinds)."""
+    import numpy as np
+    import oracle
+    from paper_2603_05035_b200 import inputs
+    seed = w.seed + call
+    H = inputs.to_f64_numpy(inputs.make_hidden(n_s, w.d, w.dtype, seed, w.rms_norm))
+    W = inputs.to_f64_numpy(inputs.make_weight(w.d, w.p, w.dtype, seed))
+    t0 = time.perf_counter()
+    A, X, _, _ = oracle.sample_mixing_verified(n_s + k_s, w.kind(call), seed)
+    S = oracle.shield_rows(H, k_s, w.shield_scale, seed) if k_s else None
+    Y = oracle.chain(A, X, H, S, W)
+    dt = time.perf_counter() - t0
+    assert np.isfinite(Y).all()
+    return dt
+
+
+def oracle_sample_desc(n_s, k_s, w):
+    return (f"whole path (sample A, shields, mix, project, unmix) in fp64 on n={n_s} data rows + {k_s} "
+            f"shield rows per call, d={w.d}, p={w.p}; tokens/s = {n_s} / seconds per call")
+
+
+def run_reference(args):
+    import oracle
+    from paper_2603_05035_b200 import inputs
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    oracle.build()
+    w = inputs.WORKLOADS[WORKLOAD]
+    n_s, k_s = 128, 6
+    for i in range(args.warmup):
+        oracle_sample_step(w, 16, 1, i)
+    times = [oracle_sample_step(w, n_s, k_s, i) for i in range(args.steps)]
+    total = sum(times)
+    value = n_s * args.steps / total
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "n": w.n, "k": w.k, "d": w.d, "p": w.p, "calls_per_step": 1,
+                   "note": "CPU oracle on a bounded sample; one step = one call of the sample"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": oracle_sample_desc(n_s, k_s, w)},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ---------------------------------------------------------------------------------------------
+# our arm
+# ---------------------------------------------------------------------------------------------
+
+def run_ours(args):
+    import torch
+    import paper_2603_05035_b200 as gelo
+    from paper_2603_05035_b200 import inputs
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.gpus != world and world > 1:
+        raise SystemExit(f"--gpus {args.gpus} but WORLD_SIZE={world}")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    w = inputs.WORKLOADS[WORKLOAD]
+    n, k, d, p, m = w.n, w.k, w.d, w.p, w.m
+    calls = w.calls
+    td = inputs.torch_dtype(w.dtype)
+    dev = torch.device("cuda", local_rank)
+    peaks = _peaks()
+
+    ctx = gelo.Context(local_rank)
+    ctx.ensure_workspace(n, k, d, p, w.dtype)
+    # replicas draw different inputs and mixing seeds
+    base = rank * 1000
+    Hs, Ws, seeds = [], [], []
+    for c in range(calls):
+        h = inputs.make_hidden(n, d, w.dtype, w.seed + base + c, w.rms_norm, dev)
+        wt = inputs.make_weight(d, p, w.dtype, w.seed + base + c, dev)
+        Hs.append(h); Ws.append(wt); seeds.append(w.seed + base + c)
+    Q = torch.empty((n, p // 3), device=dev, dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
+    checksum = torch.zeros((), device=dev, dtype=torch.float32)
+
+    def sweep(step):
+        for c in range(calls):
+            ctx.qkv_offload(Hs[c], Ws[c], n, k, d, p, w.kind(c), seeds[c] + 100000 * step, w.shield_scale,
+                            w.dtype, Q, K, V)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for i in range(args.warmup):
+        sweep(-1 - i)
+    barrier()
+    if ctx.last_status() != gelo.OK:
+        raise SystemExit("device-side error during warm-up")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    ctx.launch_count(reset=True)
+    barrier()
+    e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for s in range(args.steps):
+        sweep(s)
+    e1.record()
+    barrier()
+    ms = e0.elapsed_time(e1)
+    launches = ctx.launch_count()
+    clocks = sampler.stop() if rank == 0 else None
+    status = ctx.last_status()
+    if status != gelo.OK:
+        raise SystemExit(f"device-side error {status} in the timed region")
+    checksum += Q.float().abs().mean()
+
+    # ---- per-stage device times (CUDA events on the launching stream), a few calls each ----
+    stage_ms = {}
+    lda = ctx.mixing_ld(m)
+    A = torch.empty((m, lda), device=dev, dtype=td); X = torch.empty_like(A)
+    S = torch.empty((k, d), device=dev, dtype=td)
+    U = torch.empty((m, d), device=dev, dtype=td); Yp = torch.empty((m, p), device=dev, dtype=td)
+
+    def timed(name, fn, reps):
+        fn(0)
+        torch.cuda.synchronize()
+        a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+        a.record()
+        for r in range(reps):
+            fn(r + 1)
+        b.record()
+        torch.cuda.synchronize()
+        stage_ms[name] = a.elapsed_time(b) / reps
+
+    timed("sample_orthogonal", lambda r: ctx.sample_mixing(m, gelo.ORTHOGONAL, 900 + r, w.dtype, A, X, lda), 2)
+    timed("sample_nonorthogonal", lambda r: ctx.sample_mixing(m, gelo.NONORTHOGONAL, 900 + r, w.dtype, A, X, lda), 2)
+    timed("shield_rows", lambda r: ctx.shield_rows(Hs[r % calls], n, d, k, w.shield_scale, 5 + r, w.dtype, S), 8)
+    timed("mix", lambda r: ctx.mix(A, lda, Hs[r % calls], S, n, k, d, w.dtype, U), 8)
+    timed("project", lambda r: ctx.project(U, Ws[r % calls], m, d, p, w.dtype, Yp), 8)
+    timed("unmix", lambda r: ctx.unmix(X, lda, Yp, n, k, p, w.dtype, Q, K, V), 8)
+    timed("plain_project", lambda r: ctx.project(Hs[r % calls], Ws[r % calls], n, d, p, w.dtype, Yp), 8)
+    chain_ms = stage_ms["mix"] + stage_ms["project"] + stage_ms["unmix"]
+    chain_flops = 2.0 * m * m * d + 2.0 * m * d * p + 2.0 * n * m * p
+    plain_flops = 2.0 * n * d * p
+
+    # ---- end to end through the host-buffer entry point (H2D of H, D2H of Q/K/V inside) ----
+    Hh = [h.cpu().pin_memory() for h in Hs[:4]]
+    Qh = torch.empty((n, p // 3), dtype=td).pin_memory(); Kh = torch.empty_like(Qh).pin_memory()
+    Vh = torch.empty_like(Qh).pin_memory()
+    e2e_calls = max(4, min(calls, 8))
+    for c in range(2):
+        ctx.qkv_offload_host(Hh[c % 4], Ws[c], n, k, d, p, w.kind(c), seeds[c], w.shield_scale, w.dtype, Qh, Kh, Vh)
+    barrier()
+    t0 = time.perf_counter()
+    for c in range(e2e_calls):
+        ctx.qkv_offload_host(Hh[c % 4], Ws[c], n, k, d, p, w.kind(c), seeds[c] + 7, w.shield_scale, w.dtype,
+                             Qh, Kh, Vh)
+    torch.cuda.synchronize()
+    e2e_s = time.perf_counter() - t0
+    checksum += Qh.float().abs().mean().to(dev)
+
+    t_ms = torch.tensor([ms, e2e_s * 1e3], device=dev, dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
+    ms_max, e2e_ms_max = float(t_ms[0]), float(t_ms[1])
+    tokens = float(n) * calls * args.steps * world
+    value = tokens / (ms_max * 1e-3)
+    e2e_value = float(n) * e2e_calls * world / (e2e_ms_max * 1e-3)
+
+    if rank == 0:
+        es = 2 if w.dtype == "bf16" else 4
+        # dominant product kernel of the chain: the projection GEMM (one launch per call)
+        proj_flops = 2.0 * m * d * p
+        achieved = proj_flops / (stage_ms["project"] * 1e-3) / 1e12
+        roofline = {"kernel": "projection GEMM Y' = U W (one launch per call)", "bound": "tensor",
+                    "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                    "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16 GEMM)",
+                    "traffic": None}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
+            "config": {"workload": WORKLOAD, "n": n, "k": k, "m": m, "d": d, "p": p, "calls_per_step": calls,
+                       "mixing": "alternating orthogonal / non-orthogonal, fresh A per call",
+                       "shield_scale": w.shield_scale, "l2": "inputs_larger_than_l2",
+                       "replicas": world},
+            "clocks": clocks,
+            "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": calls * n * d * es,
+                    "d2h_bytes_per_step": calls * n * p * es, "calls_timed": e2e_calls},
+            "gpu_launches": launches,
+            "roofline": roofline,
+            "stage_ms": {k_: round(v, 4) for k_, v in stage_ms.items()},
+            "chain": {"ms": chain_ms, "tflops": chain_flops / (chain_ms * 1e-3) / 1e12,
+                      "overhead_vs_plain_gemm": chain_ms / stage_ms["plain_project"],
+                      "flop_floor_vs_plain": chain_flops / plain_flops,
+                      "frac_of_peak": chain_flops / (chain_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
+            "checksum": float(checksum),
+        }
+        if world == 1 and not args.no_cpu_baseline:
+            import oracle
+            oracle.build()
+            n_s, k_s = 128, 6
+            dt_s = oracle_sample_step(w, n_s, k_s, 0)
+            line["cpu_baseline"] = {"value": n_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(),
+                                    "kind": "oracle", "sample": oracle_sample_desc(n_s, k_s, w)}
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    ctx.close()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=3)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

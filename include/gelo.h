@@ -1,0 +1,188 @@
+/*
+ * gelo.h -- C ABI of the B200 (sm_100a) library for GELO's obfuscated Q/K/V offload.
+ *
+ * One call of the path (paper Section 3.2 "Core Algorithm", Eq. 1-4, with the two
+ * Gram-leak mitigations of Section 3.2.1):
+ *
+ *     sample a fresh secret invertible A (m x m, m = n + k)       step 1.2
+ *     S  = k shield rows, scaled to the median row norm of H      Mitigation 2, Eq. 7-8
+ *     U  = A [H; S]                                               Eq. 1
+ *     Y' = U W                                                    Eq. 2
+ *     Y  = (A^-1 Y')[0:n, :]  -> Q | K | V                        Eq. 3
+ *
+ * so that Y = H W (Eq. 4).
+ *
+ * Conventions for every entry point
+ *   - Return value: a gelo_status.  Nothing throws or aborts across this boundary.
+ *     Errors that the host can see (bad arguments, missing workspace, unsupported
+ *     shapes) are returned before anything is launched.  Conditions only the
+ *     device can see (condition bound missed after the last attempt, a bounded
+ *     wait that ran out) are recorded in a status word that gelo_last_status reads.
+ *   - "dev" pointers are device pointers on the context's GPU, owned by the caller,
+ *     16-byte aligned, row-major and contiguous unless a row stride is given.
+ *     "host" pointers are ordinary host memory (pinned memory makes the copies
+ *     asynchronous).  The library never frees or keeps caller memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
+ *     enqueued on it; calls return without waiting unless stated otherwise.
+ *   - Element type: GELO_F32 stores float, GELO_BF16 stores bfloat16; products always
+ *     accumulate in fp32.
+ *   - A and A^-1 are m x m with a row stride `lda` (in elements) that is a multiple of
+ *     8 and >= m; gelo_mixing_ld(m) returns the stride the library prefers.  Columns
+ *     m..lda-1 are padding: never read as data, contents unspecified.
+ *   - All other matrices are dense: H n x d, S k x d, U m x d, W d x p, Y' m x p,
+ *     Q/K/V n x (p/3).  d and p must be multiples of 8.
+ *   - Scratch memory comes from the caller through gelo_set_workspace; no entry point
+ *     except gelo_create / gelo_destroy allocates or frees device memory.
+ */
+#ifndef GELO_H
+#define GELO_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    GELO_OK = 0,
+    GELO_ERR_INVALID = 1,      /* bad argument (null pointer, negative size, bad stride, ...) */
+    GELO_ERR_WORKSPACE = 2,    /* no workspace set, or it is too small for this call */
+    GELO_ERR_COND = 3,         /* no A with kappa_2 <= bound within the attempt limit */
+    GELO_ERR_TIMEOUT = 4,      /* a bounded device-side wait ran out; outputs are invalid */
+    GELO_ERR_CUDA = 5,         /* a CUDA runtime or driver call failed */
+    GELO_ERR_UNSUPPORTED = 6   /* valid request this build cannot serve (wrong GPU, p % 3 != 0 with a split, ...) */
+} gelo_status;
+
+typedef enum { GELO_ORTHOGONAL = 0, GELO_NONORTHOGONAL = 1 } gelo_kind;
+typedef enum { GELO_F32 = 0, GELO_BF16 = 1 } gelo_dtype;
+
+/* Philox stream ids used by the library (third counter word). */
+enum { GELO_STREAM_G0 = 0, GELO_STREAM_G1 = 1, GELO_STREAM_SHIELD = 2, GELO_STREAM_POWER = 3 };
+
+typedef struct gelo_ctx gelo_ctx;
+
+/* ---- context ------------------------------------------------------------------- */
+
+/* Creates a context on CUDA device `device` (must be compute capability 10.x, else
+ * GELO_ERR_UNSUPPORTED).  Allocates a few hundred bytes of device and pinned host
+ * memory for the status word.  *ctx is NULL on failure. */
+int gelo_create(gelo_ctx** ctx, int device);
+int gelo_destroy(gelo_ctx* ctx);
+
+/* Bytes of scratch that any call with these sizes needs (n data rows, k shield rows,
+ * model width d, projection width p, element type t).  0 if an argument is invalid. */
+size_t gelo_workspace_bytes(int n, int k, int d, int p, int dtype);
+
+/* Hands the context a caller-owned device buffer (256-byte aligned).  It must stay
+ * valid until replaced or the context is destroyed.  Calls on one context share it, so
+ * they must be ordered on one stream. */
+int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes);
+
+/* Non-orthogonal construction A = Q0 + gamma * G1 (Mitigation 1; default gamma 0.5),
+ * the accepted bound on kappa_2(A) (default 100) and the number of attempts (default 8,
+ * each with the next attempt number in the Philox counter). */
+int gelo_set_nonorthogonal(gelo_ctx* ctx, float gamma, float cond_bound, int max_attempts);
+
+/* Preferred row stride (elements) of an m x m mixing matrix: m rounded up to 64. */
+int gelo_mixing_ld(int m);
+
+/* Status word of the context: waits for `stream`, then returns the first device-side
+ * error recorded since the last call of this function (GELO_OK if none) and clears it. */
+int gelo_last_status(gelo_ctx* ctx, void* stream);
+
+/* Number of kernels this context has launched since creation (or since the last reset). */
+long long gelo_launch_count(gelo_ctx* ctx, int reset);
+
+const char* gelo_status_string(int status);
+
+/* ---- sampling (Section 3.2 step 1.2: "sample a fresh, random invertible matrix") ---- */
+
+/* Debug export of the random stream: out_dev[i] = the Philox4x32-10 word of element
+ * first+i of (seed, stream_id, attempt).  Element e uses block e/4 -- counter
+ * (lo32(e/4), hi32(e/4), stream_id, attempt), key (lo32(seed), hi32(seed)) -- word e%4. */
+int gelo_philox_words(gelo_ctx* ctx, uint64_t seed, uint32_t stream_id, uint32_t attempt,
+                      uint64_t first, uint64_t count, uint32_t* out_dev, void* stream);
+
+/* out_dev (rows x cols fp32, row stride ld) = scale * N(0,1).  Element (i,j) is stream
+ * element i*cols + j; words (0,1) and (2,3) of a block are Box-Muller pairs, the even
+ * word giving r*cos(2 pi u_b), the odd word r*sin(2 pi u_b), r = sqrt(-2 ln u_a),
+ * u = ((word >> 8) + 1/2) / 2^24. */
+int gelo_sample_gaussian(gelo_ctx* ctx, int rows, int cols, int ld, uint64_t seed,
+                         uint32_t stream_id, uint32_t attempt, float scale, float* out_dev,
+                         void* stream);
+
+/* Q_dev = the orthogonal factor of the Householder QR of G_dev (both m x m fp32, stride
+ * ld), columns signed so that diag(R) > 0; Qt_dev (optional) = its transpose.  G_dev is
+ * overwritten.  Needs workspace for (m, 0). */
+int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev, float* Qt_dev,
+                       void* stream);
+
+/* Ainv_dev = A_dev^-1 by blocked LU with partial pivoting (both m x m fp32, stride ld);
+ * A_dev is preserved.  Needs workspace for (m, 0). */
+int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ainv_dev, void* stream);
+
+/* cond_dev[0] = estimate of kappa_2(A) = sigma_max(A) * sigma_max(A^-1) by power
+ * iteration on A^T A and A^-T A^-1 (a lower estimate, within a few percent). */
+int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
+                       float* cond_dev, void* stream);
+
+/* Samples the secret mixing pair for one batch.
+ *   GELO_ORTHOGONAL:    A = Q of QR(G0), G0 ~ N(0,1) from stream 0;  A^-1 = A^T.
+ *   GELO_NONORTHOGONAL: A = Q0 + gamma * G1 / sqrt(m) (G1 from stream 1), rounded to the
+ *                       element type, then A^-1 of that stored A; accepted when the
+ *                       kappa_2 estimate * 1.1 <= bound, else resampled with the next
+ *                       attempt number.  This kind WAITS for `stream` once per attempt
+ *                       to read the verdict; GELO_ERR_COND after the last attempt.
+ * A_dev, Ainv_dev: m x m in `dtype`, stride lda.  cond_dev (optional, device float)
+ * receives the estimate (1 for orthogonal).  Same (m, kind, seed) => same bytes. */
+int gelo_sample_mixing(gelo_ctx* ctx, int m, int kind, uint64_t seed, int dtype,
+                       void* A_dev, void* Ainv_dev, int lda, float* cond_dev, void* stream);
+
+/* ---- shield rows (Mitigation 2, Eq. 7-8) --------------------------------------------- */
+
+/* S_dev (k x d) = (scale * median_i ||H_i||_2 / sqrt(d)) * N(0,1) draws of stream 2.
+ * The median of an even number of rows is the mean of the middle two.  k = 0 is a no-op.
+ * Row norms use workspace scratch. */
+int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale,
+                     uint64_t seed, int dtype, void* S_dev, void* stream);
+
+/* ---- the three products (Eq. 1-3) ------------------------------------------------------ */
+
+/* U_dev ((n+k) x d) = A [H; S]; the stacked operand is never materialised.  S_dev may be
+ * NULL iff k == 0. */
+int gelo_mix(gelo_ctx* ctx, const void* A_dev, int lda, const void* H_dev, const void* S_dev,
+             int n, int k, int d, int dtype, void* U_dev, void* stream);
+
+/* Yp_dev (m x p) = U_dev (m x d) * W_dev (d x p): the offloaded GEMM; with U = H this is
+ * also the plain, unprotected projection. */
+int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int d, int p,
+                 int dtype, void* Yp_dev, void* stream);
+
+/* Rows 0..n-1 of Ainv * Yp (shield rows are dropped by never computing them), split by
+ * column thirds into Q_dev, K_dev, V_dev (each n x p/3; p % 3 == 0 and p/3 % 8 == 0).  If
+ * K_dev and V_dev are both NULL the whole n x p result goes to Q_dev. */
+int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev, int n, int k,
+               int p, int dtype, void* Q_dev, void* K_dev, void* V_dev, void* stream);
+
+/* ---- the whole call --------------------------------------------------------------------- */
+
+/* sample -> shields -> mix -> project -> unmix for one batch, all from workspace scratch.
+ * H_dev n x d, W_dev d x p; outputs as in gelo_unmix.  Waits for `stream` only when
+ * kind is GELO_NONORTHOGONAL (condition-number verdict). */
+int gelo_qkv_offload(gelo_ctx* ctx, const void* H_dev, const void* W_dev, int n, int k, int d,
+                     int p, int kind, uint64_t seed, float shield_scale, int dtype,
+                     void* Q_dev, void* K_dev, void* V_dev, void* stream);
+
+/* Same call for a caller whose activations live in host memory: H_host (n x d) is copied
+ * to the device, the result is copied back into Q_host, K_host, V_host (each n x p/3), and
+ * the function returns after the copies have completed.  W_dev stays a device pointer
+ * (weights are resident, paper Section 3.2 step 1.4). */
+int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, int n, int k,
+                          int d, int p, int kind, uint64_t seed, float shield_scale, int dtype,
+                          void* Q_host, void* K_host, void* V_host, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GELO_H */

@@ -1,0 +1,472 @@
+// C-ABI entry points of the GELO offload library (see include/gelo.h): argument
+// validation, workspace carving and the launch sequences.  No entry point except
+// gelo_create / gelo_destroy allocates device memory.
+#include <new>
+
+#include "common.cuh"
+
+using namespace gelo;
+
+namespace {
+
+inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+inline int round_up(int x, int to) { return (x + to - 1) / to * to; }
+
+// Every scratch buffer of one call with sizes (n, k, d, p, dtype); carved in a fixed order so
+// that gelo_workspace_bytes and the calls agree.
+struct Layout {
+    int m = 0, ldi = 0;
+    float* G = nullptr;       // m x ldi  Gaussian, then R
+    float* Qraw = nullptr;    // m x ldi
+    float* A32 = nullptr;     // m x ldi
+    float* X32 = nullptr;     // m x ldi
+    QrScratch qr;
+    LuScratch lu;
+    CondScratch cond;
+    ShieldScratch sh;
+    float* cond_val = nullptr;
+    void* A = nullptr;        // m x ldi, path dtype
+    void* Ainv = nullptr;
+    void* S = nullptr;        // k x d
+    void* U = nullptr;        // m x d
+    void* Yp = nullptr;       // m x p
+    void* Hd = nullptr;       // n x d   staging of the host variant
+    void* Yd = nullptr;       // n x p
+};
+
+Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
+{
+    Layout L;
+    const size_t es = elem_size(dtype);
+    L.m = n + k;
+    L.ldi = gelo_mixing_ld(L.m);
+    const size_t mat = (size_t)L.m * L.ldi;
+    L.G = static_cast<float*>(a.take(mat * 4));
+    L.Qraw = static_cast<float*>(a.take(mat * 4));
+    L.A32 = static_cast<float*>(a.take(mat * 4));
+    L.X32 = static_cast<float*>(a.take(mat * 4));
+    L.qr = carve_qr(a, L.m, L.ldi);
+    L.lu = carve_lu(a, L.m, L.ldi);
+    L.cond = carve_cond(a, L.m);
+    L.sh = carve_shield(a, n);
+    L.cond_val = static_cast<float*>(a.take(16));
+    L.A = a.take(mat * es);
+    L.Ainv = a.take(mat * es);
+    L.S = a.take((size_t)(k > 0 ? k : 1) * d * es);
+    L.U = a.take((size_t)L.m * d * es);
+    L.Yp = a.take((size_t)L.m * p * es);
+    if (host_staging) {
+        L.Hd = a.take((size_t)n * d * es);
+        L.Yd = a.take((size_t)n * p * es);
+    }
+    return L;
+}
+
+bool carve_ctx(gelo_ctx* ctx, int n, int k, int d, int p, int dtype, bool host_staging, Layout* out)
+{
+    if (!ctx->ws) return false;
+    Arena a;
+    a.base = static_cast<char*>(ctx->ws);
+    a.cap = ctx->ws_bytes;
+    *out = carve(a, n, k, d, p, dtype, host_staging);
+    return a.ok;
+}
+
+bool bad_dtype(int t) { return t != GELO_F32 && t != GELO_BF16; }
+bool bad_ld(int lda, int m) { return lda < m || (lda % 8) != 0; }
+bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+__global__ void set_scalar_kernel(float* p, float v) { *p = v; }
+
+int gemm_dispatch(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
+{
+    if (g.dtype == GELO_BF16 && gemm_tc_supports(g)) return launch_gemm_tc(ctx, g, st);
+    return launch_gemm_simt(ctx, g, st);
+}
+
+// A (and A^-1) for one attempt into L.A32 / L.X32 or straight into the outputs.
+int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, uint32_t attempt,
+                   int dtype, void* A_out, void* Ainv_out, int lda, float* cond_dev, cudaStream_t st)
+{
+    const int ldi = L.ldi;
+    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st));
+    GELO_TRY(run_householder_qr(ctx, m, L.G, ldi, L.Qraw, L.qr, st));
+    if (kind == GELO_ORTHOGONAL) {
+        GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, dtype, A_out, Ainv_out, lda, st));
+        if (cond_dev) {
+            set_scalar_kernel<<<1, 1, 0, st>>>(cond_dev, 1.0f);
+            GELO_TRY(after_launch(ctx));
+        }
+        return GELO_OK;
+    }
+    // Q0 (signed, fp32) -> A = Q0 + gamma / sqrt(m) * G1 -> stored type -> inverse of the stored A
+    GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, GELO_F32, L.A32, nullptr, ldi, st));
+    const float s = ctx->gamma / sqrtf((float)m);
+    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st));
+    GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st));
+    if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
+    GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
+    GELO_TRY(launch_narrow(ctx, m, L.X32, ldi, dtype, Ainv_out, lda, st));
+    return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st);
+}
+
+int sample_mixing_impl(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, int dtype,
+                       void* A_out, void* Ainv_out, int lda, float* cond_dev, cudaStream_t st)
+{
+    if (kind == GELO_ORTHOGONAL)
+        return sample_attempt(ctx, L, m, kind, seed, 0u, dtype, A_out, Ainv_out, lda, cond_dev, st);
+    for (int attempt = 0; attempt < ctx->max_attempts; ++attempt) {
+        GELO_TRY(sample_attempt(ctx, L, m, kind, seed, (uint32_t)attempt, dtype, A_out, Ainv_out, lda, cond_dev, st));
+        GELO_CUDA_OK(cudaMemcpyAsync(ctx->status_host, ctx->status_dev, kStatusWords * sizeof(int),
+                                     cudaMemcpyDeviceToHost, st));
+        GELO_CUDA_OK(cudaStreamSynchronize(st));
+        if (ctx->status_host[1] == 1) return GELO_OK;
+    }
+    return GELO_ERR_COND;
+}
+
+int mix_impl(gelo_ctx* ctx, const void* A, int lda, const void* H, const void* S, int n, int k, int d,
+             int dtype, void* U, cudaStream_t st)
+{
+    GemmArgs g;
+    g.M = n + k; g.N = d; g.K = n + k;
+    g.A = A; g.lda = lda;
+    g.B = H; g.ldb = d;
+    if (k > 0) { g.B2 = S; g.b_split = n; }
+    g.C[0] = U; g.ldc = d; g.dtype = dtype;
+    return gemm_dispatch(ctx, g, st);
+}
+
+int project_impl(gelo_ctx* ctx, const void* U, const void* W, int m, int d, int p, int dtype, void* Yp,
+                 cudaStream_t st)
+{
+    GemmArgs g;
+    g.M = m; g.N = p; g.K = d;
+    g.A = U; g.lda = d; g.B = W; g.ldb = p;
+    g.C[0] = Yp; g.ldc = p; g.dtype = dtype;
+    return gemm_dispatch(ctx, g, st);
+}
+
+int unmix_impl(gelo_ctx* ctx, const void* Ainv, int lda, const void* Yp, int n, int k, int p, int dtype,
+               void* Q, void* K, void* V, cudaStream_t st)
+{
+    GemmArgs g;
+    g.M = n; g.N = p; g.K = n + k;
+    g.A = Ainv; g.lda = lda; g.B = Yp; g.ldb = p;
+    g.dtype = dtype;
+    if (K || V) { g.nsplit = 3; g.C[0] = Q; g.C[1] = K; g.C[2] = V; g.ldc = p / 3; }
+    else { g.nsplit = 1; g.C[0] = Q; g.ldc = p; }
+    return gemm_dispatch(ctx, g, st);
+}
+
+int check_split(int p, const void* Q, const void* K, const void* V)
+{
+    if (!Q) return GELO_ERR_INVALID;
+    if ((K == nullptr) != (V == nullptr)) return GELO_ERR_INVALID;
+    if (K && (p % 3 != 0 || (p / 3) % 8 != 0)) return GELO_ERR_UNSUPPORTED;
+    return GELO_OK;
+}
+
+int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, int n, int k, int d, int p,
+                 int kind, uint64_t seed, float shield_scale, int dtype, void* Q, void* K, void* V,
+                 cudaStream_t st)
+{
+    const int m = n + k;
+    GELO_TRY(sample_mixing_impl(ctx, L, m, kind, seed, dtype, L.A, L.Ainv, L.ldi, nullptr, st));
+    GELO_TRY(run_shield_rows(ctx, H, n, d, k, shield_scale, seed, dtype, L.S, L.sh, st));
+    GELO_TRY(mix_impl(ctx, L.A, L.ldi, H, k > 0 ? L.S : nullptr, n, k, d, dtype, L.U, st));
+    GELO_TRY(project_impl(ctx, L.U, W, m, d, p, dtype, L.Yp, st));
+    return unmix_impl(ctx, L.Ainv, L.ldi, L.Yp, n, k, p, dtype, Q, K, V, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int gelo_create(gelo_ctx** out, int device)
+{
+    if (!out) return GELO_ERR_INVALID;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess) return GELO_ERR_CUDA;
+    if (device < 0 || device >= count) return GELO_ERR_INVALID;
+    cudaDeviceProp prop;
+    GELO_CUDA_OK(cudaGetDeviceProperties(&prop, device));
+    if (prop.major != 10) return GELO_ERR_UNSUPPORTED;
+    DeviceGuard guard(device);
+    if (!guard.ok) return GELO_ERR_CUDA;
+    gelo_ctx* ctx = new (std::nothrow) gelo_ctx();
+    if (!ctx) return GELO_ERR_CUDA;
+    ctx->device = device;
+    ctx->sm_count = prop.multiProcessorCount;
+    if (cudaMalloc(&ctx->status_dev, kStatusWords * sizeof(int)) != cudaSuccess ||
+        cudaMemset(ctx->status_dev, 0, kStatusWords * sizeof(int)) != cudaSuccess ||
+        cudaHostAlloc(&ctx->status_host, kStatusWords * sizeof(int), cudaHostAllocDefault) != cudaSuccess) {
+        if (ctx->status_dev) cudaFree(ctx->status_dev);
+        delete ctx;
+        return GELO_ERR_CUDA;
+    }
+    cudaDriverEntryPointQueryResult qres;
+    void* fn = nullptr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+        ctx->tmap_encode = fn;
+    *out = ctx;
+    return GELO_OK;
+}
+
+int gelo_destroy(gelo_ctx* ctx)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    cudaFree(ctx->status_dev);
+    cudaFreeHost(ctx->status_host);
+    delete ctx;
+    return GELO_OK;
+}
+
+size_t gelo_workspace_bytes(int n, int k, int d, int p, int dtype)
+{
+    if (n < 0 || k < 0 || d < 0 || p < 0 || bad_dtype(dtype) || n + k <= 0) return 0;
+    Arena a;
+    a.cap = ~size_t(0) >> 1;
+    carve(a, n, k, d, p, dtype, true);
+    return a.off + 256;
+}
+
+int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    if (dev_ws && (reinterpret_cast<uintptr_t>(dev_ws) & 255u)) return GELO_ERR_INVALID;
+    ctx->ws = dev_ws;
+    ctx->ws_bytes = dev_ws ? bytes : 0;
+    return GELO_OK;
+}
+
+int gelo_set_nonorthogonal(gelo_ctx* ctx, float gamma, float cond_bound, int max_attempts)
+{
+    if (!ctx || !(gamma >= 0.0f) || !(cond_bound >= 1.0f) || max_attempts < 1 || max_attempts > 64)
+        return GELO_ERR_INVALID;
+    ctx->gamma = gamma;
+    ctx->cond_bound = cond_bound;
+    ctx->max_attempts = max_attempts;
+    return GELO_OK;
+}
+
+int gelo_mixing_ld(int m) { return m <= 0 ? 0 : round_up(m, 64); }
+
+int gelo_last_status(gelo_ctx* ctx, void* stream)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    cudaStream_t st = as_stream(stream);
+    GELO_CUDA_OK(cudaMemcpyAsync(ctx->status_host, ctx->status_dev, kStatusWords * sizeof(int),
+                                 cudaMemcpyDeviceToHost, st));
+    GELO_CUDA_OK(cudaMemsetAsync(ctx->status_dev, 0, sizeof(int), st));
+    GELO_CUDA_OK(cudaStreamSynchronize(st));
+    return ctx->status_host[0];
+}
+
+long long gelo_launch_count(gelo_ctx* ctx, int reset)
+{
+    if (!ctx) return -1;
+    const long long v = ctx->launches;
+    if (reset) ctx->launches = 0;
+    return v;
+}
+
+const char* gelo_status_string(int s)
+{
+    switch (s) {
+        case GELO_OK: return "ok";
+        case GELO_ERR_INVALID: return "invalid argument";
+        case GELO_ERR_WORKSPACE: return "workspace missing or too small";
+        case GELO_ERR_COND: return "no mixing matrix within the condition-number bound";
+        case GELO_ERR_TIMEOUT: return "a bounded device-side wait ran out";
+        case GELO_ERR_CUDA: return "CUDA call failed";
+        case GELO_ERR_UNSUPPORTED: return "unsupported request";
+        default: return "unknown status";
+    }
+}
+
+int gelo_philox_words(gelo_ctx* ctx, uint64_t seed, uint32_t stream_id, uint32_t attempt, uint64_t first,
+                      uint64_t count, uint32_t* out_dev, void* stream)
+{
+    if (!ctx || (!out_dev && count)) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return launch_philox_words(ctx, seed, stream_id, attempt, first, count, out_dev, as_stream(stream));
+}
+
+int gelo_sample_gaussian(gelo_ctx* ctx, int rows, int cols, int ld, uint64_t seed, uint32_t stream_id,
+                         uint32_t attempt, float scale, float* out_dev, void* stream)
+{
+    if (!ctx || rows < 0 || cols < 0 || ld < cols) return GELO_ERR_INVALID;
+    if (rows == 0 || cols == 0) return GELO_OK;
+    if (!out_dev || misaligned(out_dev)) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return launch_gaussian(ctx, rows, cols, ld, seed, stream_id, attempt, scale, nullptr, out_dev, as_stream(stream));
+}
+
+int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev, float* Qt_dev, void* stream)
+{
+    if (!ctx || m <= 0 || !G_dev || !Q_dev || ld < m) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    if (ld == L.ldi) {
+        GELO_TRY(run_householder_qr(ctx, m, G_dev, ld, L.Qraw, L.qr, st));
+        return launch_finish_mixing(ctx, m, L.Qraw, ld, G_dev, ld, GELO_F32, Q_dev, Qt_dev, ld, st);
+    }
+    GELO_CUDA_OK(cudaMemcpy2DAsync(L.G, (size_t)L.ldi * 4, G_dev, (size_t)ld * 4, (size_t)m * 4, m,
+                                   cudaMemcpyDeviceToDevice, st));
+    GELO_TRY(run_householder_qr(ctx, m, L.G, L.ldi, L.Qraw, L.qr, st));
+    GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, L.ldi, L.G, L.ldi, GELO_F32, Q_dev, Qt_dev, ld, st));
+    return cudaMemcpy2DAsync(G_dev, (size_t)ld * 4, L.G, (size_t)L.ldi * 4, (size_t)m * 4, m,
+                             cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
+}
+
+int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ainv_dev, void* stream)
+{
+    if (!ctx || m <= 0 || !A_dev || !Ainv_dev || ld < m) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    if (ld == L.ldi) return run_lu_inverse(ctx, m, A_dev, ld, Ainv_dev, L.lu, st);
+    GELO_CUDA_OK(cudaMemcpy2DAsync(L.A32, (size_t)L.ldi * 4, A_dev, (size_t)ld * 4, (size_t)m * 4, m,
+                                   cudaMemcpyDeviceToDevice, st));
+    GELO_TRY(run_lu_inverse(ctx, m, L.A32, L.ldi, L.X32, L.lu, st));
+    return cudaMemcpy2DAsync(Ainv_dev, (size_t)ld * 4, L.X32, (size_t)L.ldi * 4, (size_t)m * 4, m,
+                             cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
+}
+
+int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
+                       float* cond_dev, void* stream)
+{
+    if (!ctx || m <= 0 || !A_dev || !Ainv_dev || !cond_dev || ld < m) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
+    return run_cond_estimate(ctx, m, A_dev, Ainv_dev, ld, ctx->cond_bound, cond_dev, L.cond, as_stream(stream));
+}
+
+int gelo_sample_mixing(gelo_ctx* ctx, int m, int kind, uint64_t seed, int dtype, void* A_dev, void* Ainv_dev,
+                       int lda, float* cond_dev, void* stream)
+{
+    if (!ctx || m <= 0 || !A_dev || !Ainv_dev || bad_dtype(dtype) || bad_ld(lda, m) ||
+        (kind != GELO_ORTHOGONAL && kind != GELO_NONORTHOGONAL) || misaligned(A_dev) || misaligned(Ainv_dev))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, m, 0, 0, 0, dtype, false, &L)) return GELO_ERR_WORKSPACE;
+    return sample_mixing_impl(ctx, L, m, kind, seed, dtype, A_dev, Ainv_dev, lda, cond_dev, as_stream(stream));
+}
+
+int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale, uint64_t seed,
+                     int dtype, void* S_dev, void* stream)
+{
+    if (!ctx || n <= 0 || d <= 0 || k < 0 || bad_dtype(dtype) || (d % 8) != 0 || !H_dev || misaligned(H_dev))
+        return GELO_ERR_INVALID;
+    if (k == 0) return GELO_OK;
+    if (!S_dev || misaligned(S_dev)) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    if (!ctx->ws) return GELO_ERR_WORKSPACE;
+    Arena a;
+    a.base = static_cast<char*>(ctx->ws);
+    a.cap = ctx->ws_bytes;
+    ShieldScratch sh = carve_shield(a, n);
+    if (!a.ok) return GELO_ERR_WORKSPACE;
+    return run_shield_rows(ctx, H_dev, n, d, k, scale, seed, dtype, S_dev, sh, as_stream(stream));
+}
+
+int gelo_mix(gelo_ctx* ctx, const void* A_dev, int lda, const void* H_dev, const void* S_dev, int n, int k,
+             int d, int dtype, void* U_dev, void* stream)
+{
+    if (!ctx || n <= 0 || k < 0 || d <= 0 || (d % 8) != 0 || bad_dtype(dtype) || !A_dev || !H_dev || !U_dev ||
+        bad_ld(lda, n + k) || ((k > 0) != (S_dev != nullptr)) || misaligned(A_dev) || misaligned(H_dev) ||
+        misaligned(S_dev) || misaligned(U_dev))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return mix_impl(ctx, A_dev, lda, H_dev, S_dev, n, k, d, dtype, U_dev, as_stream(stream));
+}
+
+int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int d, int p, int dtype,
+                 void* Yp_dev, void* stream)
+{
+    if (!ctx || m <= 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype) || !U_dev ||
+        !W_dev || !Yp_dev || misaligned(U_dev) || misaligned(W_dev) || misaligned(Yp_dev))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return project_impl(ctx, U_dev, W_dev, m, d, p, dtype, Yp_dev, as_stream(stream));
+}
+
+int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev, int n, int k, int p, int dtype,
+               void* Q_dev, void* K_dev, void* V_dev, void* stream)
+{
+    if (!ctx || n <= 0 || k < 0 || p <= 0 || (p % 8) != 0 || bad_dtype(dtype) || !Ainv_dev || !Yp_dev ||
+        bad_ld(lda, n + k) || misaligned(Ainv_dev) || misaligned(Yp_dev) || misaligned(Q_dev) ||
+        misaligned(K_dev) || misaligned(V_dev))
+        return GELO_ERR_INVALID;
+    GELO_TRY(check_split(p, Q_dev, K_dev, V_dev));
+    DeviceGuard guard(ctx->device);
+    return unmix_impl(ctx, Ainv_dev, lda, Yp_dev, n, k, p, dtype, Q_dev, K_dev, V_dev, as_stream(stream));
+}
+
+int gelo_qkv_offload(gelo_ctx* ctx, const void* H_dev, const void* W_dev, int n, int k, int d, int p, int kind,
+                     uint64_t seed, float shield_scale, int dtype, void* Q_dev, void* K_dev, void* V_dev,
+                     void* stream)
+{
+    if (!ctx || n <= 0 || k < 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype) ||
+        !H_dev || !W_dev || (kind != GELO_ORTHOGONAL && kind != GELO_NONORTHOGONAL) || misaligned(H_dev) ||
+        misaligned(W_dev) || misaligned(Q_dev) || misaligned(K_dev) || misaligned(V_dev))
+        return GELO_ERR_INVALID;
+    GELO_TRY(check_split(p, Q_dev, K_dev, V_dev));
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, n, k, d, p, dtype, false, &L)) return GELO_ERR_WORKSPACE;
+    return offload_impl(ctx, L, H_dev, W_dev, n, k, d, p, kind, seed, shield_scale, dtype, Q_dev, K_dev, V_dev,
+                        as_stream(stream));
+}
+
+int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, int n, int k, int d, int p,
+                          int kind, uint64_t seed, float shield_scale, int dtype, void* Q_host, void* K_host,
+                          void* V_host, void* stream)
+{
+    if (!ctx || n <= 0 || k < 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype) ||
+        !H_host || !W_dev || (kind != GELO_ORTHOGONAL && kind != GELO_NONORTHOGONAL) || misaligned(W_dev))
+        return GELO_ERR_INVALID;
+    GELO_TRY(check_split(p, Q_host, K_host, V_host));
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, n, k, d, p, dtype, true, &L)) return GELO_ERR_WORKSPACE;
+    cudaStream_t st = as_stream(stream);
+    const size_t es = elem_size(dtype);
+    GELO_CUDA_OK(cudaMemcpyAsync(L.Hd, H_host, (size_t)n * d * es, cudaMemcpyHostToDevice, st));
+    char* y = static_cast<char*>(L.Yd);
+    const bool split = K_host != nullptr;
+    const size_t third = (size_t)n * (p / 3) * es;
+    GELO_TRY(offload_impl(ctx, L, L.Hd, W_dev, n, k, d, p, kind, seed, shield_scale, dtype, y,
+                          split ? y + third : nullptr, split ? y + 2 * third : nullptr, st));
+    if (split) {
+        GELO_CUDA_OK(cudaMemcpyAsync(Q_host, y, third, cudaMemcpyDeviceToHost, st));
+        GELO_CUDA_OK(cudaMemcpyAsync(K_host, y + third, third, cudaMemcpyDeviceToHost, st));
+        GELO_CUDA_OK(cudaMemcpyAsync(V_host, y + 2 * third, third, cudaMemcpyDeviceToHost, st));
+    } else {
+        GELO_CUDA_OK(cudaMemcpyAsync(Q_host, y, (size_t)n * p * es, cudaMemcpyDeviceToHost, st));
+    }
+    GELO_CUDA_OK(cudaStreamSynchronize(st));
+    return GELO_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,156 @@
+// Shared host-side declarations of the GELO library: context, status block,
+// workspace carving and the internal launchers that the entry points chain.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "../../include/gelo.h"
+
+namespace gelo {
+
+// Panel width of the blocked QR / LU factorisations.
+constexpr int kPanel = 32;
+
+// Device status block (ints).  [0]: first device-side error (gelo_status), sticky until read.
+// [1]: verdict of the last condition-number check (1 = accepted).  [2]: detail word.
+constexpr int kStatusWords = 8;
+
+struct Arena {
+    char* base = nullptr;
+    size_t off = 0;
+    size_t cap = 0;
+    bool ok = true;
+    void* take(size_t bytes) {
+        size_t start = (off + 255) & ~size_t(255);
+        if (start + bytes > cap) { ok = false; off = start + bytes; return nullptr; }
+        off = start + bytes;
+        return base ? base + start : nullptr;
+    }
+};
+
+}  // namespace gelo
+
+struct gelo_ctx {
+    int device = 0;
+    int sm_count = 0;
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    int* status_dev = nullptr;
+    int* status_host = nullptr;   // pinned mirror
+    float gamma = 0.5f;
+    float cond_bound = 100.0f;
+    int max_attempts = 8;
+    long long launches = 0;
+    void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
+};
+
+namespace gelo {
+
+#define GELO_CUDA_OK(expr)                                     \
+    do {                                                       \
+        cudaError_t gelo_e_ = (expr);                          \
+        if (gelo_e_ != cudaSuccess) return GELO_ERR_CUDA;      \
+    } while (0)
+
+#define GELO_TRY(expr)                                         \
+    do {                                                       \
+        int gelo_s_ = (expr);                                  \
+        if (gelo_s_ != GELO_OK) return gelo_s_;                \
+    } while (0)
+
+// Counts a launch and turns a launch error into a status.
+static inline int after_launch(gelo_ctx* ctx) {
+    ctx->launches += 1;
+    return cudaPeekAtLastError() == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
+}
+
+static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
+static inline size_t elem_size(int dtype) { return dtype == GELO_BF16 ? 2 : 4; }
+
+// ---- sampling ---------------------------------------------------------------------
+
+int launch_philox_words(gelo_ctx*, uint64_t seed, uint32_t stream_id, uint32_t attempt,
+                        uint64_t first, uint64_t count, uint32_t* out, cudaStream_t);
+
+// out[i*ld + j] = (base ? base[i*ld + j] : 0) + scale * z(i*cols + j)
+int launch_gaussian(gelo_ctx*, int rows, int cols, int ld, uint64_t seed, uint32_t stream_id,
+                    uint32_t attempt, float scale, const float* base, float* out, cudaStream_t);
+
+// ---- fp32 SIMT GEMM ----------------------------------------------------------------
+
+struct GemmArgs {
+    int M = 0, N = 0, K = 0;
+    const void* A = nullptr; int lda = 0; bool transA = false;   // op(A): M x K
+    const void* B = nullptr; int ldb = 0; bool transB = false;   // op(B): K x N
+    const void* B2 = nullptr; int b_split = 0;                   // rows >= b_split of op(B) come from B2 (not with transB)
+    void* C[3] = {nullptr, nullptr, nullptr}; int ldc = 0;       // column block c / (N / nsplit) selects C[...]
+    int nsplit = 1;
+    float alpha = 1.0f, beta = 0.0f;
+    int dtype = GELO_F32;                                        // storage type of A, B and C
+};
+int launch_gemm_simt(gelo_ctx*, const GemmArgs&, cudaStream_t);
+
+// ---- bf16 tensor-core GEMM (tcgen05 / TMEM / TMA) ------------------------------------
+
+// Same argument meaning as GemmArgs with dtype = GELO_BF16, transA = transB = false,
+// alpha = 1, beta = 0.  Returns GELO_ERR_UNSUPPORTED for shapes it cannot take.
+int launch_gemm_tc(gelo_ctx*, const GemmArgs&, cudaStream_t);
+bool gemm_tc_supports(const GemmArgs&);
+
+// ---- factorizations -------------------------------------------------------------------
+
+struct QrScratch {       // all fp32
+    float* V = nullptr;  // m x ld reflectors (unit diagonal, zeros above), all panels
+    float* T = nullptr;  // ceil(m / kPanel) blocks of kPanel x kPanel
+    float* W1 = nullptr; // kPanel x ld
+    float* W2 = nullptr; // kPanel x ld
+};
+size_t qr_scratch_bytes(int m, int ld);
+QrScratch carve_qr(Arena&, int m, int ld);
+// Factorises R (m x m, stride ld, overwritten; its diagonal holds diag(R) afterwards) and
+// writes the orthogonal factor Q with G = Q R.  The caller flips column j of Q where
+// R_jj < 0 (launch_finish_mixing with sign_diag = R) to reach the unique factor.
+int run_householder_qr(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, cudaStream_t);
+
+struct LuScratch {
+    float* M = nullptr;   // m x ld working copy
+    int* ipiv = nullptr;  // m
+    int* perm = nullptr;  // m
+};
+LuScratch carve_lu(Arena&, int m, int ld);
+int run_lu_inverse(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, cudaStream_t);
+
+struct CondScratch {
+    float* vec = nullptr;     // iterate, image and row-slab partial sums for both operators
+    float* scal = nullptr;    // 16 floats
+};
+CondScratch carve_cond(Arena&, int m);
+// cond_out[0] = estimate; status_dev[1] = (estimate * 1.1 <= bound)
+int run_cond_estimate(gelo_ctx*, int m, const float* A, const float* Ainv, int ld, float bound,
+                      float* cond_out, const CondScratch&, cudaStream_t);
+
+// ---- layout helpers ----------------------------------------------------------------------
+
+// dst (rows x cols, stride ldd, dtype) = colscale-signed copy of src (fp32); dstT = its transpose.
+// sign_diag (optional, fp32 matrix with stride lds): column j is multiplied by sign(sign_diag[j*lds + j]).
+int launch_finish_mixing(gelo_ctx*, int m, const float* src, int lds_src, const float* sign_diag,
+                         int lds_diag, int dtype, void* dst, void* dstT, int ldd, cudaStream_t);
+// dst (fp32, stride ldd) = widen(src (dtype, stride lds)) for an m x m matrix
+int launch_widen(gelo_ctx*, int m, const void* src, int lds, int dtype, float* dst, int ldd, cudaStream_t);
+// dst (dtype) = round(src fp32), m x m
+int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t);
+
+// ---- shields ---------------------------------------------------------------------------------
+
+struct ShieldScratch {
+    float* norms = nullptr;   // n
+    float* med = nullptr;     // 2
+};
+ShieldScratch carve_shield(Arena&, int n);
+int run_shield_rows(gelo_ctx*, const void* H, int n, int d, int k, float scale, uint64_t seed,
+                    int dtype, void* S, const ShieldScratch&, cudaStream_t);
+
+}  // namespace gelo

@@ -1,0 +1,126 @@
+// Shield rows (paper Mitigation 2, Eq. 7-8): k Gaussian rows scaled to a multiple of the
+// median Euclidean row norm of H, appended below the data rows before mixing.
+//   1. row norms of H            -- one HBM pass, one warp per row, 16-byte loads
+//   2. median by rank counting   -- every element counts how many others precede it
+//   3. S = (scale * med / sqrt(d)) * N(0,1) from Philox stream 2
+#include "common.cuh"
+#include "philox.cuh"
+
+namespace gelo {
+
+namespace {
+
+__device__ __forceinline__ float sumsq8(const uint4& q)
+{
+    const __nv_bfloat162* h = reinterpret_cast<const __nv_bfloat162*>(&q);
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __bfloat1622float2(h[i]);
+        s = fmaf(f.x, f.x, s);
+        s = fmaf(f.y, f.y, s);
+    }
+    return s;
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, int n, int d, float* __restrict__ norms)
+{
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    const T* h = H + (size_t)row * d;
+    float s = 0.0f;
+    if (sizeof(T) == 4) {
+        const float4* h4 = reinterpret_cast<const float4*>(h);
+        for (int j = lane; j < d / 4; j += 32) {
+            const float4 v = __ldg(h4 + j);
+            s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); s = fmaf(v.z, v.z, s); s = fmaf(v.w, v.w, s);
+        }
+    } else {
+        const uint4* h8 = reinterpret_cast<const uint4*>(h);
+        for (int j = lane; j < d / 8; j += 32) s += sumsq8(__ldg(h8 + j));
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+    if (lane == 0) norms[row] = sqrtf(s);
+}
+
+// med[0], med[1] = the elements of rank (n-1)/2 and n/2 (ties broken by index).
+__global__ void __launch_bounds__(256) median_rank_kernel(const float* __restrict__ norms, int n, float* __restrict__ med)
+{
+    __shared__ float tile[256];
+    const int i = blockIdx.x * blockDim.x + threadIdx.x;
+    const float mine = (i < n) ? norms[i] : 0.0f;
+    int rank = 0;
+    for (int base = 0; base < n; base += 256) {
+        const int j = base + threadIdx.x;
+        tile[threadIdx.x] = (j < n) ? norms[j] : 0.0f;
+        __syncthreads();
+        const int lim = min(256, n - base);
+        for (int t = 0; t < lim; ++t) {
+            const float o = tile[t];
+            rank += (o < mine || (o == mine && base + t < i)) ? 1 : 0;
+        }
+        __syncthreads();
+    }
+    if (i < n) {
+        if (rank == (n - 1) / 2) med[0] = mine;
+        if (rank == n / 2) med[1] = mine;
+    }
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int k, int d, float scale,
+                                                          const float* __restrict__ med, uint64_t seed)
+{
+    const uint64_t total = (uint64_t)k * d;
+    const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t e0 = q << 2;
+    if (e0 >= total) return;                      // d % 8 == 0, so blocks never straddle the end
+    const float f = scale * (0.5f * (med[0] + med[1])) / sqrtf((float)d);
+    float z[4];
+    gaussian_block(seed, q, GELO_STREAM_SHIELD, 0u, z);
+    if (sizeof(T) == 4) {
+        *reinterpret_cast<float4*>(reinterpret_cast<float*>(S) + e0) = make_float4(f * z[0], f * z[1], f * z[2], f * z[3]);
+    } else {
+        __nv_bfloat162 lo = __floats2bfloat162_rn(f * z[0], f * z[1]);
+        __nv_bfloat162 hi = __floats2bfloat162_rn(f * z[2], f * z[3]);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__nv_bfloat16*>(S) + e0) = pk;
+    }
+}
+
+}  // namespace
+
+ShieldScratch carve_shield(Arena& a, int n)
+{
+    ShieldScratch s;
+    s.norms = static_cast<float*>(a.take((size_t)(n > 0 ? n : 1) * sizeof(float)));
+    s.med = static_cast<float*>(a.take(4 * sizeof(float)));
+    return s;
+}
+
+int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float scale, uint64_t seed,
+                    int dtype, void* S, const ShieldScratch& s, cudaStream_t st)
+{
+    if (k <= 0) return GELO_OK;
+    if (dtype == GELO_BF16)
+        row_norm_kernel<__nv_bfloat16><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(H), n, d, s.norms);
+    else
+        row_norm_kernel<float><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const float*>(H), n, d, s.norms);
+    GELO_TRY(after_launch(ctx));
+    median_rank_kernel<<<ceil_div(n, 256), 256, 0, st>>>(s.norms, n, s.med);
+    GELO_TRY(after_launch(ctx));
+    const uint64_t blocks = ((uint64_t)k * d + 3) / 4;
+    const unsigned grid = (unsigned)((blocks + 255) / 256);
+    if (dtype == GELO_BF16)
+        shield_fill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<__nv_bfloat16*>(S), k, d, scale, s.med, seed);
+    else
+        shield_fill_kernel<float><<<grid, 256, 0, st>>>(static_cast<float*>(S), k, d, scale, s.med, seed);
+    return after_launch(ctx);
+}
+
+}  // namespace gelo
