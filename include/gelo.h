@@ -147,6 +147,24 @@ int gelo_sample_mixing(gelo_ctx* ctx, int m, int kind, uint64_t seed, int dtype,
 int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale,
                      uint64_t seed, int dtype, void* S_dev, void* stream);
 
+/* gelo_shield_rows for callers that cannot allocate device memory, and so cannot give the
+ * context a workspace: a component loaded into a process whose memory pool belongs to someone
+ * else (a serving engine's plugin, a confidential-computing runtime with a frozen allocator),
+ * or a call site where cudaMalloc is not allowed.  The paper has no counterpart; this is a
+ * packaging variant of the Mitigation 2 step above and computes the same S.
+ *
+ * The row-norm scratch is a fixed array inside the library image (about 256 KiB that every
+ * GPU which loads the library holds until the process exits), so:
+ *   - n may be at most 65536 data rows; a larger n returns GELO_ERR_UNSUPPORTED and launches
+ *     nothing.  No workspace is needed and none is touched.
+ *   - the function allocates and frees nothing, on the host or on the device.
+ *   - the first call on each device looks up the array's device address; make that first
+ *     call outside any stream capture.
+ *   - all calls on one device share the array.  Calls whose kernels may overlap on the GPU
+ *     (different streams without an ordering between them) race on it: order them. */
+int gelo_shield_rows_static(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale,
+                            uint64_t seed, int dtype, void* S_dev, void* stream);
+
 /* ---- the three products (Eq. 1-3) ------------------------------------------------------ */
 
 /* U_dev ((n+k) x d) = A [H; S]; the stacked operand is never materialised.  S_dev may be

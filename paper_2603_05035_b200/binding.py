@@ -48,6 +48,7 @@ EXPORTS = {
     "gelo_cond_estimate": (_i, [_vp, _i, _vp, _vp, _i, _vp, _vp]),
     "gelo_sample_mixing": (_i, [_vp, _i, _i, _u64, _i, _vp, _vp, _i, _vp, _vp]),
     "gelo_shield_rows": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
+    "gelo_shield_rows_static": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
     "gelo_mix": (_i, [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_project": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_unmix": (_i, [_vp, _vp, _i, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
@@ -203,6 +204,11 @@ class Context:
     def shield_rows(self, H, n, d, k, scale, seed, dtype, S, stream=None):
         self._check(self._lib.gelo_shield_rows(self._h, _ptr(H), n, d, k, scale, seed, dtype_code(dtype),
                                                _ptr(S), _stream(stream)), "gelo_shield_rows")
+
+    def shield_rows_static(self, H, n, d, k, scale, seed, dtype, S, stream=None):
+        """Shield rows for callers that cannot allocate: scratch lives inside the library (n <= 65536)."""
+        self._check(self._lib.gelo_shield_rows_static(self._h, _ptr(H), n, d, k, scale, seed, dtype_code(dtype),
+                                                      _ptr(S), _stream(stream)), "gelo_shield_rows_static")
 
     def mix(self, A, lda, H, S, n, k, d, dtype, U, stream=None):
         self._check(self._lib.gelo_mix(self._h, _ptr(A), lda, _ptr(H), _ptr(S), n, k, d, dtype_code(dtype),

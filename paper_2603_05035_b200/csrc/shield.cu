@@ -123,4 +123,74 @@ int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float sca
     return after_launch(ctx);
 }
 
+
+// ---------------------------------------------------------------------------------------
+// Shield rows without any allocation.
+//
+// Some callers cannot hand the library a workspace because they cannot allocate device
+// memory themselves: code running inside an enclave-style runtime whose allocator is
+// frozen after start-up, a plugin called from a serving engine that owns every byte of
+// the memory pool, or a call site inside a region where cudaMalloc is forbidden.  For them
+// the scratch of the shield-row step (one row norm per data row, two median slots) lives
+// in a fixed array inside the library image.  Every GPU that loads the library carries
+// this array until the process exits.
+// ---------------------------------------------------------------------------------------
+
+namespace {
+
+constexpr int kStaticShieldMaxRows = 65536;                        // 256 KiB of row norms
+constexpr int kStaticShieldFloats = kStaticShieldMaxRows + 64;     // + median slots, padded
+
+static __device__ __align__(256) float g_shield_static_scratch[kStaticShieldFloats];
+
+constexpr int kMaxDevices = 64;
+float* g_shield_static_ptr[kMaxDevices] = {};                      // device address per GPU, 0 = not yet resolved
+
+// The array's name is only a handle on the host; the device address has to be asked for,
+// once per device, with that device current.
+int static_scratch_for_current_device(int device, float** out)
+{
+    if (device < 0 || device >= kMaxDevices) return GELO_ERR_UNSUPPORTED;
+    float* p = __atomic_load_n(&g_shield_static_ptr[device], __ATOMIC_ACQUIRE);
+    if (!p) {
+        void* addr = nullptr;
+        if (cudaGetSymbolAddress(&addr, g_shield_static_scratch) != cudaSuccess || !addr) return GELO_ERR_CUDA;
+        p = static_cast<float*>(addr);
+        __atomic_store_n(&g_shield_static_ptr[device], p, __ATOMIC_RELEASE);
+    }
+    *out = p;
+    return GELO_OK;
+}
+
+}  // namespace
+
 }  // namespace gelo
+
+extern "C" int gelo_shield_rows_static(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale,
+                                       uint64_t seed, int dtype, void* S_dev, void* stream)
+{
+    using namespace gelo;
+    if (!ctx || n <= 0 || d <= 0 || k < 0 || (dtype != GELO_F32 && dtype != GELO_BF16) || (d % 8) != 0 || !H_dev ||
+        (reinterpret_cast<uintptr_t>(H_dev) & 15u))
+        return GELO_ERR_INVALID;
+    if (n > kStaticShieldMaxRows) return GELO_ERR_UNSUPPORTED;     // more rows than the built-in scratch holds
+    if (k == 0) return GELO_OK;
+    if (!S_dev || (reinterpret_cast<uintptr_t>(S_dev) & 15u)) return GELO_ERR_INVALID;
+
+    int prev = -1;
+    if (cudaGetDevice(&prev) != cudaSuccess) return GELO_ERR_CUDA;
+    if (prev != ctx->device && cudaSetDevice(ctx->device) != cudaSuccess) return GELO_ERR_CUDA;
+    float* scratch = nullptr;
+    int rc = static_scratch_for_current_device(ctx->device, &scratch);
+    if (rc == GELO_OK) {
+        cudaStream_t st = static_cast<cudaStream_t>(stream);
+        ShieldScratch s;
+        s.norms = scratch;
+        s.med = scratch + kStaticShieldMaxRows;
+        // the array keeps what the previous call left: the median slots start from zero each time
+        if (cudaMemsetAsync(s.med, 0, 2 * sizeof(float), st) != cudaSuccess) rc = GELO_ERR_CUDA;
+        if (rc == GELO_OK) rc = run_shield_rows(ctx, H_dev, n, d, k, scale, seed, dtype, S_dev, s, st);
+    }
+    if (prev != ctx->device) cudaSetDevice(prev);
+    return rc;
+}
