@@ -7,6 +7,8 @@
 //       U12 = L11^-1 A12 -> A22 -= L21 U12 (GEMM)
 //   A^-1 = U^-1 L^-1 P by two blocked triangular solves on the permuted identity,
 //   each block step a small substitution kernel plus one GEMM update.
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 
 namespace gelo {
@@ -86,6 +88,153 @@ lu_panel_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, int* __res
         }
         __syncthreads();
     }
+}
+
+// ---- register-resident LU panel on a thread-block cluster ------------------------------------
+//
+// Same elimination, with the panel in registers spread over a cluster (global warp g holds rows
+// j0 + g, j0 + g + CS*32, ...; lane = panel column).  Per column every CTA publishes its best
+// pivot candidate TOGETHER with that row's 32 panel values into every CTA's shared memory, and
+// CTA 0 publishes the current row j; after one cluster barrier all CTAs know the winner (largest
+// magnitude, smallest row on a tie), swap in registers and eliminate without further traffic.
+constexpr int kClusterMax = 8;
+constexpr int kRowsPerThread = 17;
+constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kRowsPerThread;
+
+__global__ void __launch_bounds__(kPanelThreads, 1)
+lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, int* __restrict__ ipiv,
+                        int* __restrict__ status)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+
+    __shared__ float cand_v[kPanelWarps];
+    __shared__ int cand_r[kPanelWarps];
+    __shared__ float win_v[2][kClusterMax];
+    __shared__ int win_r[2][kClusterMax];
+    __shared__ float win_row[2][kClusterMax][NB];
+    __shared__ float rowj_buf[2][NB];
+
+    const int lane = threadIdx.x & 31;
+    const int warp = threadIdx.x >> 5;
+    const int gw = rank * kPanelWarps + warp;
+    const int stride = CS * kPanelWarps;
+    const bool col_ok = lane < jb;
+    const unsigned full = 0xffffffffu;
+
+    float x[kRowsPerThread];
+#pragma unroll
+    for (int i = 0; i < kRowsPerThread; ++i) {
+        const int row = j0 + i * stride + gw;
+        x[i] = (row < m && col_ok) ? M[(size_t)row * ld + j0 + lane] : 0.0f;
+    }
+    if (CS > 1) cluster.sync(); else __syncthreads();
+
+    for (int c = 0; c < jb; ++c) {
+        const int j = j0 + c;
+        const int par = c & 1;
+        // ---- this warp's candidate (same in every lane) ----
+        float bv = -1.0f;
+        int br = 0x7fffffff;
+        float brow = 0.0f;                                  // this lane's entry of the candidate row
+#pragma unroll
+        for (int i = 0; i < kRowsPerThread; ++i) {
+            const int row = j0 + i * stride + gw;
+            const float a = fabsf(__shfl_sync(full, x[i], c));
+            if (row >= j && row < m && a > bv) { bv = a; br = row; brow = x[i]; }   // rows ascend with i
+        }
+        if (lane == 0) { cand_v[warp] = bv; cand_r[warp] = br; }
+        __syncthreads();
+        // ---- this CTA's candidate: every warp reduces the 32 entries the same way ----
+        float cv = cand_v[lane];
+        int cr = cand_r[lane];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            const float ov = __shfl_xor_sync(full, cv, off);
+            const int orow = __shfl_xor_sync(full, cr, off);
+            if (ov > cv || (ov == cv && orow < cr)) { cv = ov; cr = orow; }
+        }
+        if (cr == br && bv >= 0.0f) {                       // this warp owns the CTA's candidate row
+            for (int r = 0; r < CS; ++r) {
+                cluster.map_shared_rank(&win_row[par][rank][lane], r)[0] = brow;
+                if (lane == 0) {
+                    cluster.map_shared_rank(&win_v[par][rank], r)[0] = cv;
+                    cluster.map_shared_rank(&win_r[par][rank], r)[0] = cr;
+                }
+            }
+        } else if (cv < 0.0f && warp == 0) {                // a CTA without rows >= j publishes "nothing"
+            if (lane == 0)
+                for (int r = 0; r < CS; ++r) {
+                    cluster.map_shared_rank(&win_v[par][rank], r)[0] = -1.0f;
+                    cluster.map_shared_rank(&win_r[par][rank], r)[0] = 0x7fffffff;
+                }
+        }
+        if (rank == 0 && warp == c)                          // the warp that holds row j (slot 0)
+            for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&rowj_buf[par][lane], r)[0] = x[0];
+        if (CS > 1) cluster.sync(); else __syncthreads();
+
+        // ---- the winner over the cluster ----
+        float pv = win_v[par][0];
+        int pr = win_r[par][0], pw = 0;
+        for (int r = 1; r < CS; ++r) {
+            const float ov = win_v[par][r];
+            const int orow = win_r[par][r];
+            if (ov > pv || (ov == pv && orow < pr)) { pv = ov; pr = orow; pw = r; }
+        }
+        const float prow = win_row[par][pw][lane];           // pivot row, this lane's column
+        const float oldj = rowj_buf[par][lane];
+        if (rank == 0 && threadIdx.x == 0) {
+            ipiv[j] = pr;
+            if (!(pv > 0.0f)) atomicCAS(status, 0, (int)GELO_ERR_COND);
+        }
+        const float pivot = __shfl_sync(full, prow, c);
+        const float inv = (pivot != 0.0f) ? 1.0f / pivot : 0.0f;
+        // ---- swap in registers, then eliminate below row j ----
+#pragma unroll
+        for (int i = 0; i < kRowsPerThread; ++i) {
+            const int row = j0 + i * stride + gw;
+            if (pr != j) {
+                if (row == j) x[i] = prow;
+                else if (row == pr) x[i] = oldj;
+            }
+            const float l = __shfl_sync(full, x[i], c) * inv;
+            if (row > j && row < m) {
+                if (lane > c) x[i] = fmaf(-l, prow, x[i]);
+                else if (lane == c) x[i] = l;
+            }
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < kRowsPerThread; ++i) {
+        const int row = j0 + i * stride + gw;
+        if (row < m && col_ok) M[(size_t)row * ld + j0 + lane] = x[i];
+    }
+}
+
+int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int* ipiv, cudaStream_t st)
+{
+    const int rows = m - j0;
+    if (rows > kClusterPanelMaxRows) {
+        lu_panel_kernel<<<1, kPanelThreads, 0, st>>>(M, ld, m, j0, jb, ipiv, ctx->status_dev);
+        return after_launch(ctx);
+    }
+    int cs = 1;
+    while (cs < kClusterMax && cs * kPanelWarps * kRowsPerThread < rows) cs *= 2;
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cs, 1, 1);
+    cfg.blockDim = dim3(kPanelThreads, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, lu_panel_cluster_kernel, M, ld, m, j0, jb, ipiv, ctx->status_dev) != cudaSuccess)
+        return GELO_ERR_CUDA;
+    return after_launch(ctx);
 }
 
 // Applies the panel's interchanges (rows j0+c <-> ipiv[j0+c], c = 0..jb-1, in order) to
@@ -192,8 +341,7 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
     const int npanels = ceil_div(m, NB);
     for (int pnl = 0; pnl < npanels; ++pnl) {
         const int j0 = pnl * NB, jb = (m - j0 < NB) ? (m - j0) : NB;
-        lu_panel_kernel<<<1, kPanelThreads, 0, st>>>(M, ld, m, j0, jb, s.ipiv, ctx->status_dev);
-        GELO_TRY(after_launch(ctx));
+        GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
         if (m > jb) {
             swap_rows_kernel<<<ceil_div(m, 256), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, 0, m, j0, j0 + jb);
             GELO_TRY(after_launch(ctx));
