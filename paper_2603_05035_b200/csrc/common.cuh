@@ -102,10 +102,21 @@ bool gemm_tc_supports(const GemmArgs&);
 
 // ---- factorizations -------------------------------------------------------------------
 
+// ---- rank-32 updates of the factorisations (HBM streamers) ---------------------------------
+
+constexpr int kMaxSlabs = 32;   // row slabs of the split V^T C product
+// W (kPanel x nc, stride ldw) = op(T) * (V^T C);  V: nr x kv (stride ldv), C: nr x nc (stride ldc),
+// T: kPanel x kPanel; Wp: kMaxSlabs * kPanel * ldw floats of scratch.
+int launch_vtc(gelo_ctx*, const float* V, int ldv, int kv, const float* C, int ldc, int nr, int nc,
+               const float* T, bool transpose_t, float* Wp, float* W, int ldw, cudaStream_t);
+// C (M x N) -= A (M x K) * B (K x N), K <= kPanel
+int launch_rank_update(gelo_ctx*, const float* A, int lda, const float* B, int ldb, float* C, int ldc,
+                       int M, int N, int K, cudaStream_t);
+
 struct QrScratch {       // all fp32
     float* V = nullptr;  // m x ld reflectors (unit diagonal, zeros above), all panels
     float* T = nullptr;  // ceil(m / kPanel) blocks of kPanel x kPanel
-    float* W1 = nullptr; // kPanel x ld
+    float* Wp = nullptr; // kMaxSlabs x kPanel x ld partial products
     float* W2 = nullptr; // kPanel x ld
 };
 size_t qr_scratch_bytes(int m, int ld);

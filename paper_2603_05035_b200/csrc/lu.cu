@@ -350,13 +350,9 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
         if (nc <= 0) continue;
         tri_solve_block_kernel<false><<<ceil_div(nc, 256), 256, 0, st>>>(M, ld, M, ld, j0, jb, j0 + jb, m);
         GELO_TRY(after_launch(ctx));
-        GemmArgs g;   // A22 -= L21 U12
-        g.M = nc; g.N = nc; g.K = jb;
-        g.A = M + (size_t)(j0 + jb) * ld + j0; g.lda = ld;
-        g.B = M + (size_t)j0 * ld + j0 + jb; g.ldb = ld;
-        g.C[0] = M + (size_t)(j0 + jb) * ld + j0 + jb; g.ldc = ld;
-        g.alpha = -1.0f; g.beta = 1.0f;
-        GELO_TRY(launch_gemm_simt(ctx, g, st));
+        // A22 -= L21 U12
+        GELO_TRY(launch_rank_update(ctx, M + (size_t)(j0 + jb) * ld + j0, ld, M + (size_t)j0 * ld + j0 + jb, ld,
+                                    M + (size_t)(j0 + jb) * ld + j0 + jb, ld, nc, nc, jb, st));
     }
     // ---- X = P, then L Y = P, then U X = Y ----
     const size_t perm_smem = (size_t)m * sizeof(int);
@@ -372,26 +368,17 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
         GELO_TRY(after_launch(ctx));
         const int nr = m - i0 - ib;
         if (nr <= 0) continue;
-        GemmArgs g;   // X[i0+ib:, :] -= L[i0+ib:, i0:i0+ib] X[i0:i0+ib, :]
-        g.M = nr; g.N = m; g.K = ib;
-        g.A = M + (size_t)(i0 + ib) * ld + i0; g.lda = ld;
-        g.B = X + (size_t)i0 * ld; g.ldb = ld;
-        g.C[0] = X + (size_t)(i0 + ib) * ld; g.ldc = ld;
-        g.alpha = -1.0f; g.beta = 1.0f;
-        GELO_TRY(launch_gemm_simt(ctx, g, st));
+        // X[i0+ib:, :] -= L[i0+ib:, i0:i0+ib] X[i0:i0+ib, :]
+        GELO_TRY(launch_rank_update(ctx, M + (size_t)(i0 + ib) * ld + i0, ld, X + (size_t)i0 * ld, ld,
+                                    X + (size_t)(i0 + ib) * ld, ld, nr, m, ib, st));
     }
     for (int pnl = npanels - 1; pnl >= 0; --pnl) {
         const int i0 = pnl * NB, ib = (m - i0 < NB) ? (m - i0) : NB;
         tri_solve_block_kernel<true><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);
         GELO_TRY(after_launch(ctx));
         if (i0 <= 0) continue;
-        GemmArgs g;   // X[0:i0, :] -= U[0:i0, i0:i0+ib] X[i0:i0+ib, :]
-        g.M = i0; g.N = m; g.K = ib;
-        g.A = M + i0; g.lda = ld;
-        g.B = X + (size_t)i0 * ld; g.ldb = ld;
-        g.C[0] = X; g.ldc = ld;
-        g.alpha = -1.0f; g.beta = 1.0f;
-        GELO_TRY(launch_gemm_simt(ctx, g, st));
+        // X[0:i0, :] -= U[0:i0, i0:i0+ib] X[i0:i0+ib, :]
+        GELO_TRY(launch_rank_update(ctx, M + i0, ld, X + (size_t)i0 * ld, ld, X, ld, i0, m, ib, st));
     }
     return GELO_OK;
 }

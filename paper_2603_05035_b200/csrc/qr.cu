@@ -157,16 +157,19 @@ qr_panel_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
 // ---- register-resident panel on a thread-block cluster -----------------------------------
 //
 // The same Householder panel, but the whole panel lives in registers spread over a cluster of
-// CS CTAs (CS * 32 warps; global warp g holds rows j0 + g, j0 + g + CS*32, ...; lane = panel
-// column).  Per column there is ONE reduction: warp partial sums -> shared memory -> one vector
-// per CTA, which every CTA stores into every other CTA's shared memory (distributed shared
-// memory) followed by one cluster barrier.  The lanes that are idle in that reduction (columns
-// already factorised) use it to accumulate V^T v for the triangular factor T, so no separate
-// Gram pass is needed.  All sums run in a fixed order: results are bit-reproducible.
+// CS CTAs (CS * 32 warps; global warp g holds rows j0 + g + i * CS * 32, i = 0 .. RPT-1; lane =
+// panel column).  Per column there is ONE reduction: warp partial sums -> shared memory -> one
+// vector per CTA, which every CTA stores into every other CTA's shared memory (distributed
+// shared memory) followed by one cluster barrier.  Only the first row of a warp can lie on or
+// above the pivot row, so all other rows run branch-free.  The lanes that are idle in the
+// reduction (columns already factorised) carry V^T v for the triangular factor T, gathered
+// during the previous column's update, so no separate Gram pass is needed.  All sums run in a
+// fixed order: results are bit-reproducible.
 constexpr int kClusterMax = 8;
-constexpr int kRowsPerThread = 17;                         // 8 CTAs * 32 warps * 17 rows >= 4352
-constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kRowsPerThread;
+constexpr int kMaxRowsPerThread = 17;                      // 8 CTAs * 32 warps * 17 rows = 4352
+constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kMaxRowsPerThread;
 
+template <int RPT>
 __global__ void __launch_bounds__(kPanelThreads, 1)
 qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
                         float* __restrict__ V, float* __restrict__ T)
@@ -190,42 +193,38 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
     const bool col_ok = lane < jb;
     const unsigned full = 0xffffffffu;
 
-    float x[kRowsPerThread];
+    float x[RPT], xc[RPT];
 #pragma unroll
-    for (int i = 0; i < kRowsPerThread; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
         x[i] = (row < m && col_ok) ? R[(size_t)row * ld + j0 + lane] : 0.0f;
     }
     for (int idx = threadIdx.x; idx < NB * (NB + 1); idx += kPanelThreads) (&gram[0][0])[idx] = 0.0f;
     if (CS > 1) cluster.sync(); else __syncthreads();     // every CTA of the cluster is running before remote stores
 
+    float g = 0.0f;                                        // v_{c-1}^T v_lane, gathered during the previous update
     for (int c = 0; c <= jb; ++c) {
-        const int j = j0 + c;
         const int par = c & 1;
-        const int csrc = c & 31, psrc = (c - 1) & 31;
-        // lanes >= c: x_c^T x_lane over rows > j;   lanes < c-1: v_{c-1}^T v_lane over rows >= j-1
+        const int csrc = c & 31;
+        // ---- lanes >= c: x_c^T x_lane over the rows below the pivot row j = j0 + c ----
         float acc = 0.0f;
 #pragma unroll
-        for (int i = 0; i < kRowsPerThread; ++i) {
-            const int row = j0 + i * stride + gw;
-            const float xc = __shfl_sync(full, x[i], csrc);
-            const float xp = __shfl_sync(full, x[i], psrc);
-            if (lane >= c) {
-                if (row > j) acc = fmaf(xc, x[i], acc);
-            } else if (lane < c - 1) {
-                if (row == j - 1) acc += x[i];
-                else if (row > j - 1) acc = fmaf(xp, x[i], acc);
-            }
+        for (int i = 1; i < RPT; ++i) {
+            xc[i] = __shfl_sync(full, x[i], csrc);
+            acc = fmaf(xc[i], x[i], acc);
         }
-        red[warp][lane] = acc;
+        xc[0] = __shfl_sync(full, x[0], csrc);
+        if (gw > c) acc = fmaf(xc[0], x[0], acc);          // a warp's first row is below row j only past warp c
+        red[warp][lane] = (lane >= c) ? acc : ((lane < c - 1) ? g : 0.0f);
         __syncthreads();
-        if (warp == 0) {
-            float s = 0.0f;
-#pragma unroll 8
-            for (int w = 0; w < kPanelWarps; ++w) s += red[w][lane];
-            for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&slot[par][rank][lane], r)[0] = s;
+        {
+            // warp w sums entry w over the 32 warps (butterfly: fixed order) and lane r ships it to CTA r
+            float s = red[lane][warp];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(full, s, off);
+            if (lane < CS) cluster.map_shared_rank(&slot[par][rank][warp], lane)[0] = s;
         }
-        if (c < jb && rank == 0 && warp == c) {            // the warp that holds row j (its slot 0)
+        if (c < jb && rank == 0 && warp == c) {            // the warp whose first row is row j
             for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&rowbuf[par][lane], r)[0] = x[0];
         }
         if (CS > 1) cluster.sync(); else __syncthreads();
@@ -247,23 +246,30 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
         const float wv = (lane > c && col_ok) ? fmaf(scale, d_own, rj) : 0.0f;
         const float tw = tau * wv;
         if (threadIdx.x == 0) tau_s[c] = tau;
+        // ---- apply H_c; lanes < c gather v_c^T v_lane for T ----
+        g = 0.0f;
 #pragma unroll
-        for (int i = 0; i < kRowsPerThread; ++i) {
-            const int row = j0 + i * stride + gw;
-            const float v = __shfl_sync(full, x[i], c) * scale;
-            if (row == j) {
-                if (lane > c) x[i] -= tw;
-                else if (lane == c) x[i] = beta;
-            } else if (row > j) {
-                if (lane > c) x[i] = fmaf(-tw, v, x[i]);
-                else if (lane == c) x[i] = v;
-            }
+        for (int i = 1; i < RPT; ++i) {
+            const float v = xc[i] * scale;
+            if (lane > c) x[i] = fmaf(-tw, v, x[i]);
+            else if (lane == c) x[i] = v;
+            else g = fmaf(v, x[i], g);
+        }
+        if (gw > c) {
+            const float v = xc[0] * scale;
+            if (lane > c) x[0] = fmaf(-tw, v, x[0]);
+            else if (lane == c) x[0] = v;
+            else g = fmaf(v, x[0], g);
+        } else if (gw == c) {                               // row j itself: v_c(j) = 1
+            if (lane > c) x[0] -= tw;
+            else if (lane == c) x[0] = beta;
+            else g += x[0];
         }
     }
 
     // ---- write back: R above / on the diagonal, reflectors below it ----
 #pragma unroll
-    for (int i = 0; i < kRowsPerThread; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
         if (row < m && col_ok) {
             const int diag = j0 + lane;
@@ -290,16 +296,9 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
     }
 }
 
-// Launches the panel on the smallest cluster whose registers hold the rows.
-int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, float* V, float* T, cudaStream_t st)
+template <int RPT>
+cudaError_t launch_cluster_panel(int cs, cudaStream_t st, float* R, int ld, int m, int j0, int jb, float* V, float* T)
 {
-    const int rows = m - j0;
-    if (rows > kClusterPanelMaxRows) {
-        qr_panel_kernel<<<1, kPanelThreads, 0, st>>>(R, ld, m, j0, jb, V, T);
-        return after_launch(ctx);
-    }
-    int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * kRowsPerThread < rows) cs *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cs, 1, 1);
     cfg.blockDim = dim3(kPanelThreads, 1, 1);
@@ -310,7 +309,31 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
     attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, qr_panel_cluster_kernel, R, ld, m, j0, jb, V, T) != cudaSuccess) return GELO_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, qr_panel_cluster_kernel<RPT>, R, ld, m, j0, jb, V, T);
+}
+
+// Launches the panel on the cluster / rows-per-thread combination that wastes the fewest row slots.
+int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, float* V, float* T, cudaStream_t st)
+{
+    const int rows = m - j0;
+    if (rows > kClusterPanelMaxRows) {
+        qr_panel_kernel<<<1, kPanelThreads, 0, st>>>(R, ld, m, j0, jb, V, T);
+        return after_launch(ctx);
+    }
+    int cs = 1;
+    while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
+    const int rpt = ceil_div(rows, cs * kPanelWarps);
+    cudaError_t e;
+    if (rpt <= 2) e = launch_cluster_panel<2>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 3) e = launch_cluster_panel<3>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 5) e = launch_cluster_panel<5>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 7) e = launch_cluster_panel<7>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 9) e = launch_cluster_panel<9>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 11) e = launch_cluster_panel<11>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 13) e = launch_cluster_panel<13>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 15) e = launch_cluster_panel<15>(cs, st, R, ld, m, j0, jb, V, T);
+    else e = launch_cluster_panel<17>(cs, st, R, ld, m, j0, jb, V, T);
+    if (e != cudaSuccess) return GELO_ERR_CUDA;
     return after_launch(ctx);
 }
 
@@ -338,7 +361,7 @@ QrScratch carve_qr(Arena& a, int m, int ld)
     QrScratch s;
     s.V = static_cast<float*>(a.take((size_t)m * ld * sizeof(float)));
     s.T = static_cast<float*>(a.take((size_t)ceil_div(m, NB) * NB * NB * sizeof(float)));
-    s.W1 = static_cast<float*>(a.take((size_t)NB * ld * sizeof(float)));
+    s.Wp = static_cast<float*>(a.take((size_t)kMaxSlabs * NB * ld * sizeof(float)));
     s.W2 = static_cast<float*>(a.take((size_t)NB * ld * sizeof(float)));
     return s;
 }
@@ -355,18 +378,9 @@ int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const Q
         if (nc <= 0) continue;
         float* C = R + (size_t)j0 * ld + j0 + jb;
         const float* Vp = s.V + (size_t)j0 * ld + j0;
-        GemmArgs g1;   // W1 (jb x nc) = V^T C
-        g1.M = jb; g1.N = nc; g1.K = nr; g1.A = Vp; g1.lda = ld; g1.transA = true;
-        g1.B = C; g1.ldb = ld; g1.C[0] = s.W1; g1.ldc = ld;
-        GELO_TRY(launch_gemm_simt(ctx, g1, st));
-        GemmArgs g2;   // W2 = T^T W1
-        g2.M = jb; g2.N = nc; g2.K = jb; g2.A = Tp; g2.lda = NB; g2.transA = true;
-        g2.B = s.W1; g2.ldb = ld; g2.C[0] = s.W2; g2.ldc = ld;
-        GELO_TRY(launch_gemm_simt(ctx, g2, st));
-        GemmArgs g3;   // C -= V W2
-        g3.M = nr; g3.N = nc; g3.K = jb; g3.A = Vp; g3.lda = ld;
-        g3.B = s.W2; g3.ldb = ld; g3.C[0] = C; g3.ldc = ld; g3.alpha = -1.0f; g3.beta = 1.0f;
-        GELO_TRY(launch_gemm_simt(ctx, g3, st));
+        // C <- (I - V T^T V^T) C :  W2 = T^T (V^T C), then C -= V W2
+        GELO_TRY(launch_vtc(ctx, Vp, ld, jb, C, ld, nr, nc, Tp, true, s.Wp, s.W2, ld, st));
+        GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, nc, jb, st));
     }
     // ---- accumulate Q backwards from the identity ----
     set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
@@ -377,18 +391,9 @@ int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const Q
         const float* Tp = s.T + (size_t)pnl * NB * NB;
         const float* Vp = s.V + (size_t)j0 * ld + j0;
         float* C = Q + (size_t)j0 * ld + j0;
-        GemmArgs g1;   // W1 (jb x nr) = V^T Q[j0:, j0:]
-        g1.M = jb; g1.N = nr; g1.K = nr; g1.A = Vp; g1.lda = ld; g1.transA = true;
-        g1.B = C; g1.ldb = ld; g1.C[0] = s.W1; g1.ldc = ld;
-        GELO_TRY(launch_gemm_simt(ctx, g1, st));
-        GemmArgs g2;   // W2 = T W1
-        g2.M = jb; g2.N = nr; g2.K = jb; g2.A = Tp; g2.lda = NB;
-        g2.B = s.W1; g2.ldb = ld; g2.C[0] = s.W2; g2.ldc = ld;
-        GELO_TRY(launch_gemm_simt(ctx, g2, st));
-        GemmArgs g3;   // Q[j0:, j0:] -= V W2
-        g3.M = nr; g3.N = nr; g3.K = jb; g3.A = Vp; g3.lda = ld;
-        g3.B = s.W2; g3.ldb = ld; g3.C[0] = C; g3.ldc = ld; g3.alpha = -1.0f; g3.beta = 1.0f;
-        GELO_TRY(launch_gemm_simt(ctx, g3, st));
+        // Q[j0:, j0:] <- (I - V T V^T) Q[j0:, j0:]
+        GELO_TRY(launch_vtc(ctx, Vp, ld, jb, C, ld, nr, nr, Tp, false, s.Wp, s.W2, ld, st));
+        GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, nr, jb, st));
     }
     return GELO_OK;
 }
