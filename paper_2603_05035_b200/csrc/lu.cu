@@ -93,14 +93,16 @@ lu_panel_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, int* __res
 // ---- register-resident LU panel on a thread-block cluster ------------------------------------
 //
 // Same elimination, with the panel in registers spread over a cluster (global warp g holds rows
-// j0 + g, j0 + g + CS*32, ...; lane = panel column).  Per column every CTA publishes its best
-// pivot candidate TOGETHER with that row's 32 panel values into every CTA's shared memory, and
-// CTA 0 publishes the current row j; after one cluster barrier all CTAs know the winner (largest
-// magnitude, smallest row on a tie), swap in registers and eliminate without further traffic.
+// j0 + g + i * CS * 32, i = 0 .. RPT-1; lane = panel column).  Per column every CTA publishes its
+// best pivot candidate TOGETHER with that row's 32 panel values into every CTA's shared memory,
+// and CTA 0 publishes the current row j; after one cluster barrier all CTAs know the winner
+// (largest magnitude, smallest row on a tie), swap in registers and eliminate without further
+// traffic.  Only a warp's first row can lie above row j, so the other rows run branch-free.
 constexpr int kClusterMax = 8;
-constexpr int kRowsPerThread = 17;
-constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kRowsPerThread;
+constexpr int kMaxRowsPerThread = 17;
+constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kMaxRowsPerThread;
 
+template <int RPT>
 __global__ void __launch_bounds__(kPanelThreads, 1)
 lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, int* __restrict__ ipiv,
                         int* __restrict__ status)
@@ -124,9 +126,9 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
     const bool col_ok = lane < jb;
     const unsigned full = 0xffffffffu;
 
-    float x[kRowsPerThread];
+    float x[RPT], xc[RPT];
 #pragma unroll
-    for (int i = 0; i < kRowsPerThread; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
         x[i] = (row < m && col_ok) ? M[(size_t)row * ld + j0 + lane] : 0.0f;
     }
@@ -135,16 +137,18 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
     for (int c = 0; c < jb; ++c) {
         const int j = j0 + c;
         const int par = c & 1;
-        // ---- this warp's candidate (same in every lane) ----
+        // ---- this warp's candidate (same in every lane); rows ascend with i, strict > keeps the first ----
         float bv = -1.0f;
-        int br = 0x7fffffff;
-        float brow = 0.0f;                                  // this lane's entry of the candidate row
+        int bi = -1;
+        xc[0] = __shfl_sync(full, x[0], c);
+        if (gw >= c && j0 + gw < m) { bv = fabsf(xc[0]); bi = 0; }
 #pragma unroll
-        for (int i = 0; i < kRowsPerThread; ++i) {
-            const int row = j0 + i * stride + gw;
-            const float a = fabsf(__shfl_sync(full, x[i], c));
-            if (row >= j && row < m && a > bv) { bv = a; br = row; brow = x[i]; }   // rows ascend with i
+        for (int i = 1; i < RPT; ++i) {
+            xc[i] = __shfl_sync(full, x[i], c);
+            const float a = fabsf(xc[i]);
+            if (a > bv && j0 + i * stride + gw < m) { bv = a; bi = i; }
         }
+        const int br = (bi >= 0) ? j0 + bi * stride + gw : 0x7fffffff;
         if (lane == 0) { cand_v[warp] = bv; cand_r[warp] = br; }
         __syncthreads();
         // ---- this CTA's candidate: every warp reduces the 32 entries the same way ----
@@ -156,22 +160,20 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
             const int orow = __shfl_xor_sync(full, cr, off);
             if (ov > cv || (ov == cv && orow < cr)) { cv = ov; cr = orow; }
         }
-        if (cr == br && bv >= 0.0f) {                       // this warp owns the CTA's candidate row
-            for (int r = 0; r < CS; ++r) {
-                cluster.map_shared_rank(&win_row[par][rank][lane], r)[0] = brow;
-                if (lane == 0) {
-                    cluster.map_shared_rank(&win_v[par][rank], r)[0] = cv;
-                    cluster.map_shared_rank(&win_r[par][rank], r)[0] = cr;
-                }
+        if (bi >= 0 && cr == br) {                          // this warp owns the CTA's candidate row
+            float brow = x[0];
+#pragma unroll
+            for (int i = 1; i < RPT; ++i) if (i == bi) brow = x[i];
+            if (lane < CS) {
+                cluster.map_shared_rank(&win_v[par][rank], lane)[0] = cv;
+                cluster.map_shared_rank(&win_r[par][rank], lane)[0] = cr;
             }
-        } else if (cv < 0.0f && warp == 0) {                // a CTA without rows >= j publishes "nothing"
-            if (lane == 0)
-                for (int r = 0; r < CS; ++r) {
-                    cluster.map_shared_rank(&win_v[par][rank], r)[0] = -1.0f;
-                    cluster.map_shared_rank(&win_r[par][rank], r)[0] = 0x7fffffff;
-                }
+            for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&win_row[par][rank][lane], r)[0] = brow;
+        } else if (cv < 0.0f && warp == 0 && lane < CS) {   // a CTA without rows >= j publishes "nothing"
+            cluster.map_shared_rank(&win_v[par][rank], lane)[0] = -1.0f;
+            cluster.map_shared_rank(&win_r[par][rank], lane)[0] = 0x7fffffff;
         }
-        if (rank == 0 && warp == c)                          // the warp that holds row j (slot 0)
+        if (rank == 0 && warp == c)                          // the warp whose first row is row j
             for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&rowj_buf[par][lane], r)[0] = x[0];
         if (CS > 1) cluster.sync(); else __syncthreads();
 
@@ -191,37 +193,41 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
         }
         const float pivot = __shfl_sync(full, prow, c);
         const float inv = (pivot != 0.0f) ? 1.0f / pivot : 0.0f;
-        // ---- swap in registers, then eliminate below row j ----
+        // ---- swap in registers ----
+        if (pr != j) {
+            const int poff = pr - j0;
+            if (poff % stride == gw) {                       // this warp holds row pr: it receives old row j
+                const int pi = poff / stride;
+                const float oc = __shfl_sync(full, oldj, c);
 #pragma unroll
-        for (int i = 0; i < kRowsPerThread; ++i) {
-            const int row = j0 + i * stride + gw;
-            if (pr != j) {
-                if (row == j) x[i] = prow;
-                else if (row == pr) x[i] = oldj;
+                for (int i = 0; i < RPT; ++i) if (i == pi) { x[i] = oldj; xc[i] = oc; }
             }
-            const float l = __shfl_sync(full, x[i], c) * inv;
-            if (row > j && row < m) {
-                if (lane > c) x[i] = fmaf(-l, prow, x[i]);
-                else if (lane == c) x[i] = l;
-            }
+            if (gw == c) x[0] = prow;                        // rank 0, warp c: row j receives the pivot row
+        }
+        // ---- eliminate below row j ----
+#pragma unroll
+        for (int i = 1; i < RPT; ++i) {
+            const float l = xc[i] * inv;
+            if (lane > c) x[i] = fmaf(-l, prow, x[i]);
+            else if (lane == c) x[i] = l;
+        }
+        if (gw > c) {
+            const float l = xc[0] * inv;
+            if (lane > c) x[0] = fmaf(-l, prow, x[0]);
+            else if (lane == c) x[0] = l;
         }
     }
 #pragma unroll
-    for (int i = 0; i < kRowsPerThread; ++i) {
+    for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
         if (row < m && col_ok) M[(size_t)row * ld + j0 + lane] = x[i];
     }
 }
 
-int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int* ipiv, cudaStream_t st)
+template <int RPT>
+cudaError_t launch_cluster_lu_panel(int cs, cudaStream_t st, float* M, int ld, int m, int j0, int jb, int* ipiv,
+                                    int* status)
 {
-    const int rows = m - j0;
-    if (rows > kClusterPanelMaxRows) {
-        lu_panel_kernel<<<1, kPanelThreads, 0, st>>>(M, ld, m, j0, jb, ipiv, ctx->status_dev);
-        return after_launch(ctx);
-    }
-    int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * kRowsPerThread < rows) cs *= 2;
     cudaLaunchConfig_t cfg = {};
     cfg.gridDim = dim3(cs, 1, 1);
     cfg.blockDim = dim3(kPanelThreads, 1, 1);
@@ -232,8 +238,31 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, lu_panel_cluster_kernel, M, ld, m, j0, jb, ipiv, ctx->status_dev) != cudaSuccess)
-        return GELO_ERR_CUDA;
+    return cudaLaunchKernelEx(&cfg, lu_panel_cluster_kernel<RPT>, M, ld, m, j0, jb, ipiv, status);
+}
+
+int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int* ipiv, cudaStream_t st)
+{
+    const int rows = m - j0;
+    if (rows > kClusterPanelMaxRows) {
+        lu_panel_kernel<<<1, kPanelThreads, 0, st>>>(M, ld, m, j0, jb, ipiv, ctx->status_dev);
+        return after_launch(ctx);
+    }
+    int cs = 1;
+    while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
+    const int rpt = ceil_div(rows, cs * kPanelWarps);
+    int* sd = ctx->status_dev;
+    cudaError_t e;
+    if (rpt <= 2) e = launch_cluster_lu_panel<2>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 3) e = launch_cluster_lu_panel<3>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 5) e = launch_cluster_lu_panel<5>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 7) e = launch_cluster_lu_panel<7>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 9) e = launch_cluster_lu_panel<9>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 11) e = launch_cluster_lu_panel<11>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 13) e = launch_cluster_lu_panel<13>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 15) e = launch_cluster_lu_panel<15>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else e = launch_cluster_lu_panel<17>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    if (e != cudaSuccess) return GELO_ERR_CUDA;
     return after_launch(ctx);
 }
 
