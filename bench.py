@@ -181,7 +181,8 @@ def run_ours(args):
     peaks = _peaks()
 
     ctx = gelo.Context(local_rank)
-    ctx.ensure_workspace(n, k, d, p, w.dtype)
+    ctx.set_lanes(args.lanes)
+    ctx.ensure_batch_workspace(n, k, d, p, w.dtype, args.lanes)
     # replicas draw different inputs and mixing seeds
     base = rank * 1000
     Hs, Ws, seeds = [], [], []
@@ -192,10 +193,12 @@ def run_ours(args):
     Q = torch.empty((n, p // 3), device=dev, dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
     checksum = torch.zeros((), device=dev, dtype=torch.float32)
 
+    kinds = [w.kind(c) for c in range(calls)]
+
     def sweep(step):
-        for c in range(calls):
-            ctx.qkv_offload(Hs[c], Ws[c], n, k, d, p, w.kind(c), seeds[c] + 100000 * step, w.shield_scale,
-                            w.dtype, Q, K, V)
+        # one batched call per sweep: the library samples the A of several calls concurrently
+        ctx.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, [s_ + 100000 * step for s_ in seeds], w.shield_scale,
+                              w.dtype, [Q] * calls, [K] * calls, [V] * calls)
 
     def barrier():
         if dist is not None:
@@ -271,14 +274,14 @@ def run_ours(args):
     Hh = [Hs[c % calls].cpu().pin_memory() for c in range(4)]
     Qh = torch.empty((n, p // 3), dtype=td).pin_memory(); Kh = torch.empty_like(Qh).pin_memory()
     Vh = torch.empty_like(Qh).pin_memory()
-    e2e_calls = max(4, min(calls, 8))
-    for c in range(2):
-        ctx.qkv_offload_host(Hh[c % 4], Ws[c % calls], n, k, d, p, w.kind(c), seeds[c % calls], w.shield_scale, w.dtype, Qh, Kh, Vh)
+    e2e_calls = calls
+    Hh_list = [Hh[c % 4] for c in range(calls)]
+    ctx.qkv_offload_batch_host(Hh_list[:4], Ws[:4], n, k, d, p, kinds[:4], seeds[:4], w.shield_scale, w.dtype,
+                               [Qh] * 4, [Kh] * 4, [Vh] * 4)
     barrier()
     t0 = time.perf_counter()
-    for c in range(e2e_calls):
-        ctx.qkv_offload_host(Hh[c % 4], Ws[c % calls], n, k, d, p, w.kind(c), seeds[c % calls] + 7, w.shield_scale, w.dtype,
-                             Qh, Kh, Vh)
+    ctx.qkv_offload_batch_host(Hh_list, Ws, n, k, d, p, kinds, [s_ + 7 for s_ in seeds], w.shield_scale, w.dtype,
+                               [Qh] * calls, [Kh] * calls, [Vh] * calls)
     torch.cuda.synchronize()
     e2e_s = time.perf_counter() - t0
     checksum += Qh.float().abs().mean().to(dev)
@@ -307,6 +310,7 @@ def run_ours(args):
             "config": {"workload": WORKLOAD, "n": n, "k": k, "m": m, "d": d, "p": p, "calls_per_step": calls,
                        "mixing": "alternating orthogonal / non-orthogonal, fresh A per call",
                        "shield_scale": w.shield_scale, "l2": "inputs_larger_than_l2",
+                       "api": "gelo_qkv_offload_batch", "lanes": args.lanes,
                        "replicas": world},
             "clocks": clocks,
             "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": calls * n * d * es,
@@ -342,6 +346,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--lanes", type=int, default=4, help="concurrent sampling lanes of the batched call (1..8)")
     ap.add_argument("--calls", type=int, default=0, help="projection calls per step (default: the workload's 32)")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed sweeps (for profiler launch lists)")

@@ -200,6 +200,42 @@ int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, 
                           int d, int p, int kind, uint64_t seed, float shield_scale, int dtype,
                           void* Q_host, void* K_host, void* V_host, void* stream);
 
+/* ---- batches of independent calls ---------------------------------------------------------- */
+
+/* The same path for `calls` independent batches (for instance the Q/K/V projections of the
+ * layers of one prefill sweep; paper Section 3.2: "a fresh ... matrix A for this batch (never
+ * reused across batches)").  Sampling A needs only the seed, so up to `lanes` calls sample
+ * their mixing pairs concurrently on streams owned by the context while `stream` runs the
+ * shield rows and the three products of earlier calls; results are those of gelo_qkv_offload
+ * with the same (kind, seed) per call.
+ *   H_dev[i] n x d, W_dev[i] d x p, kinds[i], seeds[i]: inputs of call i (host arrays of
+ *   device pointers / values, read before the function returns).
+ *   Q_dev[i], K_dev[i], V_dev[i]: outputs of call i, as in gelo_unmix (K_dev[i] == V_dev[i] ==
+ *   NULL for all i selects unsplit output).  Calls may share output buffers; they are written
+ *   in call order.
+ * Non-orthogonal calls use their first attempt only and never wait for the device: a missed
+ * condition bound is reported by gelo_last_status as GELO_ERR_COND.  Needs a workspace of
+ * gelo_batch_workspace_bytes(..., lanes) bytes.  Work on the lane streams is ordered after
+ * everything already on `stream`, and `stream` ends up ordered after all of it. */
+int gelo_qkv_offload_batch(gelo_ctx* ctx, int calls, const void* const* H_dev, const void* const* W_dev,
+                           int n, int k, int d, int p, const int* kinds, const uint64_t* seeds,
+                           float shield_scale, int dtype, void* const* Q_dev, void* const* K_dev,
+                           void* const* V_dev, void* stream);
+
+/* Same with activations and results in host memory (pinned memory lets the copies overlap the
+ * sampling lanes): H_host[i] is copied in, Q/K/V_host[i] are copied out, and the function returns
+ * after the last copy has completed. */
+int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_host,
+                                const void* const* W_dev, int n, int k, int d, int p, const int* kinds,
+                                const uint64_t* seeds, float shield_scale, int dtype,
+                                void* const* Q_host, void* const* K_host, void* const* V_host,
+                                void* stream);
+
+/* Number of concurrent sampling lanes of the batched calls (1..8, default 4) and the workspace
+ * they need.  0 bytes if an argument is invalid. */
+int gelo_set_lanes(gelo_ctx* ctx, int lanes);
+size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lanes);
+
 #ifdef __cplusplus
 }
 #endif

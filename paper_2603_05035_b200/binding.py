@@ -53,6 +53,10 @@ EXPORTS = {
     "gelo_project": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_unmix": (_i, [_vp, _vp, _i, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_qkv_offload_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_set_lanes": (_i, [_vp, _i]),
+    "gelo_batch_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "gelo_qkv_offload_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
 }
 
@@ -162,6 +166,20 @@ class Context:
             self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
         return need
 
+    def set_lanes(self, lanes: int):
+        self._check(self._lib.gelo_set_lanes(self._h, lanes), "gelo_set_lanes")
+        self.lanes = int(lanes)
+
+    def ensure_batch_workspace(self, n, k, d, p, dtype, lanes=None):
+        """Workspace for the batched entry points with `lanes` concurrent sampling lanes."""
+        lanes = int(lanes if lanes is not None else getattr(self, "lanes", 4))
+        need = int(self._lib.gelo_batch_workspace_bytes(n, k, d, p, dtype_code(dtype), lanes))
+        if need == 0:
+            raise ValueError("invalid sizes")
+        if self._ws is None or self._ws.numel() < need:
+            self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
+        return need
+
     def set_nonorthogonal(self, gamma=0.5, cond_bound=100.0, max_attempts=8):
         self._check(self._lib.gelo_set_nonorthogonal(self._h, gamma, cond_bound, max_attempts),
                     "gelo_set_nonorthogonal")
@@ -226,6 +244,33 @@ class Context:
         self._check(self._lib.gelo_qkv_offload(self._h, _ptr(H), _ptr(W), n, k, d, p, kind, seed, shield_scale,
                                                dtype_code(dtype), _ptr(Q), _ptr(K), _ptr(V), _stream(stream)),
                     "gelo_qkv_offload")
+
+    @staticmethod
+    def _ptr_array(items, count):
+        arr = (ctypes.c_void_p * count)()
+        for i in range(count):
+            arr[i] = _ptr(items[i]) if items is not None else None
+        return arr
+
+    def _batch(self, fn, name, H, W, n, k, d, p, kinds, seeds, shield_scale, dtype, Q, K, V, stream):
+        calls = len(H)
+        if not (len(W) == len(kinds) == len(seeds) == len(Q) == calls):
+            raise ValueError("per-call lists must have one entry per call")
+        kinds_a = (ctypes.c_int * calls)(*[int(x) for x in kinds])
+        seeds_a = (ctypes.c_uint64 * calls)(*[int(x) for x in seeds])
+        self._check(fn(self._h, calls, self._ptr_array(H, calls), self._ptr_array(W, calls), n, k, d, p, kinds_a,
+                       seeds_a, shield_scale, dtype_code(dtype), self._ptr_array(Q, calls),
+                       self._ptr_array(K, calls), self._ptr_array(V, calls), _stream(stream)), name)
+
+    def qkv_offload_batch(self, H, W, n, k, d, p, kinds, seeds, shield_scale, dtype, Q, K=None, V=None, stream=None):
+        """Lists with one entry per call; sampling of different calls runs on concurrent lanes."""
+        self._batch(self._lib.gelo_qkv_offload_batch, "gelo_qkv_offload_batch", H, W, n, k, d, p, kinds, seeds,
+                    shield_scale, dtype, Q, K, V, stream)
+
+    def qkv_offload_batch_host(self, H_host, W, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host=None,
+                               V_host=None, stream=None):
+        self._batch(self._lib.gelo_qkv_offload_batch_host, "gelo_qkv_offload_batch_host", H_host, W, n, k, d, p,
+                    kinds, seeds, shield_scale, dtype, Q_host, K_host, V_host, stream)
 
     def qkv_offload_host(self, H_host, W, n, k, d, p, kind, seed, shield_scale, dtype, Q_host, K_host=None,
                          V_host=None, stream=None):

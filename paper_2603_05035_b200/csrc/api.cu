@@ -96,7 +96,8 @@ int gemm_dispatch(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
 
 // A (and A^-1) for one attempt into L.A32 / L.X32 or straight into the outputs.
 int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, uint32_t attempt,
-                   int dtype, void* A_out, void* Ainv_out, int lda, float* cond_dev, cudaStream_t st)
+                   int dtype, void* A_out, void* Ainv_out, int lda, float* cond_dev, cudaStream_t st,
+                   bool deferred = false)
 {
     const int ldi = L.ldi;
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st));
@@ -117,7 +118,8 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
     GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
     GELO_TRY(launch_narrow(ctx, m, L.X32, ldi, dtype, Ainv_out, lda, st));
-    return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st);
+    return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st,
+                             deferred);
 }
 
 int sample_mixing_impl(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, int dtype,
@@ -189,6 +191,105 @@ int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, i
     return unmix_impl(ctx, L.Ainv, L.ldi, L.Yp, n, k, p, dtype, Q, K, V, st);
 }
 
+
+// The whole path for a batch of independent calls.  Sampling A depends only on the seed, so up to
+// `lanes` calls sample their mixing pairs concurrently on the context's lane streams (each with its
+// own scratch) while the main stream runs shields and the three products of earlier calls.
+//   lane stream:  [wait lane_free] sample A_i, A_i^-1 -> record lane_ready
+//   main stream:  shield rows_i -> [wait lane_ready] mix, project, unmix -> record lane_free
+// Non-orthogonal samples use the first attempt only; a missed condition bound is reported through
+// the status word (GELO_ERR_COND) instead of a resample, because nothing here waits for the device.
+int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const void* const* W, int n, int k, int d,
+                       int p, const int* kinds, const uint64_t* seeds, float shield_scale, int dtype,
+                       void* const* Q, void* const* K, void* const* V, cudaStream_t st, bool host)
+{
+    const int m = n + k;
+    const int D = calls < ctx->lanes ? calls : ctx->lanes;
+    if (!ctx->ws) return GELO_ERR_WORKSPACE;
+    Arena a;
+    a.base = static_cast<char*>(ctx->ws);
+    a.cap = ctx->ws_bytes;
+    Layout L[kMaxLanes];
+    L[0] = carve(a, n, k, d, p, dtype, host);
+    for (int i = 1; i < D; ++i) L[i] = carve(a, n, k, 0, 0, dtype, false);
+    if (!a.ok) return GELO_ERR_WORKSPACE;
+    const size_t es = elem_size(dtype);
+    const bool split = K[0] != nullptr;
+    const size_t third = (size_t)n * (p / 3) * es;
+
+    GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
+    for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaStreamWaitEvent(ctx->lane_stream[l], ctx->batch_start, 0));
+
+    auto enqueue_sample = [&](int i) -> int {
+        const int l = i % D;
+        cudaStream_t ls = ctx->lane_stream[l];
+        if (i >= D) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->lane_free[l], 0));
+        GELO_TRY(sample_attempt(ctx, L[l], m, kinds[i], seeds[i], 0u, dtype, L[l].A, L[l].Ainv, L[l].ldi, nullptr, ls, true));
+        GELO_CUDA_OK(cudaEventRecord(ctx->lane_ready[l], ls));
+        return GELO_OK;
+    };
+
+    for (int i = 0; i < D; ++i) GELO_TRY(enqueue_sample(i));
+    for (int i = 0; i < calls; ++i) {
+        const int l = i % D;
+        const void* Hi = H[i];
+        char* y = static_cast<char*>(L[0].Yd);
+        void *Qi = Q[i], *Ki = split ? K[i] : nullptr, *Vi = split ? V[i] : nullptr;
+        if (host) {
+            GELO_CUDA_OK(cudaMemcpyAsync(L[0].Hd, H[i], (size_t)n * d * es, cudaMemcpyHostToDevice, st));
+            Hi = L[0].Hd;
+            Qi = y; Ki = split ? y + third : nullptr; Vi = split ? y + 2 * third : nullptr;
+        }
+        GELO_TRY(run_shield_rows(ctx, Hi, n, d, k, shield_scale, seeds[i], dtype, L[0].S, L[0].sh, st));
+        GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
+        GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st));
+        GELO_TRY(project_impl(ctx, L[0].U, W[i], m, d, p, dtype, L[0].Yp, st));
+        GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, L[0].Yp, n, k, p, dtype, Qi, Ki, Vi, st));
+        GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
+        if (host) {
+            if (split) {
+                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, third, cudaMemcpyDeviceToHost, st));
+                GELO_CUDA_OK(cudaMemcpyAsync(K[i], y + third, third, cudaMemcpyDeviceToHost, st));
+                GELO_CUDA_OK(cudaMemcpyAsync(V[i], y + 2 * third, third, cudaMemcpyDeviceToHost, st));
+            } else {
+                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, (size_t)n * p * es, cudaMemcpyDeviceToHost, st));
+            }
+        }
+        if (i + D < calls) GELO_TRY(enqueue_sample(i + D));
+    }
+    if (host) GELO_CUDA_OK(cudaStreamSynchronize(st));
+    return GELO_OK;
+}
+
+int check_batch_args(gelo_ctx* ctx, int calls, const void* const* H, const void* const* W, int n, int k, int d, int p,
+                     const int* kinds, const uint64_t* seeds, int dtype, void* const* Q, void* const* K,
+                     void* const* V, bool host)
+{
+    if (!ctx || calls < 0 || n <= 0 || k < 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype))
+        return GELO_ERR_INVALID;
+    if (calls == 0) return GELO_OK;
+    if (!H || !W || !kinds || !seeds || !Q || !K || !V) return GELO_ERR_INVALID;
+    const bool split = K[0] != nullptr;
+    for (int i = 0; i < calls; ++i) {
+        if (!H[i] || !W[i] || misaligned(W[i]) || (kinds[i] != GELO_ORTHOGONAL && kinds[i] != GELO_NONORTHOGONAL))
+            return GELO_ERR_INVALID;
+        if ((K[i] != nullptr) != split) return GELO_ERR_INVALID;
+        if (!host && (misaligned(H[i]) || misaligned(Q[i]) || misaligned(K[i]) || misaligned(V[i])))
+            return GELO_ERR_INVALID;
+        GELO_TRY(check_split(p, Q[i], K[i], V[i]));
+    }
+    return GELO_OK;
+}
+
+size_t batch_workspace(int n, int k, int d, int p, int dtype, int lanes)
+{
+    Arena a;
+    a.cap = ~size_t(0) >> 1;
+    carve(a, n, k, d, p, dtype, true);
+    for (int i = 1; i < lanes; ++i) carve(a, n, k, 0, 0, dtype, false);
+    return a.off + 256;
+}
+
 }  // namespace
 
 extern "C" {
@@ -216,6 +317,12 @@ int gelo_create(gelo_ctx** out, int device)
         delete ctx;
         return GELO_ERR_CUDA;
     }
+    bool lanes_ok = cudaEventCreateWithFlags(&ctx->batch_start, cudaEventDisableTiming) == cudaSuccess;
+    for (int l = 0; l < kMaxLanes && lanes_ok; ++l)
+        lanes_ok = cudaStreamCreateWithFlags(&ctx->lane_stream[l], cudaStreamNonBlocking) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->lane_ready[l], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->lane_free[l], cudaEventDisableTiming) == cudaSuccess;
+    if (!lanes_ok) { gelo_destroy(ctx); return GELO_ERR_CUDA; }
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
     if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
@@ -229,6 +336,12 @@ int gelo_destroy(gelo_ctx* ctx)
 {
     if (!ctx) return GELO_ERR_INVALID;
     DeviceGuard guard(ctx->device);
+    for (int l = 0; l < kMaxLanes; ++l) {
+        if (ctx->lane_stream[l]) { cudaStreamSynchronize(ctx->lane_stream[l]); cudaStreamDestroy(ctx->lane_stream[l]); }
+        if (ctx->lane_ready[l]) cudaEventDestroy(ctx->lane_ready[l]);
+        if (ctx->lane_free[l]) cudaEventDestroy(ctx->lane_free[l]);
+    }
+    if (ctx->batch_start) cudaEventDestroy(ctx->batch_start);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
     delete ctx;
@@ -467,6 +580,41 @@ int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, 
     }
     GELO_CUDA_OK(cudaStreamSynchronize(st));
     return GELO_OK;
+}
+
+size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lanes)
+{
+    if (n < 0 || k < 0 || d < 0 || p < 0 || bad_dtype(dtype) || n + k <= 0 || lanes < 1 || lanes > kMaxLanes) return 0;
+    return batch_workspace(n, k, d, p, dtype, lanes);
+}
+
+int gelo_set_lanes(gelo_ctx* ctx, int lanes)
+{
+    if (!ctx || lanes < 1 || lanes > kMaxLanes) return GELO_ERR_INVALID;
+    ctx->lanes = lanes;
+    return GELO_OK;
+}
+
+int gelo_qkv_offload_batch(gelo_ctx* ctx, int calls, const void* const* H_dev, const void* const* W_dev, int n, int k,
+                           int d, int p, const int* kinds, const uint64_t* seeds, float shield_scale, int dtype,
+                           void* const* Q_dev, void* const* K_dev, void* const* V_dev, void* stream)
+{
+    GELO_TRY(check_batch_args(ctx, calls, H_dev, W_dev, n, k, d, p, kinds, seeds, dtype, Q_dev, K_dev, V_dev, false));
+    if (calls == 0) return GELO_OK;
+    DeviceGuard guard(ctx->device);
+    return offload_batch_impl(ctx, calls, H_dev, W_dev, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_dev, K_dev,
+                              V_dev, as_stream(stream), false);
+}
+
+int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_host, const void* const* W_dev, int n,
+                                int k, int d, int p, const int* kinds, const uint64_t* seeds, float shield_scale,
+                                int dtype, void* const* Q_host, void* const* K_host, void* const* V_host, void* stream)
+{
+    GELO_TRY(check_batch_args(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, dtype, Q_host, K_host, V_host, true));
+    if (calls == 0) return GELO_OK;
+    DeviceGuard guard(ctx->device);
+    return offload_batch_impl(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host,
+                              V_host, as_stream(stream), true);
 }
 
 }  // extern "C"

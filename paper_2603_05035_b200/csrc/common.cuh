@@ -17,6 +17,7 @@ constexpr int kPanel = 32;
 // Device status block (ints).  [0]: first device-side error (gelo_status), sticky until read.
 // [1]: verdict of the last condition-number check (1 = accepted).  [2]: detail word.
 constexpr int kStatusWords = 8;
+constexpr int kMaxLanes = 8;
 
 struct Arena {
     char* base = nullptr;
@@ -45,6 +46,12 @@ struct gelo_ctx {
     int max_attempts = 8;
     long long launches = 0;
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
+    // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
+    int lanes = 4;
+    cudaStream_t lane_stream[gelo::kMaxLanes] = {};
+    cudaEvent_t lane_ready[gelo::kMaxLanes] = {};   // A and A^-1 of the lane are complete
+    cudaEvent_t lane_free[gelo::kMaxLanes] = {};    // the products that read them have been enqueued and finished
+    cudaEvent_t batch_start = nullptr;
 };
 
 namespace gelo {
@@ -141,7 +148,7 @@ struct CondScratch {
 CondScratch carve_cond(Arena&, int m);
 // cond_out[0] = estimate; status_dev[1] = (estimate * 1.1 <= bound)
 int run_cond_estimate(gelo_ctx*, int m, const float* A, const float* Ainv, int ld, float bound,
-                      float* cond_out, const CondScratch&, cudaStream_t);
+                      float* cond_out, const CondScratch&, cudaStream_t, bool deferred = false);
 
 // ---- layout helpers ----------------------------------------------------------------------
 

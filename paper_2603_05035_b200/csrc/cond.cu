@@ -71,11 +71,14 @@ __global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v, int l
     (void)last; (void)bound; (void)cond_out; (void)status;
 }
 
-__global__ void cond_verdict_kernel(CondViews v, float bound, float* cond_out, int* status)
+__global__ void cond_verdict_kernel(CondViews v, float bound, float* cond_out, int* status, int deferred)
 {
     const float c = v.scal[0] * v.scal[1];
     if (cond_out) cond_out[0] = c;
-    status[1] = (c * 1.1f <= bound && c == c) ? 1 : 0;
+    const int ok = (c * 1.1f <= bound && c == c) ? 1 : 0;
+    status[1] = ok;
+    // nobody reads the verdict between attempts in deferred mode: a miss becomes a sticky error
+    if (deferred && !ok) atomicCAS(status, 0, (int)GELO_ERR_COND);
 }
 
 // y = Op xhat, one warp per row
@@ -123,7 +126,7 @@ CondScratch carve_cond(Arena& a, int m)
 }
 
 int run_cond_estimate(gelo_ctx* ctx, int m, const float* A, const float* Ainv, int ld, float bound,
-                      float* cond_out, const CondScratch& s, cudaStream_t st)
+                      float* cond_out, const CondScratch& s, cudaStream_t st, bool deferred)
 {
     CondViews v;
     v.op[0] = A; v.op[1] = Ainv; v.ld = ld; v.m = m; v.mpad = ((m + 63) / 64) * 64;
@@ -146,7 +149,7 @@ int run_cond_estimate(gelo_ctx* ctx, int m, const float* A, const float* Ainv, i
         cond_normalise_kernel<<<2, 1024, 0, st>>>(v, 0, bound, cond_out, ctx->status_dev);
         GELO_TRY(after_launch(ctx));
     }
-    cond_verdict_kernel<<<1, 1, 0, st>>>(v, bound, cond_out, ctx->status_dev);
+    cond_verdict_kernel<<<1, 1, 0, st>>>(v, bound, cond_out, ctx->status_dev, deferred ? 1 : 0);
     return after_launch(ctx);
 }
 

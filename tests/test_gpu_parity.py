@@ -350,3 +350,64 @@ def test_workspace_errors():
     torch.cuda.synchronize()
     assert c.launch_count() > 0 and c.last_status() == binding.OK
     c.close()
+
+
+# ------------------------------------------------------------------------- batched calls
+
+@pytest.mark.parametrize("name,calls,lanes", [("tiny_f32", 6, 4), ("decode_bf16", 5, 2), ("decode_bf16", 3, 8)])
+def test_batched_offload_matches_single_calls(oracle, name, calls, lanes):
+    """Concurrent sampling lanes must not change any result: same bytes as one call at a time."""
+    w = inputs.WORKLOADS[name]
+    n, k, d, p = w.n, w.k, w.d, w.p
+    c = binding.Context(0)
+    c.set_lanes(lanes)
+    c.ensure_batch_workspace(n, k, d, p, w.dtype, lanes)
+    kinds = [ORTHOGONAL if i % 2 == 0 else NONORTHOGONAL for i in range(calls)]
+    Hs, Ws, seeds = [], [], []
+    for i in range(calls):
+        H, W, seed = inputs.make_call_inputs(w, i, "cuda")
+        Hs.append(H); Ws.append(W); seeds.append(seed)
+    td = TDT[w.dtype]
+    mk = lambda: [torch.full((n, p // 3), float("nan"), device="cuda", dtype=td) for _ in range(calls)]
+    Qb, Kb, Vb = mk(), mk(), mk()
+    c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Qb, Kb, Vb)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    for i in range(calls):
+        Q = torch.empty((n, p // 3), device="cuda", dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
+        c.qkv_offload(Hs[i], Ws[i], n, k, d, p, kinds[i], seeds[i], w.shield_scale, w.dtype, Q, K, V)
+        torch.cuda.synchronize()
+        assert torch.equal(Q, Qb[i]) and torch.equal(K, Kb[i]) and torch.equal(V, Vb[i])
+        y = np.hstack([f64(Qb[i]), f64(Kb[i]), f64(Vb[i])])
+        assert oracle.rel_fro(y, oracle.direct(f64(Hs[i]), f64(Ws[i]))) <= TOL[w.dtype]
+    # host variant
+    Hh = [h.cpu().pin_memory() for h in Hs]
+    mkh = lambda: [torch.empty((n, p // 3), dtype=td).pin_memory() for _ in range(calls)]
+    Qh, Kh, Vh = mkh(), mkh(), mkh()
+    c.qkv_offload_batch_host(Hh, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Qh, Kh, Vh)
+    for i in range(calls):
+        assert torch.equal(Qh[i], Qb[i].cpu()) and torch.equal(Vh[i], Vb[i].cpu())
+    assert c.last_status() == binding.OK
+    c.close()
+
+
+def test_batched_offload_full_size(oracle):
+    w = inputs.WORKLOADS["prefill_bf16"]
+    n, k, d, p = w.n, w.k, w.d, w.p
+    calls = 6
+    c = binding.Context(0)
+    c.ensure_batch_workspace(n, k, d, p, w.dtype, 4)
+    Hs, Ws, seeds = [], [], []
+    for i in range(calls):
+        H, W, seed = inputs.make_call_inputs(w, i, "cuda")
+        Hs.append(H); Ws.append(W); seeds.append(seed)
+    kinds = [w.kind(i) for i in range(calls)]
+    outs = [[torch.empty((n, p // 3), device="cuda", dtype=torch.bfloat16) for _ in range(calls)] for _ in range(3)]
+    c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, *outs)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    for i in (0, 3, 5):
+        y = np.hstack([f64(outs[0][i]), f64(outs[1][i]), f64(outs[2][i])])
+        rows = sample_rows(n, 48, seed=i)
+        assert oracle.rel_fro(y[rows], oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)) <= TOL["bf16"]
+    c.close()
