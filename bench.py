@@ -33,6 +33,9 @@ if ROOT not in sys.path:
 METRIC = "obfuscated-QKV tokens/s at Llama-2-7B shapes"
 UNIT = "tokens/s"
 WORKLOAD = "prefill_bf16"
+# DRAM bytes per launch of a kernel class (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture,
+# see profiles/); None until counters have been taken for the current kernel.
+TRAFFIC = {}
 
 
 def _peaks():
@@ -294,15 +297,39 @@ def run_ours(args):
     value = tokens / (ms_max * 1e-3)
     e2e_value = float(n) * e2e_calls * world / (e2e_ms_max * 1e-3)
 
+    # ---- per-launch device times of the main kernel classes (CUDA events on the launching stream):
+    #      one orthogonal and one non-orthogonal call, sampling lanes off so that launches do not overlap ----
+    ctx.set_lanes(1)
+    ctx.profile_start()
+    ctx.qkv_offload_batch(Hs[:2], Ws[:2], n, k, d, p, [gelo.ORTHOGONAL, gelo.NONORTHOGONAL], [s_ + 31 for s_ in seeds[:2]],
+                          w.shield_scale, w.dtype, [Q] * 2, [K] * 2, [V] * 2)
+    prof = ctx.profile_stop()
+    ctx.set_lanes(args.lanes)
+    kernels = {}
+    for name, st_ in prof.items():
+        if st_["launches"] == 0:
+            continue
+        rate = st_["work"] / (st_["ms"] * 1e-3)
+        kernels[name] = {"launches": st_["launches"], "ms": round(st_["ms"], 4),
+                         "avg_us": round(1e3 * st_["ms"] / st_["launches"], 3),
+                         "achieved": rate / (1e12 if st_["unit"] == "flops" else 1e9),
+                         "unit": "TFLOP/s" if st_["unit"] == "flops" else "GB/s"}
+    dominant = max(kernels, key=lambda k_: kernels[k_]["ms"])
+
     if rank == 0:
         es = 2 if w.dtype == "bf16" else 4
-        # dominant product kernel of the chain: the projection GEMM (one launch per call)
-        proj_flops = 2.0 * m * d * p
-        achieved = proj_flops / (stage_ms["project"] * 1e-3) / 1e12
-        roofline = {"kernel": "projection GEMM Y' = U W (one launch per call)", "bound": "tensor",
-                    "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                    "frac": achieved / peaks["bf16_tflops"], "peak_source": peaks["source"] + " (burst bf16 GEMM)",
-                    "traffic": None}
+        dk = kernels[dominant]
+        if dk["unit"] == "TFLOP/s":
+            peak, bound, src = peaks["bf16_tflops"], "tensor", peaks["source"] + " (burst bf16 GEMM)"
+        else:
+            peak, bound, src = peaks["hbm_gbs"], "hbm", peaks["source"] + " (copy bandwidth)"
+        descr = {"rank_update": "rank_update_kernel: C -= A B with 32-column panels in the QR / LU trailing updates",
+                 "vtc": "vtc_partial_kernel: V^T C of the QR trailing updates",
+                 "gemm_tc": "gemm_tc_kernel: tcgen05 bf16 GEMM of mix / project / unmix",
+                 "qr_panel": "qr_panel_cluster_kernel", "lu_panel": "lu_panel_cluster_kernel"}[dominant]
+        roofline = {"kernel": descr, "bound": bound, "achieved": dk["achieved"], "peak": peak, "unit": dk["unit"],
+                    "frac": dk["achieved"] / peak, "peak_source": src, "avg_launch_us": dk["avg_us"],
+                    "launches_timed": dk["launches"], "traffic": TRAFFIC.get(dominant)}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
@@ -317,6 +344,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": calls * n * p * es, "calls_timed": e2e_calls},
             "gpu_launches": launches,
             "roofline": roofline,
+            "kernels": kernels,
             "stage_ms": {k_: round(v, 4) for k_, v in stage_ms.items()},
             "chain": {"ms": chain_ms, "tflops": chain_flops / (chain_ms * 1e-3) / 1e12,
                       "overhead_vs_plain_gemm": chain_ms / stage_ms["plain_project"],

@@ -57,6 +57,8 @@ EXPORTS = {
     "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_lanes": (_i, [_vp, _i]),
     "gelo_batch_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
+    "gelo_profile_start": (_i, [_vp]),
+    "gelo_profile_stop": (_i, [_vp, _vp, _vp]),
     "gelo_qkv_offload_host": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
 }
 
@@ -179,6 +181,20 @@ class Context:
         if self._ws is None or self._ws.numel() < need:
             self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
         return need
+
+    PROFILE_CLASSES = ("rank_update", "vtc", "gemm_tc", "qr_panel", "lu_panel")
+    PROFILE_UNITS = ("bytes", "bytes", "flops", "bytes", "bytes")
+
+    def profile_start(self):
+        self._check(self._lib.gelo_profile_start(self._h), "gelo_profile_start")
+
+    def profile_stop(self, stream=None):
+        """{class: {"launches", "ms", "work", "unit"}} for the launches since profile_start."""
+        out = (ctypes.c_double * 15)()
+        self._check(self._lib.gelo_profile_stop(self._h, _stream(stream), ctypes.cast(out, ctypes.c_void_p)),
+                    "gelo_profile_stop")
+        return {name: {"launches": int(out[3 * i]), "ms": out[3 * i + 1], "work": out[3 * i + 2],
+                       "unit": self.PROFILE_UNITS[i]} for i, name in enumerate(self.PROFILE_CLASSES)}
 
     def set_nonorthogonal(self, gamma=0.5, cond_bound=100.0, max_attempts=8):
         self._check(self._lib.gelo_set_nonorthogonal(self._h, gamma, cond_bound, max_attempts),

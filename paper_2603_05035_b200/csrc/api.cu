@@ -617,4 +617,35 @@ int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_h
                               V_host, as_stream(stream), true);
 }
 
+int gelo_profile_start(gelo_ctx* ctx)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    for (auto& e : ctx->prof) { cudaEventDestroy(e.e0); cudaEventDestroy(e.e1); }
+    ctx->prof.clear();
+    ctx->prof_on = true;
+    return GELO_OK;
+}
+
+int gelo_profile_stop(gelo_ctx* ctx, void* stream, double* out)
+{
+    if (!ctx || !out) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    ctx->prof_on = false;
+    GELO_CUDA_OK(cudaStreamSynchronize(as_stream(stream)));
+    for (int l = 0; l < kMaxLanes; ++l) GELO_CUDA_OK(cudaStreamSynchronize(ctx->lane_stream[l]));
+    for (int i = 0; i < 3 * PROF_CLASSES; ++i) out[i] = 0.0;
+    for (auto& e : ctx->prof) {
+        float ms = 0.0f;
+        if (cudaEventElapsedTime(&ms, e.e0, e.e1) == cudaSuccess && e.cls >= 0 && e.cls < PROF_CLASSES) {
+            out[3 * e.cls + 0] += 1.0;
+            out[3 * e.cls + 1] += ms;
+            out[3 * e.cls + 2] += e.work;
+        }
+        cudaEventDestroy(e.e0);
+        cudaEventDestroy(e.e1);
+    }
+    ctx->prof.clear();
+    return GELO_OK;
+}
+
 }  // extern "C"

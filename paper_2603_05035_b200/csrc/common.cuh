@@ -7,6 +7,8 @@
 #include <stddef.h>
 #include <stdint.h>
 
+#include <vector>
+
 #include "../../include/gelo.h"
 
 namespace gelo {
@@ -18,6 +20,11 @@ constexpr int kPanel = 32;
 // [1]: verdict of the last condition-number check (1 = accepted).  [2]: detail word.
 constexpr int kStatusWords = 8;
 constexpr int kMaxLanes = 8;
+
+// Kernel classes that the optional per-launch timing distinguishes.
+enum ProfClass { PROF_RANK_UPDATE = 0, PROF_VTC = 1, PROF_GEMM_TC = 2, PROF_QR_PANEL = 3, PROF_LU_PANEL = 4,
+                 PROF_CLASSES = 5 };
+struct ProfEntry { int cls; double work; cudaEvent_t e0, e1; };
 
 struct Arena {
     char* base = nullptr;
@@ -52,6 +59,9 @@ struct gelo_ctx {
     cudaEvent_t lane_ready[gelo::kMaxLanes] = {};   // A and A^-1 of the lane are complete
     cudaEvent_t lane_free[gelo::kMaxLanes] = {};    // the products that read them have been enqueued and finished
     cudaEvent_t batch_start = nullptr;
+    // optional per-launch timing (gelo_profile_start / gelo_profile_stop)
+    bool prof_on = false;
+    std::vector<gelo::ProfEntry> prof;
 };
 
 namespace gelo {
@@ -73,6 +83,20 @@ static inline int after_launch(gelo_ctx* ctx) {
     ctx->launches += 1;
     return cudaPeekAtLastError() == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
 }
+
+// Brackets one launch with CUDA events on its stream while per-launch timing is on.
+struct ProfScope {
+    gelo_ctx* ctx; cudaStream_t st; cudaEvent_t e1 = nullptr;
+    ProfScope(gelo_ctx* c, int cls, double work, cudaStream_t s) : ctx(c), st(s) {
+        if (!c->prof_on) return;
+        ProfEntry e; e.cls = cls; e.work = work; e.e0 = nullptr; e.e1 = nullptr;
+        if (cudaEventCreate(&e.e0) != cudaSuccess || cudaEventCreate(&e.e1) != cudaSuccess) return;
+        cudaEventRecord(e.e0, s);
+        e1 = e.e1;
+        c->prof.push_back(e);
+    }
+    ~ProfScope() { if (e1) cudaEventRecord(e1, st); }
+};
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
 static inline size_t elem_size(int dtype) { return dtype == GELO_BF16 ? 2 : 4; }

@@ -387,7 +387,10 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
     p.status = ctx->status_dev;
     const int tiles = ceil_div(g.M, BM) * ceil_div(g.N, BN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, mb2, p);
+    {
+        ProfScope ps(ctx, PROF_GEMM_TC, 2.0 * g.M * (double)g.N * g.K, st);
+        gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, mb2, p);
+    }
     return after_launch(ctx);
 }
 

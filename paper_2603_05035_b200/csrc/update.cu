@@ -285,7 +285,10 @@ int launch_vtc(gelo_ctx* ctx, const float* V, int ldv, int kv, const float* C, i
     const int rows_per_slab = ceil_div(ceil_div(nr, slabs), kVtcRows) * kVtcRows;
     const int used_slabs = ceil_div(nr, rows_per_slab);
     dim3 g1(ceil_div(nc, 128), used_slabs);
+    {
+    ProfScope ps(ctx, PROF_VTC, 4.0 * nr * (double)(nc + kv) + 4.0 * NB * (double)nc * used_slabs, st);
     vtc_partial_kernel<<<g1, 256, kVtcSmemBytes, st>>>(V, ldv, kv, C, ldc, nr, nc, rows_per_slab, Wp, ldw);
+    }
     GELO_TRY(after_launch(ctx));
     w_reduce_kernel<<<ceil_div(nc, 32), 256, 0, st>>>(Wp, ldw, used_slabs, nc, T, transpose_t ? 1 : 0, W);
     return after_launch(ctx);
@@ -297,7 +300,11 @@ int launch_rank_update(gelo_ctx* ctx, const float* A, int lda, const float* B, i
     if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
     if (K > NB) return GELO_ERR_INVALID;
     dim3 grid(ceil_div(N, 128), ceil_div(M, 128));
-    rank_update_kernel<<<grid, 256, 0, st>>>(A, lda, B, ldb, C, ldc, M, N, K);
+    {
+        // algorithmic bytes: C read and written once, A and B read once
+        ProfScope ps(ctx, PROF_RANK_UPDATE, 8.0 * M * (double)N + 4.0 * K * (double)(M + N), st);
+        rank_update_kernel<<<grid, 256, 0, st>>>(A, lda, B, ldb, C, ldc, M, N, K);
+    }
     return after_launch(ctx);
 }
 
