@@ -127,6 +127,14 @@ int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ain
 int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
                        float* cond_dev, void* stream);
 
+/* C_dev (M x N fp32, stride ldc) -= A_dev (M x K fp32, stride lda) * B_dev (K x N fp32, stride ldb), K <= 128:
+ * the level-3 update of the blocked QR / LU, on the tensor cores with every operand held as a bf16
+ * (high, low) pair and the product accumulated as hi*hi + hi*lo + lo*hi in fp32 (relative error of the
+ * product about 1e-5).  ldc must be a multiple of 4 and >= N rounded up to 8; columns N .. that bound are
+ * scratch.  Needs workspace for (max(M, N), 0). */
+int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int lda, const float* B_dev, int ldb,
+                    float* C_dev, int ldc, void* stream);
+
 /* Samples the secret mixing pair for one batch.
  *   GELO_ORTHOGONAL:    A = Q of QR(G0), G0 ~ N(0,1) from stream 0;  A^-1 = A^T.
  *   GELO_NONORTHOGONAL: A = Q0 + gamma * G1 / sqrt(m) (G1 from stream 1), rounded to the

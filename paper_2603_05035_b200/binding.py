@@ -46,6 +46,7 @@ EXPORTS = {
     "gelo_qr_orthogonal": (_i, [_vp, _i, _vp, _i, _vp, _vp, _vp]),
     "gelo_lu_inverse": (_i, [_vp, _i, _vp, _i, _vp, _vp]),
     "gelo_cond_estimate": (_i, [_vp, _i, _vp, _vp, _i, _vp, _vp]),
+    "gelo_update_f32": (_i, [_vp, _i, _i, _i, _vp, _i, _vp, _i, _vp, _i, _vp]),
     "gelo_sample_mixing": (_i, [_vp, _i, _i, _u64, _i, _vp, _vp, _i, _vp, _vp]),
     "gelo_shield_rows": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
     "gelo_shield_rows_static": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
@@ -229,6 +230,10 @@ class Context:
     def cond_estimate(self, m, A, Ainv, ld, cond, stream=None):
         self._check(self._lib.gelo_cond_estimate(self._h, m, _ptr(A), _ptr(Ainv), ld, _ptr(cond),
                                                  _stream(stream)), "gelo_cond_estimate")
+
+    def update_f32(self, M, N, K, A, lda, B, ldb, C, ldc, stream=None):
+        self._check(self._lib.gelo_update_f32(self._h, M, N, K, _ptr(A), lda, _ptr(B), ldb, _ptr(C), ldc,
+                                              _stream(stream)), "gelo_update_f32")
 
     def sample_mixing(self, m, kind, seed, dtype, A, Ainv, lda, cond=None, stream=None):
         self._check(self._lib.gelo_sample_mixing(self._h, m, kind, seed, dtype_code(dtype), _ptr(A), _ptr(Ainv),

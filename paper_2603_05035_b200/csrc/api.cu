@@ -23,6 +23,7 @@ struct Layout {
     QrScratch qr;
     LuScratch lu;
     CondScratch cond;
+    TcScratch tc;
     ShieldScratch sh;
     float* cond_val = nullptr;
     void* A = nullptr;        // m x ldi, path dtype
@@ -48,6 +49,7 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     L.qr = carve_qr(a, L.m, L.ldi);
     L.lu = carve_lu(a, L.m, L.ldi);
     L.cond = carve_cond(a, L.m);
+    L.tc = carve_tc(a, L.m, L.ldi);
     L.sh = carve_shield(a, n);
     L.cond_val = static_cast<float*>(a.take(16));
     L.A = a.take(mat * es);
@@ -646,6 +648,18 @@ int gelo_profile_stop(gelo_ctx* ctx, void* stream, double* out)
     }
     ctx->prof.clear();
     return GELO_OK;
+}
+
+int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int lda, const float* B_dev, int ldb,
+                    float* C_dev, int ldc, void* stream)
+{
+    if (!ctx || M <= 0 || N <= 0 || K <= 0 || K > kOuter || !A_dev || !B_dev || !C_dev || lda < K || ldb < N ||
+        ldc < ((N + 7) & ~7) || (ldc % 4) != 0 || misaligned(C_dev))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    Layout L;
+    if (!carve_ctx(ctx, M > N ? M : N, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
+    return tc_update_f32(ctx, L.tc, M, N, K, A_dev, lda, B_dev, ldb, C_dev, ldc, as_stream(stream));
 }
 
 }  // extern "C"

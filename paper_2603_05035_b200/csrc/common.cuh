@@ -130,6 +130,10 @@ int launch_gemm_simt(gelo_ctx*, const GemmArgs&, cudaStream_t);
 // alpha = 1, beta = 0.  Returns GELO_ERR_UNSUPPORTED for shapes it cannot take.
 int launch_gemm_tc(gelo_ctx*, const GemmArgs&, cudaStream_t);
 bool gemm_tc_supports(const GemmArgs&);
+// Split-precision product on the tensor cores (operands as bf16 high / low pairs); see gemm_tc.cu.
+int launch_gemm_tc_split(gelo_ctx*, int M, int N, int K, const void* Ahi, const void* Alo, int lda,
+                         const void* Bhi, const void* Blo, int ldb, float* sub_from, int ldc, void* emit_hi,
+                         void* emit_lo, int lde, bool narrow_tiles, cudaStream_t);
 
 // ---- factorizations -------------------------------------------------------------------
 
@@ -184,6 +188,28 @@ int launch_finish_mixing(gelo_ctx*, int m, const float* src, int lds_src, const 
 int launch_widen(gelo_ctx*, int m, const void* src, int lds, int dtype, float* dst, int ldd, cudaStream_t);
 // dst (dtype) = round(src fp32), m x m
 int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t);
+
+// (hi, lo) bf16 pair of an fp32 block, optionally transposed (output is cols x rows then)
+int launch_split(gelo_ctx*, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
+                 bool transpose, cudaStream_t);
+
+// Scratch of the tensor-core level-3 updates (outer blocks of kOuter columns).
+constexpr int kOuter = 128;
+struct TcScratch {
+    void* panA[2] = {nullptr, nullptr};    // m x kOuter          block column (V or L), hi / lo
+    void* panAt[2] = {nullptr, nullptr};   // kOuter x ld         its transpose
+    void* rowB[2] = {nullptr, nullptr};    // kOuter x ld         block row (W, U12 or X rows)
+    void* rowB2[2] = {nullptr, nullptr};   // kOuter x ld
+    void* tt[2] = {nullptr, nullptr};      // kOuter x kOuter     triangular factor (transposed or not)
+    void* big[2] = {nullptr, nullptr};     // m x ld              trailing matrix as a pair
+    float* t128 = nullptr;                 // kOuter x kOuter fp32
+    float* gram = nullptr;                 // kOuter x kOuter fp32
+    float* wf32 = nullptr;                 // kOuter x ld fp32
+};
+TcScratch carve_tc(Arena&, int m, int ld);
+// C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores in split precision
+int tc_update_f32(gelo_ctx*, const TcScratch&, int M, int N, int K, const float* A, int lda, const float* B, int ldb,
+                  float* C, int ldc, cudaStream_t);
 
 // ---- shields ---------------------------------------------------------------------------------
 

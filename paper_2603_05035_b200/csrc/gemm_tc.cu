@@ -1,19 +1,23 @@
-// bf16 tensor-core GEMM for the three products of the offload (Eq. 1-3) on sm_100a:
-// tcgen05.mma with the accumulator in tensor memory, operands staged in shared memory by
-// TMA, fp32 accumulation, bf16 (or fp32) output.
+// bf16 tensor-core GEMM on sm_100a: tcgen05.mma with the accumulator in tensor memory, operands
+// staged in shared memory by TMA, fp32 accumulation.  It serves
+//   * the three products of the offload (Eq. 1-3): C = A B with bf16 operands and bf16 output,
+//     the B operand optionally the stack [H; S] of Eq. 8, the output optionally split Q | K | V;
+//   * the level-3 updates of the blocked QR / LU behind the sampling of A: fp32 matrices are held
+//     as a bf16 (high, low) pair and the product is accumulated as hi*hi + hi*lo + lo*hi in fp32,
+//     with an epilogue that either subtracts the result from an fp32 matrix in place or writes it
+//     as a new (high, low) pair.
 //
-//   C (M x N) = A (M x K, row-major, K contiguous)  *  B (K x N, row-major, N contiguous)
+//   C (M x N)  (+)=  sum over segments s of  A_s (M x K_s, row-major)  *  B_s (K_s x N, row-major)
 //
-// * A tiles (128 rows x 64 k) land K-major, B tiles (64 k x 256 columns, as four 64-column
-//   boxes) land N-major; both use the 128-byte swizzle that TMA writes and the MMA reads.
-// * The K loop may run over two stacked B matrices (H then the shield rows S, Eq. 8): the
-//   producer simply switches tensor maps; a block that straddles the seam is issued once per
-//   map and TMA's out-of-bounds zero fill removes the rows that belong to the other matrix.
-// * Ragged M, N, K are handled by the same zero fill on loads and by guarded stores.
-// * The epilogue routes column blocks to up to three outputs (Q | K | V) and casts.
-// * Persistent CTAs (one per SM), warp-specialised: warp 0 issues TMA, warp 1 issues MMA and
-//   owns the tensor-memory allocation, warps 2-5 drain the accumulator.  Two accumulator
-//   stages (2 x 256 columns) let the epilogue of one tile overlap the main loop of the next.
+// * A tiles (128 rows x 64 k) land K-major, B tiles (64 k x BN columns, as 64-column boxes) land
+//   N-major; both use the 128-byte swizzle that TMA writes and the MMA reads.
+// * A segment names one A tensor map, one B tensor map and a starting k for each; the stacked
+//   operand of the mixing product is two segments, a split-precision product is three.  TMA's
+//   out-of-bounds zero fill handles every ragged edge (including a seam inside a k-block).
+// * Persistent CTAs (one per SM), warp-specialised: warp 0 issues TMA, warp 1 issues MMA and owns
+//   the tensor-memory allocation, warps 2-9 drain the accumulator (two warps per TMEM lane
+//   quarter, half of the columns each).  Two accumulator stages let the epilogue of one tile
+//   overlap the main loop of the next.
 // * Every wait on an mbarrier is bounded; on expiry the CTA records GELO_ERR_TIMEOUT in the
 //   context's status word, stops issuing work, releases tensor memory and returns.
 #include <cuda.h>
@@ -25,28 +29,27 @@ namespace gelo {
 namespace {
 
 constexpr int BM = 128;
-constexpr int BN = 256;
 constexpr int BK = 64;
 constexpr int kStages = 4;
 constexpr int kAccStages = 2;
-constexpr int kThreads = 192;
+constexpr int kEpiWarps = 8;
+constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kABytes = BM * BK * 2;            // 16 KiB
 constexpr uint32_t kBBoxBytes = 64 * BK * 2;         // 8 KiB per 64-column box
-constexpr uint32_t kBBytes = (BN / 64) * kBBoxBytes; // 32 KiB
-constexpr uint32_t kStageBytes = kABytes + kBBytes;
-constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t kTmemCols = 512;
 constexpr unsigned long long kWaitLimit = 40ull * 1000 * 1000;   // try_wait rounds before giving up
 
+enum TcMode { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_SUB_F32 = 2, TC_EMIT_SPLIT = 3 };
+
+struct TcSegment { int a_sel, b_sel, a_k0, b_row0, kb; };
+
 struct TcParams {
     int M, N;
-    int kb_first;        // k-blocks read through map B (rows 0 .. b_split-1 of the stacked operand)
-    int kb_second;       // k-blocks read through map B2
-    int a_k0_second;     // A column of the first k-block of the second part (multiple of 8)
-    int b_row0_second;   // row of B2 that meets that column (may be negative: zero filled)
-    void* C0; void* C1; void* C2;
-    int ldc, csplit;
-    int out_f32;         // 1: fp32 output, 0: bf16
+    int nseg;
+    TcSegment seg[3];
+    int mode;
+    void* C0; void* C1; void* C2;   // STORE_*: column-split outputs; SUB_F32: C0 fp32, C1/C2 optional hi/lo; EMIT_SPLIT: C0 hi, C1 lo
+    int ldc, csplit, lde;           // lde: row stride of the hi/lo matrices written next to an fp32 C
     int* status;
 };
 
@@ -138,28 +141,81 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     return d;
 }
 
-// Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = BN.
-constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
-                                ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+
+template <int BN>
+struct TcCfg {
+    static constexpr uint32_t kBBytes = (BN / 64) * kBBoxBytes;
+    static constexpr uint32_t kStageBytes = kABytes + kBBytes;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    // Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = BN.
+    static constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+                                           ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+};
 
 __device__ __forceinline__ uint32_t pack_bf16(uint32_t a, uint32_t b)
 {
     __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
     return *reinterpret_cast<uint32_t*>(&h);
 }
-
-// ---- the kernel ------------------------------------------------------------------------------
-
-__global__ void __launch_bounds__(kThreads, 1)
-gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-               const __grid_constant__ CUtensorMap map_b2, const TcParams prm)
+__device__ __forceinline__ uint32_t pack_bf16f(float a, float b)
 {
+    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    return *reinterpret_cast<uint32_t*>(&h);
+}
+// x = hi + lo with hi = bf16(x), lo = bf16(x - hi)
+__device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo)
+{
+    const __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
+    const float2 hf = __bfloat1622float2(h);
+    const __nv_bfloat162 l = __floats2bfloat162_rn(a - hf.x, b - hf.y);
+    hi = *reinterpret_cast<const uint32_t*>(&h);
+    lo = *reinterpret_cast<const uint32_t*>(&l);
+}
+
+// One 8-column group of the epilogue: w[G*8 .. G*8+7] are the fp32 accumulator values of row gm, columns
+// gn..gn+7 (G is a template parameter so that the register array is indexed by constants only).
+template <int G>
+__device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int gn, const uint32_t (&w)[32])
+{
+    const uint32_t v[8] = {w[G * 8 + 0], w[G * 8 + 1], w[G * 8 + 2], w[G * 8 + 3],
+                           w[G * 8 + 4], w[G * 8 + 5], w[G * 8 + 6], w[G * 8 + 7]};
+    if (prm.mode == TC_STORE_BF16) {
+        const int chunk = gn / prm.csplit;
+        void* base = chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2);
+        const size_t off = (size_t)gm * prm.ldc + (gn - chunk * prm.csplit);
+        uint4 pk;
+        pk.x = pack_bf16(v[0], v[1]); pk.y = pack_bf16(v[2], v[3]);
+        pk.z = pack_bf16(v[4], v[5]); pk.w = pack_bf16(v[6], v[7]);
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
+    } else if (prm.mode == TC_STORE_F32) {
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)gm * prm.ldc + gn);
+        dst[0] = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
+        dst[1] = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
+    } else if (prm.mode == TC_EMIT_SPLIT) {
+        uint4 hi, lo;
+        split2(__uint_as_float(v[0]), __uint_as_float(v[1]), hi.x, lo.x);
+        split2(__uint_as_float(v[2]), __uint_as_float(v[3]), hi.y, lo.y);
+        split2(__uint_as_float(v[4]), __uint_as_float(v[5]), hi.z, lo.z);
+        split2(__uint_as_float(v[6]), __uint_as_float(v[7]), hi.w, lo.w);
+        const size_t off = (size_t)gm * prm.ldc + gn;
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(prm.C0) + off) = hi;
+        *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(prm.C1) + off) = lo;
+    }
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kThreads, 1)
+gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
+               const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
+               const TcParams prm)
+{
+    using Cfg = TcCfg<BN>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-byte alignment
     uint8_t* gen_base = smem_raw + (tiles_base - raw);
-    const uint32_t bar_base = tiles_base + kStages * kStageBytes;
-    uint8_t* bar_gen = gen_base + kStages * kStageBytes;
+    const uint32_t bar_base = tiles_base + kStages * Cfg::kStageBytes;
+    uint8_t* bar_gen = gen_base + kStages * Cfg::kStageBytes;
     // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2]; then tmem slot, abort
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
@@ -174,11 +230,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     const int m_tiles = (prm.M + BM - 1) / BM;
     const int n_tiles = (prm.N + BN - 1) / BN;
     const int total_tiles = m_tiles * n_tiles;
-    const int kb_total = prm.kb_first + prm.kb_second;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        for (int a = 0; a < kAccStages; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), 4); }
+        for (int a = 0; a < kAccStages; ++a) { mbar_init(acc_full_bar(a), 1); mbar_init(acc_empty_bar(a), kEpiWarps); }
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -201,21 +256,24 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
                 const int m0 = (tile % m_tiles) * BM;
                 const int n0 = (tile / m_tiles) * BN;
-                for (int kb = 0; kb < kb_total; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
-                    const bool second = kb >= prm.kb_first;
-                    const int a_k = second ? prm.a_k0_second + (kb - prm.kb_first) * BK : kb * BK;
-                    const int b_row = second ? prm.b_row0_second + (kb - prm.kb_first) * BK : kb * BK;
-                    const CUtensorMap* mb = second ? &map_b2 : &map_b;
-                    const uint32_t sa = tiles_base + s * kStageBytes;
-                    const uint32_t sb = sa + kABytes;
-                    mbar_expect_tx(full_bar(s), kStageBytes);
-                    tma_load_2d(sa, &map_a, a_k, m0, full_bar(s));
 #pragma unroll
-                    for (int j = 0; j < BN / 64; ++j)
-                        tma_load_2d(sb + j * kBBoxBytes, mb, n0 + j * 64, b_row, full_bar(s));
+                for (int sg = 0; sg < 3; ++sg) {              // constant indices keep the parameters out of local memory
+                    if (sg >= prm.nseg || !ok) break;
+                    const TcSegment seg = prm.seg[sg];
+                    const CUtensorMap* ma = seg.a_sel ? &map_a1 : &map_a0;
+                    const CUtensorMap* mb = seg.b_sel ? &map_b1 : &map_b0;
+                    for (int kb = 0; kb < seg.kb; ++kb, ++it) {
+                        const int s = it % kStages;
+                        const uint32_t ph = (it / kStages) & 1u;
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                        const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
+                        const uint32_t sb = sa + kABytes;
+                        mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
+                        tma_load_2d(sa, ma, seg.a_k0 + kb * BK, m0, full_bar(s));
+#pragma unroll
+                        for (int j = 0; j < BN / 64; ++j)
+                            tma_load_2d(sb + j * kBBoxBytes, mb, n0 + j * 64, seg.b_row0 + kb * BK, full_bar(s));
+                    }
                 }
             }
             if (!ok) { *abort_flag = 1; atomicCAS(prm.status, 0, (int)GELO_ERR_TIMEOUT); }
@@ -223,6 +281,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
+            int kb_total = 0;
+#pragma unroll
+            for (int sg = 0; sg < 3; ++sg)
+                if (sg < prm.nseg) kb_total += prm.seg[sg].kb;
             uint32_t it = 0, acc_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
@@ -236,7 +298,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                     const uint32_t ph = (it / kStages) & 1u;
                     if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
                     tc_fence_after();
-                    const uint32_t sa = tiles_base + s * kStageBytes;
+                    const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                     const uint32_t sb = sa + kABytes;
 #pragma unroll
                     for (int ks = 0; ks < BK / 16; ++ks) {
@@ -244,7 +306,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
                         const uint64_t da = smem_desc(sa + ks * 32, 16, 1024);
                         // B: N-major, 64-column boxes 8192 bytes apart, 8-row k groups 1024 bytes apart
                         const uint64_t db = smem_desc(sb + ks * 2048, kBBoxBytes, 1024);
-                        tc_mma_bf16(tmem_d, da, db, kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
+                        tc_mma_bf16(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
                     }
                     tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
                 }
@@ -254,8 +316,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             if (!ok) { *abort_flag = 1; atomicCAS(prm.status, 0, (int)GELO_ERR_TIMEOUT); }
         }
     } else {
-        // ================= epilogue (warps 2..5) =================
+        // ================= epilogue (warps 2..9) =================
         const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
+        const int half = (warp - 2) >> 2;             // which half of the tile's columns
+        constexpr int kHalfCols = BN / 2;
         uint32_t acc_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
@@ -263,38 +327,68 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant_
             const uint32_t aph = (acc_it / kAccStages) & 1u;
             const int m0 = (tile % m_tiles) * BM;
             const int n0 = (tile / m_tiles) * BN;
-            if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
-            tc_fence_after();
             const int gm = m0 + quarter * 32 + lane;
-            const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
+            const bool row_ok = gm < prm.M;
+            if (prm.mode == TC_SUB_F32) {
+                // C -= acc in place, 32 columns at a time; the C values are requested before the wait on
+                // the accumulator so that their latency overlaps the main loop
+                float* crow = static_cast<float*>(prm.C0) + (size_t)gm * prm.ldc;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
+                bool waited = false;
 #pragma unroll 1
-            for (int c = 0; c < BN; c += 32) {
-                uint32_t v[32];
-                tc_ld_32cols(taddr + c, v);
-                tc_ld_wait();
-                if (gm < prm.M) {
+                for (int c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32) {
+                    float4 cv[8];
 #pragma unroll
-                    for (int g = 0; g < 4; ++g) {
-                        const int gn = n0 + c + g * 8;
-                        if (gn < prm.N) {
-                            const int chunk = gn / prm.csplit;
-                            void* base = chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2);
-                            const size_t off = (size_t)gm * prm.ldc + (gn - chunk * prm.csplit);
-                            if (prm.out_f32) {
-                                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(base) + off);
-                                dst[0] = make_float4(__uint_as_float(v[g * 8 + 0]), __uint_as_float(v[g * 8 + 1]),
-                                                     __uint_as_float(v[g * 8 + 2]), __uint_as_float(v[g * 8 + 3]));
-                                dst[1] = make_float4(__uint_as_float(v[g * 8 + 4]), __uint_as_float(v[g * 8 + 5]),
-                                                     __uint_as_float(v[g * 8 + 6]), __uint_as_float(v[g * 8 + 7]));
-                            } else {
-                                uint4 pk;
-                                pk.x = pack_bf16(v[g * 8 + 0], v[g * 8 + 1]);
-                                pk.y = pack_bf16(v[g * 8 + 2], v[g * 8 + 3]);
-                                pk.z = pack_bf16(v[g * 8 + 4], v[g * 8 + 5]);
-                                pk.w = pack_bf16(v[g * 8 + 6], v[g * 8 + 7]);
-                                *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
+                    for (int g = 0; g < 8; ++g) {
+                        const int gn = n0 + c + g * 4;
+                        cv[g] = (row_ok && gn < prm.N) ? *reinterpret_cast<const float4*>(crow + gn)
+                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+                    if (!waited) {
+                        if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
+                        tc_fence_after();
+                        waited = true;
+                    }
+                    uint32_t v[32];
+                    tc_ld_32cols(taddr + c, v);
+                    tc_ld_wait();
+                    if (row_ok) {
+#pragma unroll
+                        for (int g = 0; g < 8; ++g) {
+                            const int gn = n0 + c + g * 4;
+                            if (gn < prm.N) {
+                                float4 r = cv[g];
+                                r.x -= __uint_as_float(v[4 * g + 0]); r.y -= __uint_as_float(v[4 * g + 1]);
+                                r.z -= __uint_as_float(v[4 * g + 2]); r.w -= __uint_as_float(v[4 * g + 3]);
+                                *reinterpret_cast<float4*>(crow + gn) = r;
+                                if (prm.C1) {
+                                    uint2 hi, lo;
+                                    split2(r.x, r.y, hi.x, lo.x);
+                                    split2(r.z, r.w, hi.y, lo.y);
+                                    const size_t off = (size_t)gm * prm.lde + gn;
+                                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.C1) + off) = hi;
+                                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.C2) + off) = lo;
+                                }
                             }
                         }
+                    }
+                }
+                if (!ok) break;
+            } else {
+                if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
+                tc_fence_after();
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
+#pragma unroll 1
+                for (int c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32) {
+                    uint32_t v[32];
+                    tc_ld_32cols(taddr + c, v);
+                    tc_ld_wait();
+                    if (row_ok) {
+                        const int gn = n0 + c;
+                        if (gn < prm.N) epilogue_group<0>(prm, gm, gn, v);
+                        if (gn + 8 < prm.N) epilogue_group<1>(prm, gm, gn + 8, v);
+                        if (gn + 16 < prm.N) epilogue_group<2>(prm, gm, gn + 16, v);
+                        if (gn + 24 < prm.N) epilogue_group<3>(prm, gm, gn + 24, v);
                     }
                 }
             }
@@ -337,6 +431,25 @@ bool make_map(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, u
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+template <int BN>
+int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
+                 const CUtensorMap& b1, const TcParams& p, double flops, cudaStream_t st)
+{
+    static bool attr_done[64] = {};
+    if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
+        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)TcCfg<BN>::kSmemBytes));
+        attr_done[ctx->device] = true;
+    }
+    const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN);
+    const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    {
+        ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
+        gemm_tc_kernel<BN><<<grid, kThreads, TcCfg<BN>::kSmemBytes, st>>>(a0, a1, b0, b1, p);
+    }
+    return after_launch(ctx);
+}
+
 }  // namespace
 
 bool gemm_tc_supports(const GemmArgs& g)
@@ -356,11 +469,7 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
 {
     if (!gemm_tc_supports(g)) return GELO_ERR_UNSUPPORTED;
     if (!ctx->tmap_encode) return GELO_ERR_CUDA;
-    static bool attr_done[64] = {};
-    if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
-        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes));
-        attr_done[ctx->device] = true;
-    }
+    constexpr int BN = 256;
     const int rows_first = g.B2 ? g.b_split : g.K;
     CUtensorMap ma, mb, mb2;
     if (!make_map(ctx, &ma, g.A, (uint64_t)g.K, (uint64_t)g.M, (uint64_t)g.lda, BK, BM)) return GELO_ERR_CUDA;
@@ -371,27 +480,65 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
     } else {
         mb2 = mb;
     }
-    TcParams p;
+    TcParams p = {};
     p.M = g.M; p.N = g.N;
-    p.kb_first = ceil_div(rows_first, BK);
+    p.nseg = 1;
+    p.seg[0] = TcSegment{0, 0, 0, 0, ceil_div(rows_first, BK)};
     if (g.B2) {
-        p.a_k0_second = g.b_split & ~7;                       // TMA needs a 16-byte aligned inner coordinate
-        p.b_row0_second = p.a_k0_second - g.b_split;          // <= 0: rows above S read as zero
-        p.kb_second = ceil_div(g.K - p.a_k0_second, BK);
-    } else {
-        p.a_k0_second = 0; p.b_row0_second = 0; p.kb_second = 0;
+        const int a_k0 = g.b_split & ~7;                      // TMA needs a 16-byte aligned inner coordinate
+        p.nseg = 2;
+        p.seg[1] = TcSegment{0, 1, a_k0, a_k0 - g.b_split /* <= 0: rows above S read as zero */,
+                             ceil_div(g.K - a_k0, BK)};
     }
+    p.mode = TC_STORE_BF16;
     p.C0 = g.C[0]; p.C1 = g.C[g.nsplit > 1 ? 1 : 0]; p.C2 = g.C[g.nsplit > 2 ? 2 : 0];
-    p.ldc = g.ldc; p.csplit = g.N / g.nsplit;
-    p.out_f32 = 0;
+    p.ldc = g.ldc; p.csplit = g.N / g.nsplit; p.lde = 0;
     p.status = ctx->status_dev;
-    const int tiles = ceil_div(g.M, BM) * ceil_div(g.N, BN);
-    const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
-    {
-        ProfScope ps(ctx, PROF_GEMM_TC, 2.0 * g.M * (double)g.N * g.K, st);
-        gemm_tc_kernel<<<grid, kThreads, kSmemBytes, st>>>(ma, mb, mb2, p);
+    return launch_tiles<BN>(ctx, ma, ma, mb, mb2, p, 2.0 * g.M * (double)g.N * g.K, st);
+}
+
+// Split-precision product for the factorisations.  A = Ahi + Alo (M x K, stride lda), B = Bhi + Blo
+// (K x N, stride ldb), all bf16; the tensor cores accumulate Ahi Bhi + Ahi Blo + Alo Bhi in fp32.
+//   sub_from != nullptr : sub_from (fp32, stride ldc) -= product, and if emit_hi != nullptr the updated
+//                         values are also written as a (hi, lo) pair with stride lde
+//   sub_from == nullptr : the product itself is written as the pair (emit_hi, emit_lo), stride lde
+int launch_gemm_tc_split(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, const void* Alo, int lda,
+                         const void* Bhi, const void* Blo, int ldb, float* sub_from, int ldc, void* emit_hi,
+                         void* emit_lo, int lde, bool narrow_tiles, cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if ((lda % 8) || (ldb % 8) || (N % 8) || !aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo))
+        return GELO_ERR_INVALID;
+    if (sub_from && ((ldc % 4) || !aligned16(sub_from))) return GELO_ERR_INVALID;
+    if (emit_hi && ((lde % 8) || !aligned16(emit_hi) || !aligned16(emit_lo))) return GELO_ERR_INVALID;
+    if (!sub_from && !emit_hi) return GELO_ERR_INVALID;
+    CUtensorMap a0, a1, b0, b1;
+    if (!make_map(ctx, &a0, Ahi, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM) ||
+        !make_map(ctx, &a1, Alo, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM) ||
+        !make_map(ctx, &b0, Bhi, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 64, BK) ||
+        !make_map(ctx, &b1, Blo, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 64, BK))
+        return GELO_ERR_CUDA;
+    TcParams p = {};
+    p.M = M; p.N = N;
+    const int kb = ceil_div(K, BK);
+    p.nseg = 3;
+    p.seg[0] = TcSegment{0, 0, 0, 0, kb};
+    p.seg[1] = TcSegment{0, 1, 0, 0, kb};
+    p.seg[2] = TcSegment{1, 0, 0, 0, kb};
+    p.status = ctx->status_dev;
+    p.csplit = N;
+    if (sub_from) {
+        p.mode = TC_SUB_F32;
+        p.C0 = sub_from; p.ldc = ldc;
+        p.C1 = emit_hi; p.C2 = emit_lo; p.lde = lde;
+    } else {
+        p.mode = TC_EMIT_SPLIT;
+        p.C0 = emit_hi; p.C1 = emit_lo; p.ldc = lde; p.lde = lde;
     }
-    return after_launch(ctx);
+    const double flops = 6.0 * M * (double)N * K;
+    if (narrow_tiles) return launch_tiles<64>(ctx, a0, a1, b0, b1, p, flops, st);
+    return launch_tiles<256>(ctx, a0, a1, b0, b1, p, flops, st);
 }
 
 }  // namespace gelo

@@ -50,7 +50,59 @@ __global__ void __launch_bounds__(256) convert_kernel(int m, const TS* __restric
     if (c < m) put(dst + (size_t)r * ldd + c, get(src + (size_t)r * lds + c));
 }
 
+// hi = bf16(x), lo = bf16(x - hi) for a rows x cols block (fp32, stride lds) -> bf16 pair (stride ldo);
+// with T the pair is written transposed (cols x rows, stride ldo) through a shared-memory tile.
+__global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ src, int lds, int rows, int cols,
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int ldo)
+{
+    const int c = blockIdx.x * 256 + threadIdx.x;
+    const int r = blockIdx.y;
+    if (c >= cols) return;
+    const float x = src[(size_t)r * lds + c];
+    const __nv_bfloat16 h = __float2bfloat16_rn(x);
+    hi[(size_t)r * ldo + c] = h;
+    lo[(size_t)r * ldo + c] = __float2bfloat16_rn(x - __bfloat162float(h));
+}
+
+__global__ void __launch_bounds__(256) split_transpose_kernel(const float* __restrict__ src, int lds, int rows, int cols,
+                                                              __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int ldo)
+{
+    __shared__ float tile[32][33];
+    const int r0 = blockIdx.y * 32, c0 = blockIdx.x * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    for (int i = ty; i < 32; i += 8) {
+        const int r = r0 + i, c = c0 + tx;
+        tile[i][tx] = (r < rows && c < cols) ? src[(size_t)r * lds + c] : 0.0f;
+    }
+    __syncthreads();
+    for (int i = ty; i < 32; i += 8) {
+        const int c = c0 + i, r = r0 + tx;              // output row = source column
+        if (c < cols && r < rows) {
+            const float x = tile[tx][i];
+            const __nv_bfloat16 h = __float2bfloat16_rn(x);
+            hi[(size_t)c * ldo + r] = h;
+            lo[(size_t)c * ldo + r] = __float2bfloat16_rn(x - __bfloat162float(h));
+        }
+    }
+}
+
 }  // namespace
+
+int launch_split(gelo_ctx* ctx, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
+                 bool transpose, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return GELO_OK;
+    if (transpose) {
+        dim3 grid(ceil_div(cols, 32), ceil_div(rows, 32));
+        split_transpose_kernel<<<grid, 256, 0, st>>>(src, lds, rows, cols, static_cast<__nv_bfloat16*>(hi),
+                                                     static_cast<__nv_bfloat16*>(lo), ldo);
+    } else {
+        dim3 grid(ceil_div(cols, 256), rows);
+        split_kernel<<<grid, 256, 0, st>>>(src, lds, rows, cols, static_cast<__nv_bfloat16*>(hi),
+                                           static_cast<__nv_bfloat16*>(lo), ldo);
+    }
+    return after_launch(ctx);
+}
 
 int launch_finish_mixing(gelo_ctx* ctx, int m, const float* src, int lds, const float* sign_diag, int ldg,
                          int dtype, void* dst, void* dstT, int ldd, cudaStream_t st)

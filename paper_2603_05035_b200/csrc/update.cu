@@ -258,6 +258,35 @@ rank_update_kernel(const float* __restrict__ A, int lda, const float* __restrict
 
 }  // namespace
 
+TcScratch carve_tc(Arena& a, int m, int ld)
+{
+    TcScratch t;
+    for (int h = 0; h < 2; ++h) {
+        t.panA[h] = a.take((size_t)m * kOuter * 2);
+        t.panAt[h] = a.take((size_t)kOuter * ld * 2);
+        t.rowB[h] = a.take((size_t)kOuter * ld * 2);
+        t.rowB2[h] = a.take((size_t)kOuter * ld * 2);
+        t.tt[h] = a.take((size_t)kOuter * kOuter * 2);
+        t.big[h] = a.take((size_t)m * ld * 2);
+    }
+    t.t128 = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
+    t.gram = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
+    t.wf32 = static_cast<float*>(a.take((size_t)kOuter * ld * 4));
+    return t;
+}
+
+int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, int M, int N, int K, const float* A, int lda, const float* B,
+                  int ldb, float* C, int ldc, cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (K > kOuter) return GELO_ERR_INVALID;
+    const int ldn = (N + 7) & ~7;
+    GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], kOuter, false, st));
+    GELO_TRY(launch_split(ctx, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, false, st));
+    return launch_gemm_tc_split(ctx, M, (N + 7) & ~7, K, t.panA[0], t.panA[1], kOuter, t.rowB[0], t.rowB[1], ldn, C, ldc,
+                                nullptr, nullptr, 0, false, st);
+}
+
 int panel_slab_count(gelo_ctx* ctx, int nr, int nc)
 {
     // enough CTAs to cover the GPU about twice (two CTAs fit per SM), slabs of at least 128 rows

@@ -411,3 +411,23 @@ def test_batched_offload_full_size(oracle):
         rows = sample_rows(n, 48, seed=i)
         assert oracle.rel_fro(y[rows], oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)) <= TOL["bf16"]
     c.close()
+
+
+# ------------------------------------------------------------------------- split-precision tensor-core update
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (300, 520, 128), (1000, 777, 96), (4300, 4172, 128), (64, 8, 32),
+                                    (130, 1, 5)])
+def test_tensor_core_update_f32(ctx, oracle, M, N, K):
+    rng = np.random.default_rng(M + N + K)
+    A = dev(rng.standard_normal((M, K)).astype(np.float32))
+    B = dev(rng.standard_normal((K, N)).astype(np.float32))
+    ldc = ((N + 63) // 64) * 64
+    C = torch.zeros((M, ldc), device="cuda", dtype=torch.float32)
+    C0 = rng.standard_normal((M, N)).astype(np.float32)
+    C[:, :N] = dev(C0)
+    ctx.update_f32(M, N, K, A, K, B, N, C, ldc)
+    ref = C0.astype(np.float64) - (oracle.matmul(f64(A), f64(B)) if M * N * K < 3e8 else f64(A) @ f64(B))
+    got = f64(C[:, :N])
+    # bf16 (high, low) pairs carry 16 significand bits: products are good to about 2^-16
+    assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 2e-5
+    assert np.max(np.abs(got - ref)) <= 4e-4 * np.sqrt(K)
