@@ -84,6 +84,12 @@ int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes);
  * each with the next attempt number in the Philox counter). */
 int gelo_set_nonorthogonal(gelo_ctx* ctx, float gamma, float cond_bound, int max_attempts);
 
+/* How the trailing updates of the blocked QR / LU are computed.  0 (default): split-precision tensor-core
+ * products for bf16 calls with m >= 256, fp32 FMA otherwise; 1: always fp32 FMA; 2: always tensor cores.
+ * The tensor-core products are good to about 1e-5 relative, which the fp32 path's 1e-4 budget does not leave
+ * room for, hence the default. */
+int gelo_set_level3(gelo_ctx* ctx, int mode);
+
 /* Preferred row stride (elements) of an m x m mixing matrix: m rounded up to 64. */
 int gelo_mixing_ld(int m);
 

@@ -38,6 +38,7 @@ EXPORTS = {
     "gelo_set_workspace": (_i, [_vp, _vp, _sz]),
     "gelo_set_nonorthogonal": (_i, [_vp, _f, _f, _i]),
     "gelo_mixing_ld": (_i, [_i]),
+    "gelo_set_level3": (_i, [_vp, _i]),
     "gelo_last_status": (_i, [_vp, _vp]),
     "gelo_launch_count": (ctypes.c_longlong, [_vp, _i]),
     "gelo_status_string": (ctypes.c_char_p, [_i]),
@@ -200,6 +201,9 @@ class Context:
     def set_nonorthogonal(self, gamma=0.5, cond_bound=100.0, max_attempts=8):
         self._check(self._lib.gelo_set_nonorthogonal(self._h, gamma, cond_bound, max_attempts),
                     "gelo_set_nonorthogonal")
+
+    def set_level3(self, mode: int):
+        self._check(self._lib.gelo_set_level3(self._h, mode), "gelo_set_level3")
 
     def mixing_ld(self, m) -> int:
         return int(self._lib.gelo_mixing_ld(m))

@@ -11,6 +11,15 @@ namespace {
 
 inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 inline int round_up(int x, int to) { return (x + to - 1) / to * to; }
+constexpr int kTcMinRows = 256;   // below this the factorisations are latency-bound anyway
+
+// Whether the factorisations of an m x m sample stored as `dtype` use the split-precision tensor-core updates.
+inline bool use_level3_tc(const gelo_ctx* ctx, int m, int dtype)
+{
+    if (ctx->level3 == 1) return false;
+    if (ctx->level3 == 2) return m > gelo::kPanel;
+    return dtype == GELO_BF16 && m >= kTcMinRows;
+}
 
 // Every scratch buffer of one call with sizes (n, k, d, p, dtype); carved in a fixed order so
 // that gelo_workspace_bytes and the calls agree.
@@ -118,7 +127,9 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st));
     GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st));
     if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
-    GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
+    // split-precision tensor-core updates (about 1e-5 relative) serve the bf16 path; the fp32 path stays exact
+    if (use_level3_tc(ctx, m, dtype)) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, ldi, L.X32, L.lu, L.tc, st));
+    else GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
     GELO_TRY(launch_narrow(ctx, m, L.X32, ldi, dtype, Ainv_out, lda, st));
     return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st,
                              deferred);
@@ -458,10 +469,13 @@ int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ain
     Layout L;
     if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
-    if (ld == L.ldi) return run_lu_inverse(ctx, m, A_dev, ld, Ainv_dev, L.lu, st);
+    const bool tcp = use_level3_tc(ctx, m, GELO_F32);
+    if (ld == L.ldi) return tcp ? run_lu_inverse_tc(ctx, m, A_dev, ld, Ainv_dev, L.lu, L.tc, st)
+                                : run_lu_inverse(ctx, m, A_dev, ld, Ainv_dev, L.lu, st);
     GELO_CUDA_OK(cudaMemcpy2DAsync(L.A32, (size_t)L.ldi * 4, A_dev, (size_t)ld * 4, (size_t)m * 4, m,
                                    cudaMemcpyDeviceToDevice, st));
-    GELO_TRY(run_lu_inverse(ctx, m, L.A32, L.ldi, L.X32, L.lu, st));
+    if (tcp) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, L.ldi, L.X32, L.lu, L.tc, st));
+    else GELO_TRY(run_lu_inverse(ctx, m, L.A32, L.ldi, L.X32, L.lu, st));
     return cudaMemcpy2DAsync(Ainv_dev, (size_t)ld * 4, L.X32, (size_t)L.ldi * 4, (size_t)m * 4, m,
                              cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
 }
@@ -660,6 +674,13 @@ int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int 
     Layout L;
     if (!carve_ctx(ctx, M > N ? M : N, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
     return tc_update_f32(ctx, L.tc, M, N, K, A_dev, lda, B_dev, ldb, C_dev, ldc, as_stream(stream));
+}
+
+int gelo_set_level3(gelo_ctx* ctx, int mode)
+{
+    if (!ctx || mode < 0 || mode > 2) return GELO_ERR_INVALID;
+    ctx->level3 = mode;
+    return GELO_OK;
 }
 
 }  // extern "C"

@@ -51,6 +51,7 @@ struct gelo_ctx {
     float gamma = 0.5f;
     float cond_bound = 100.0f;
     int max_attempts = 8;
+    int level3 = 0;               // 0: tensor cores for bf16 calls with m >= 256; 1: always fp32 FMA; 2: always tensor cores
     long long launches = 0;
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
     // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
@@ -168,6 +169,9 @@ struct LuScratch {
 };
 LuScratch carve_lu(Arena&, int m, int ld);
 int run_lu_inverse(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, cudaStream_t);
+struct TcScratch;
+int run_lu_inverse_tc(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, const TcScratch&,
+                      cudaStream_t);
 
 struct CondScratch {
     float* vec = nullptr;     // iterate, image and row-slab partial sums for both operators

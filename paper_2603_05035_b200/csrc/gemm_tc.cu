@@ -30,7 +30,6 @@ namespace {
 
 constexpr int BM = 128;
 constexpr int BK = 64;
-constexpr int kStages = 4;
 constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
@@ -142,11 +141,17 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 }
 
 
-template <int BN>
+// Epilogue staging for the in-place subtraction: every epilogue warp owns two 32 x 32 fp32 boxes (4 KiB each)
+// that TMA reduces into global memory.
+constexpr uint32_t kStageBoxBytes = 32 * 32 * 4;
+constexpr uint32_t kStagingBytes = kEpiWarps * 2 * kStageBoxBytes;
+
+template <int BN, int kStages, bool kStaging>
 struct TcCfg {
+    static constexpr uint32_t kStagingUsed = kStaging ? kStagingBytes : 0u;
     static constexpr uint32_t kBBytes = (BN / 64) * kBBoxBytes;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
-    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + 1024 /*alignment slack*/ + 256 /*barriers*/;
+    static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kStagingUsed + 1024 /*alignment slack*/ + 256 /*barriers*/;
     // Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = BN.
     static constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
                                            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
@@ -203,19 +208,20 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
     }
 }
 
-template <int BN>
+template <int BN, int kStages, bool kStaging>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
-               const TcParams prm)
+               const __grid_constant__ CUtensorMap map_c, const TcParams prm)
 {
-    using Cfg = TcCfg<BN>;
+    using Cfg = TcCfg<BN, kStages, kStaging>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-byte alignment
     uint8_t* gen_base = smem_raw + (tiles_base - raw);
-    const uint32_t bar_base = tiles_base + kStages * Cfg::kStageBytes;
-    uint8_t* bar_gen = gen_base + kStages * Cfg::kStageBytes;
+    const uint32_t staging_base = tiles_base + kStages * Cfg::kStageBytes;      // 1024-byte aligned
+    const uint32_t bar_base = staging_base + Cfg::kStagingUsed;
+    uint8_t* bar_gen = gen_base + kStages * Cfg::kStageBytes + Cfg::kStagingUsed;
     // barrier layout (8 bytes each): full[kStages], empty[kStages], acc_full[2], acc_empty[2]; then tmem slot, abort
     auto full_bar = [&](int s) { return bar_base + 8u * s; };
     auto empty_bar = [&](int s) { return bar_base + 8u * (kStages + s); };
@@ -320,7 +326,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         const int quarter = warp & 3;                 // the TMEM lane quarter this warp may read
         const int half = (warp - 2) >> 2;             // which half of the tile's columns
         constexpr int kHalfCols = BN / 2;
-        uint32_t acc_it = 0;
+        uint32_t acc_it = 0, box_it = 0;
         bool ok = true;
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
             const int a = acc_it % kAccStages;
@@ -329,51 +335,37 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             const int n0 = (tile / m_tiles) * BN;
             const int gm = m0 + quarter * 32 + lane;
             const bool row_ok = gm < prm.M;
-            if (prm.mode == TC_SUB_F32) {
-                // C -= acc in place, 32 columns at a time; the C values are requested before the wait on
-                // the accumulator so that their latency overlaps the main loop
-                float* crow = static_cast<float*>(prm.C0) + (size_t)gm * prm.ldc;
+            if (kStaging && prm.mode == TC_SUB_F32) {
+                // C -= acc without reading C: the negated accumulator goes through a swizzled shared-memory box and
+                // a TMA reduce-add into global memory (the addition happens at the L2); TMA clips at the matrix edge
+                if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
+                tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
-                bool waited = false;
+                const uint32_t my_staging = staging_base + (uint32_t)(warp - 2) * 2u * kStageBoxBytes;
 #pragma unroll 1
-                for (int c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32) {
-                    float4 cv[8];
-#pragma unroll
-                    for (int g = 0; g < 8; ++g) {
-                        const int gn = n0 + c + g * 4;
-                        cv[g] = (row_ok && gn < prm.N) ? *reinterpret_cast<const float4*>(crow + gn)
-                                                       : make_float4(0.f, 0.f, 0.f, 0.f);
-                    }
-                    if (!waited) {
-                        if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
-                        tc_fence_after();
-                        waited = true;
-                    }
+                for (int c = half * kHalfCols; c < (half + 1) * kHalfCols; c += 32, ++box_it) {
+                    const uint32_t buf = my_staging + (box_it & 1u) * kStageBoxBytes;
+                    if (lane == 0) asm volatile("cp.async.bulk.wait_group.read 1;" ::: "memory");   // box of two chunks ago is free
+                    __syncwarp();
                     uint32_t v[32];
                     tc_ld_32cols(taddr + c, v);
                     tc_ld_wait();
-                    if (row_ok) {
 #pragma unroll
-                        for (int g = 0; g < 8; ++g) {
-                            const int gn = n0 + c + g * 4;
-                            if (gn < prm.N) {
-                                float4 r = cv[g];
-                                r.x -= __uint_as_float(v[4 * g + 0]); r.y -= __uint_as_float(v[4 * g + 1]);
-                                r.z -= __uint_as_float(v[4 * g + 2]); r.w -= __uint_as_float(v[4 * g + 3]);
-                                *reinterpret_cast<float4*>(crow + gn) = r;
-                                if (prm.C1) {
-                                    uint2 hi, lo;
-                                    split2(r.x, r.y, hi.x, lo.x);
-                                    split2(r.z, r.w, hi.y, lo.y);
-                                    const size_t off = (size_t)gm * prm.lde + gn;
-                                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.C1) + off) = hi;
-                                    *reinterpret_cast<uint2*>(static_cast<__nv_bfloat16*>(prm.C2) + off) = lo;
-                                }
-                            }
-                        }
+                    for (int j4 = 0; j4 < 8; ++j4) {
+                        const uint32_t dst = buf + (uint32_t)lane * 128u + (uint32_t)((j4 ^ (lane & 7)) << 4);
+                        asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};"
+                                     ::"r"(dst), "f"(-__uint_as_float(v[4 * j4 + 0])), "f"(-__uint_as_float(v[4 * j4 + 1])),
+                                       "f"(-__uint_as_float(v[4 * j4 + 2])), "f"(-__uint_as_float(v[4 * j4 + 3])) : "memory");
                     }
+                    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+                    __syncwarp();
+                    if (lane == 0 && n0 + c < prm.N && m0 + quarter * 32 < prm.M) {
+                        asm volatile(
+                            "cp.reduce.async.bulk.tensor.2d.global.shared::cta.add.tile.bulk_group [%0, {%1, %2}], [%3];"
+                            ::"l"(&map_c), "r"(n0 + c), "r"(m0 + quarter * 32), "r"(buf) : "memory");
+                    }
+                    if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
-                if (!ok) break;
             } else {
                 if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
                 tc_fence_after();
@@ -396,6 +388,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             __syncwarp();
             if (lane == 0) mbar_arrive(acc_empty_bar(a));
         }
+        if (lane == 0) asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");   // staged boxes fully written out
         if (!ok && lane == 0) { *abort_flag = 1; atomicCAS(prm.status, 0, (int)GELO_ERR_TIMEOUT); }
     }
 
@@ -431,23 +424,39 @@ bool make_map(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, u
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-template <int BN>
+template <int BN, int kStages, bool kStaging>
 int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
-                 const CUtensorMap& b1, const TcParams& p, double flops, cudaStream_t st)
+                 const CUtensorMap& b1, const CUtensorMap& c, const TcParams& p, double flops, cudaStream_t st)
 {
+    using Cfg = TcCfg<BN, kStages, kStaging>;
+    static_assert(Cfg::kSmemBytes <= 227 * 1024, "shared memory budget");
     static bool attr_done[64] = {};
     if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
-        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                          (int)TcCfg<BN>::kSmemBytes));
+        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN, kStages, kStaging>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                          (int)Cfg::kSmemBytes));
         attr_done[ctx->device] = true;
     }
     const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN);
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
-        gemm_tc_kernel<BN><<<grid, kThreads, TcCfg<BN>::kSmemBytes, st>>>(a0, a1, b0, b1, p);
+        gemm_tc_kernel<BN, kStages, kStaging><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, p);
     }
     return after_launch(ctx);
+}
+
+// fp32 tensor map of the matrix that the subtracting epilogue reduces into: 32 x 32 boxes, 128-byte swizzle.
+bool make_map_f32_box(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, uint64_t rows, uint64_t ld)
+{
+    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
+    if (!enc) return false;
+    const cuuint64_t dims[2] = { cols, rows };
+    const cuuint64_t strides[1] = { ld * 4 };
+    const cuuint32_t box[2] = { 32, 32 };
+    const cuuint32_t estr[2] = { 1, 1 };
+    return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 }  // namespace
@@ -494,7 +503,7 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
     p.C0 = g.C[0]; p.C1 = g.C[g.nsplit > 1 ? 1 : 0]; p.C2 = g.C[g.nsplit > 2 ? 2 : 0];
     p.ldc = g.ldc; p.csplit = g.N / g.nsplit; p.lde = 0;
     p.status = ctx->status_dev;
-    return launch_tiles<BN>(ctx, ma, ma, mb, mb2, p, 2.0 * g.M * (double)g.N * g.K, st);
+    return launch_tiles<BN, 4, false>(ctx, ma, ma, mb, mb2, ma, p, 2.0 * g.M * (double)g.N * g.K, st);
 }
 
 // Split-precision product for the factorisations.  A = Ahi + Alo (M x K, stride lda), B = Bhi + Blo
@@ -508,7 +517,7 @@ int launch_gemm_tc_split(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, co
 {
     if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
     if (!ctx->tmap_encode) return GELO_ERR_CUDA;
-    if ((lda % 8) || (ldb % 8) || (N % 8) || !aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo))
+    if ((lda % 8) || (ldb % 8) || (!sub_from && (N % 8)) || !aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo))
         return GELO_ERR_INVALID;
     if (sub_from && ((ldc % 4) || !aligned16(sub_from))) return GELO_ERR_INVALID;
     if (emit_hi && ((lde % 8) || !aligned16(emit_hi) || !aligned16(emit_lo))) return GELO_ERR_INVALID;
@@ -528,17 +537,20 @@ int launch_gemm_tc_split(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, co
     p.seg[2] = TcSegment{1, 0, 0, 0, kb};
     p.status = ctx->status_dev;
     p.csplit = N;
+    CUtensorMap mc = a0;
     if (sub_from) {
+        if (emit_hi) return GELO_ERR_UNSUPPORTED;
+        if (!make_map_f32_box(ctx, &mc, sub_from, (uint64_t)N, (uint64_t)M, (uint64_t)ldc)) return GELO_ERR_CUDA;
         p.mode = TC_SUB_F32;
         p.C0 = sub_from; p.ldc = ldc;
-        p.C1 = emit_hi; p.C2 = emit_lo; p.lde = lde;
     } else {
         p.mode = TC_EMIT_SPLIT;
         p.C0 = emit_hi; p.C1 = emit_lo; p.ldc = lde; p.lde = lde;
     }
     const double flops = 6.0 * M * (double)N * K;
-    if (narrow_tiles) return launch_tiles<64>(ctx, a0, a1, b0, b1, p, flops, st);
-    return launch_tiles<256>(ctx, a0, a1, b0, b1, p, flops, st);
+    if (sub_from) return launch_tiles<256, 3, true>(ctx, a0, a1, b0, b1, mc, p, flops, st);
+    if (narrow_tiles) return launch_tiles<64, 4, false>(ctx, a0, a1, b0, b1, mc, p, flops, st);
+    return launch_tiles<256, 4, false>(ctx, a0, a1, b0, b1, mc, p, flops, st);
 }
 
 }  // namespace gelo

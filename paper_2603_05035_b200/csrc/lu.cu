@@ -363,6 +363,98 @@ LuScratch carve_lu(Arena& a, int m, int ld)
     return s;
 }
 
+// Level-3 variant: outer blocks of kOuter columns.  Inside a block the 32-column panels and rank-32
+// updates above run on the block only; everything outside the block is updated once per block by a
+// split-precision tensor-core product (K = kOuter), which cuts the passes over the big matrices by four.
+int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const LuScratch& s, const TcScratch& tc,
+                      cudaStream_t st)
+{
+    float* M = s.M;
+    GELO_CUDA_OK(cudaMemcpyAsync(M, A, (size_t)m * ld * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    for (int b0 = 0; b0 < m; b0 += kOuter) {
+        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
+        const int bend = b0 + ob;
+        for (int j0 = b0; j0 < bend; j0 += NB) {
+            const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
+            GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
+            if (ob > jb) {       // interchanges on the other columns of this block
+                swap_rows_kernel<<<ceil_div(ob, 256), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, b0, bend, j0, j0 + jb);
+                GELO_TRY(after_launch(ctx));
+            }
+            const int ncb = bend - (j0 + jb);
+            if (ncb > 0) {
+                tri_solve_block_kernel<false><<<ceil_div(ncb, 256), 256, 0, st>>>(M, ld, M, ld, j0, jb, j0 + jb, bend);
+                GELO_TRY(after_launch(ctx));
+                GELO_TRY(launch_rank_update(ctx, M + (size_t)(j0 + jb) * ld + j0, ld, M + (size_t)j0 * ld + j0 + jb, ld,
+                                            M + (size_t)(j0 + jb) * ld + j0 + jb, ld, m - j0 - jb, ncb, jb, st));
+            }
+        }
+        if (m > ob) {            // the block's interchanges on everything left and right of it
+            swap_rows_kernel<<<ceil_div(m, 256), 256, 0, st>>>(M, ld, b0, ob, s.ipiv, 0, m, b0, bend);
+            GELO_TRY(after_launch(ctx));
+        }
+        const int nc = m - bend;
+        if (nc <= 0) continue;
+        // U12 = L11^-1 A12 on the block's row strip
+        for (int i0 = b0; i0 < bend; i0 += NB) {
+            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
+            tri_solve_block_kernel<false><<<ceil_div(nc, 256), 256, 0, st>>>(M, ld, M, ld, i0, ib, bend, m);
+            GELO_TRY(after_launch(ctx));
+            const int rem = bend - (i0 + ib);
+            if (rem > 0)
+                GELO_TRY(launch_rank_update(ctx, M + (size_t)(i0 + ib) * ld + i0, ld, M + (size_t)i0 * ld + bend, ld,
+                                            M + (size_t)(i0 + ib) * ld + bend, ld, rem, nc, ib, st));
+        }
+        // A22 -= L21 U12
+        GELO_TRY(tc_update_f32(ctx, tc, nc, nc, ob, M + (size_t)bend * ld + b0, ld, M + (size_t)b0 * ld + bend, ld,
+                               M + (size_t)bend * ld + bend, ld, st));
+    }
+    // ---- X = P, then L Y = P, then U X = Y ----
+    const size_t perm_smem = (size_t)m * sizeof(int);
+    if (perm_smem > 48 * 1024)
+        GELO_CUDA_OK(cudaFuncSetAttribute(build_perm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)perm_smem));
+    build_perm_kernel<<<1, 256, perm_smem, st>>>(s.ipiv, s.perm, m);
+    GELO_TRY(after_launch(ctx));
+    permuted_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(X, ld, m, s.perm);
+    GELO_TRY(after_launch(ctx));
+    for (int b0 = 0; b0 < m; b0 += kOuter) {
+        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
+        const int bend = b0 + ob;
+        for (int i0 = b0; i0 < bend; i0 += NB) {
+            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
+            tri_solve_block_kernel<false><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);
+            GELO_TRY(after_launch(ctx));
+            const int rem = bend - (i0 + ib);
+            if (rem > 0)
+                GELO_TRY(launch_rank_update(ctx, M + (size_t)(i0 + ib) * ld + i0, ld, X + (size_t)i0 * ld, ld,
+                                            X + (size_t)(i0 + ib) * ld, ld, rem, m, ib, st));
+        }
+        if (m - bend > 0)
+            GELO_TRY(tc_update_f32(ctx, tc, m - bend, m, ob, M + (size_t)bend * ld + b0, ld, X + (size_t)b0 * ld, ld,
+                                   X + (size_t)bend * ld, ld, st));
+    }
+    const int nblocks = ceil_div(m, kOuter);
+    for (int blk = nblocks - 1; blk >= 0; --blk) {
+        const int b0 = blk * kOuter;
+        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
+        const int bend = b0 + ob;
+        const int nsub = ceil_div(ob, NB);
+        for (int sb = nsub - 1; sb >= 0; --sb) {
+            const int i0 = b0 + sb * NB;
+            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
+            tri_solve_block_kernel<true><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);
+            GELO_TRY(after_launch(ctx));
+            const int above = i0 - b0;
+            if (above > 0)
+                GELO_TRY(launch_rank_update(ctx, M + (size_t)b0 * ld + i0, ld, X + (size_t)i0 * ld, ld,
+                                            X + (size_t)b0 * ld, ld, above, m, ib, st));
+        }
+        if (b0 > 0)
+            GELO_TRY(tc_update_f32(ctx, tc, b0, m, ob, M + b0, ld, X + (size_t)b0 * ld, ld, X, ld, st));
+    }
+    return GELO_OK;
+}
+
 int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const LuScratch& s, cudaStream_t st)
 {
     if ((size_t)m * sizeof(int) > 200 * 1024) return GELO_ERR_UNSUPPORTED;

@@ -283,7 +283,7 @@ int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, int M, int N, int K, const 
     const int ldn = (N + 7) & ~7;
     GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], kOuter, false, st));
     GELO_TRY(launch_split(ctx, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, false, st));
-    return launch_gemm_tc_split(ctx, M, (N + 7) & ~7, K, t.panA[0], t.panA[1], kOuter, t.rowB[0], t.rowB[1], ldn, C, ldc,
+    return launch_gemm_tc_split(ctx, M, N, K, t.panA[0], t.panA[1], kOuter, t.rowB[0], t.rowB[1], ldn, C, ldc,
                                 nullptr, nullptr, 0, false, st);
 }
 

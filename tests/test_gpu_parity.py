@@ -431,3 +431,23 @@ def test_tensor_core_update_f32(ctx, oracle, M, N, K):
     # bf16 (high, low) pairs carry 16 significand bits: products are good to about 2^-16
     assert np.linalg.norm(got - ref) / np.linalg.norm(ref) <= 2e-5
     assert np.max(np.abs(got - ref)) <= 4e-4 * np.sqrt(K)
+
+
+@pytest.mark.parametrize("m", [130, 257, 512, 1000])
+def test_lu_inverse_tensor_core_blocks(oracle, m):
+    c = make_ctx(m, 0, 8, 24, "f32")
+    c.set_level3(2)
+    ld = c.mixing_ld(m)
+    A64, _ = oracle.sample_mixing(m, 1, seed=400 + m)
+    A64 = A64.astype(np.float32).astype(np.float64)
+    A = padded(m, ld, torch.float32); A[:, :m] = dev(A64)
+    X = padded(m, ld, torch.float32)
+    c.lu_inverse(m, A, ld, X)
+    x = f64(X[:, :m])
+    # operands carried as bf16 (high, low) pairs have 16 significand bits (2^-17 each); the two triangular
+    # solves amplify that by the conditioning of L and U: a few 1e-4 at kappa(A) ~ 5, far inside the bf16
+    # path's budget (A^-1 is rounded to bf16, 4e-3, right afterwards)
+    assert oracle.rel_fro(x, oracle.lu_inverse(A64)) <= 1e-3
+    assert np.linalg.norm(A64 @ x - np.eye(m)) / np.sqrt(m) <= 1e-3
+    assert c.last_status() == binding.OK
+    c.close()
