@@ -108,11 +108,12 @@ int gemm_dispatch(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
 // A (and A^-1) for one attempt into L.A32 / L.X32 or straight into the outputs.
 int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, uint32_t attempt,
                    int dtype, void* A_out, void* Ainv_out, int lda, float* cond_dev, cudaStream_t st,
-                   bool deferred = false)
+                   bool deferred = false, const uint64_t* seed_dev = nullptr)
 {
     const int ldi = L.ldi;
-    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st));
-    GELO_TRY(run_householder_qr(ctx, m, L.G, ldi, L.Qraw, L.qr, st));
+    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st, seed_dev));
+    if (use_level3_tc(ctx, m, dtype)) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, st));
+    else GELO_TRY(run_householder_qr(ctx, m, L.G, ldi, L.Qraw, L.qr, st));
     if (kind == GELO_ORTHOGONAL) {
         GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, dtype, A_out, Ainv_out, lda, st));
         if (cond_dev) {
@@ -124,7 +125,7 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     // Q0 (signed, fp32) -> A = Q0 + gamma / sqrt(m) * G1 -> stored type -> inverse of the stored A
     GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, GELO_F32, L.A32, nullptr, ldi, st));
     const float s = ctx->gamma / sqrtf((float)m);
-    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st));
+    GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st, seed_dev));
     GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st));
     if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
     // split-precision tensor-core updates (about 1e-5 relative) serve the bf16 path; the fp32 path stays exact
@@ -205,6 +206,53 @@ int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, i
 }
 
 
+__global__ void set_seed_kernel(uint64_t* slot, uint64_t seed) { *slot = seed; }
+
+void drop_graphs(gelo_ctx* ctx)
+{
+    for (auto& g : ctx->graphs) cudaGraphExecDestroy(g.exec);
+    ctx->graphs.clear();
+}
+
+// Samples (A, A^-1) of one batched call on a lane stream by replaying a launch graph of the whole sampling
+// sequence (about a thousand dependent launches): one host call instead of a thousand, so a single host thread
+// keeps all lanes busy.  The seed reaches the kernels through the lane's device slot.  The first use of a
+// (lane scratch, kind, size, type) combination records the graph by stream capture.
+int sample_on_lane(gelo_ctx* ctx, const Layout& L, int lane, int m, int kind, uint64_t seed, int dtype, cudaStream_t ls)
+{
+    uint64_t* slot = ctx->lane_seed_dev + lane * 8;
+    set_seed_kernel<<<1, 1, 0, ls>>>(slot, seed);
+    GELO_TRY(after_launch(ctx));
+    if (ctx->prof_on)      // per-launch timing needs real launches
+        return sample_attempt(ctx, L, m, kind, seed, 0u, dtype, L.A, L.Ainv, L.ldi, nullptr, ls, true, slot);
+    for (auto& g : ctx->graphs) {
+        if (g.key_ptr == L.G && g.m == m && g.kind == kind && g.dtype == dtype && g.level3 == ctx->level3) {
+            GELO_CUDA_OK(cudaGraphLaunch(g.exec, ls));
+            ctx->launches += g.launches;
+            return GELO_OK;
+        }
+    }
+    const long long before = ctx->launches;
+    GELO_CUDA_OK(cudaStreamBeginCapture(ls, cudaStreamCaptureModeRelaxed));
+    const int rc = sample_attempt(ctx, L, m, kind, seed, 0u, dtype, L.A, L.Ainv, L.ldi, nullptr, ls, true, slot);
+    cudaGraph_t graph = nullptr;
+    const cudaError_t ce = cudaStreamEndCapture(ls, &graph);
+    if (rc != GELO_OK || ce != cudaSuccess || !graph) {
+        if (graph) cudaGraphDestroy(graph);
+        return rc != GELO_OK ? rc : GELO_ERR_CUDA;
+    }
+    gelo_ctx::SampleGraph g;
+    g.key_ptr = L.G; g.m = m; g.kind = kind; g.dtype = dtype; g.level3 = ctx->level3;
+    g.launches = ctx->launches - before;
+    g.exec = nullptr;
+    const cudaError_t ie = cudaGraphInstantiate(&g.exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (ie != cudaSuccess) return GELO_ERR_CUDA;
+    ctx->graphs.push_back(g);
+    GELO_CUDA_OK(cudaGraphLaunch(g.exec, ls));
+    return GELO_OK;
+}
+
 // The whole path for a batch of independent calls.  Sampling A depends only on the seed, so up to
 // `lanes` calls sample their mixing pairs concurrently on the context's lane streams (each with its
 // own scratch) while the main stream runs shields and the three products of earlier calls.
@@ -237,7 +285,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         const int l = i % D;
         cudaStream_t ls = ctx->lane_stream[l];
         if (i >= D) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->lane_free[l], 0));
-        GELO_TRY(sample_attempt(ctx, L[l], m, kinds[i], seeds[i], 0u, dtype, L[l].A, L[l].Ainv, L[l].ldi, nullptr, ls, true));
+        GELO_TRY(sample_on_lane(ctx, L[l], l, m, kinds[i], seeds[i], dtype, ls));
         GELO_CUDA_OK(cudaEventRecord(ctx->lane_ready[l], ls));
         return GELO_OK;
     };
@@ -335,6 +383,7 @@ int gelo_create(gelo_ctx** out, int device)
         lanes_ok = cudaStreamCreateWithFlags(&ctx->lane_stream[l], cudaStreamNonBlocking) == cudaSuccess &&
                    cudaEventCreateWithFlags(&ctx->lane_ready[l], cudaEventDisableTiming) == cudaSuccess &&
                    cudaEventCreateWithFlags(&ctx->lane_free[l], cudaEventDisableTiming) == cudaSuccess;
+    lanes_ok = lanes_ok && cudaMalloc(&ctx->lane_seed_dev, kMaxLanes * 8 * sizeof(uint64_t)) == cudaSuccess;
     if (!lanes_ok) { gelo_destroy(ctx); return GELO_ERR_CUDA; }
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
@@ -354,6 +403,8 @@ int gelo_destroy(gelo_ctx* ctx)
         if (ctx->lane_ready[l]) cudaEventDestroy(ctx->lane_ready[l]);
         if (ctx->lane_free[l]) cudaEventDestroy(ctx->lane_free[l]);
     }
+    drop_graphs(ctx);
+    if (ctx->lane_seed_dev) cudaFree(ctx->lane_seed_dev);
     if (ctx->batch_start) cudaEventDestroy(ctx->batch_start);
     cudaFree(ctx->status_dev);
     cudaFreeHost(ctx->status_host);
@@ -374,6 +425,7 @@ int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes)
 {
     if (!ctx) return GELO_ERR_INVALID;
     if (dev_ws && (reinterpret_cast<uintptr_t>(dev_ws) & 255u)) return GELO_ERR_INVALID;
+    drop_graphs(ctx);              // recorded launches point into the old workspace
     ctx->ws = dev_ws;
     ctx->ws_bytes = dev_ws ? bytes : 0;
     return GELO_OK;
@@ -383,6 +435,7 @@ int gelo_set_nonorthogonal(gelo_ctx* ctx, float gamma, float cond_bound, int max
 {
     if (!ctx || !(gamma >= 0.0f) || !(cond_bound >= 1.0f) || max_attempts < 1 || max_attempts > 64)
         return GELO_ERR_INVALID;
+    drop_graphs(ctx);              // gamma and the bound are baked into recorded launches
     ctx->gamma = gamma;
     ctx->cond_bound = cond_bound;
     ctx->max_attempts = max_attempts;
@@ -450,13 +503,16 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
     Layout L;
     if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
+    const bool tcp = use_level3_tc(ctx, m, GELO_F32);
     if (ld == L.ldi) {
-        GELO_TRY(run_householder_qr(ctx, m, G_dev, ld, L.Qraw, L.qr, st));
+        if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, st));
+        else GELO_TRY(run_householder_qr(ctx, m, G_dev, ld, L.Qraw, L.qr, st));
         return launch_finish_mixing(ctx, m, L.Qraw, ld, G_dev, ld, GELO_F32, Q_dev, Qt_dev, ld, st);
     }
     GELO_CUDA_OK(cudaMemcpy2DAsync(L.G, (size_t)L.ldi * 4, G_dev, (size_t)ld * 4, (size_t)m * 4, m,
                                    cudaMemcpyDeviceToDevice, st));
-    GELO_TRY(run_householder_qr(ctx, m, L.G, L.ldi, L.Qraw, L.qr, st));
+    if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, st));
+    else GELO_TRY(run_householder_qr(ctx, m, L.G, L.ldi, L.Qraw, L.qr, st));
     GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, L.ldi, L.G, L.ldi, GELO_F32, Q_dev, Qt_dev, ld, st));
     return cudaMemcpy2DAsync(G_dev, (size_t)ld * 4, L.G, (size_t)L.ldi * 4, (size_t)m * 4, m,
                              cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;

@@ -60,6 +60,10 @@ struct gelo_ctx {
     cudaEvent_t lane_ready[gelo::kMaxLanes] = {};   // A and A^-1 of the lane are complete
     cudaEvent_t lane_free[gelo::kMaxLanes] = {};    // the products that read them have been enqueued and finished
     cudaEvent_t batch_start = nullptr;
+    // replayable launch graphs of the sampling sequence, one per (lane scratch, kind, size, type)
+    struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3; cudaGraphExec_t exec; long long launches; };
+    std::vector<SampleGraph> graphs;
+    uint64_t* lane_seed_dev = nullptr;              // one seed slot per lane
     // optional per-launch timing (gelo_profile_start / gelo_profile_stop)
     bool prof_on = false;
     std::vector<gelo::ProfEntry> prof;
@@ -109,7 +113,8 @@ int launch_philox_words(gelo_ctx*, uint64_t seed, uint32_t stream_id, uint32_t a
 
 // out[i*ld + j] = (base ? base[i*ld + j] : 0) + scale * z(i*cols + j)
 int launch_gaussian(gelo_ctx*, int rows, int cols, int ld, uint64_t seed, uint32_t stream_id,
-                    uint32_t attempt, float scale, const float* base, float* out, cudaStream_t);
+                    uint32_t attempt, float scale, const float* base, float* out, cudaStream_t,
+                    const uint64_t* seed_dev = nullptr);
 
 // ---- fp32 SIMT GEMM ----------------------------------------------------------------
 
@@ -154,6 +159,7 @@ struct QrScratch {       // all fp32
     float* T = nullptr;  // ceil(m / kPanel) blocks of kPanel x kPanel
     float* Wp = nullptr; // kMaxSlabs x kPanel x ld partial products
     float* W2 = nullptr; // kPanel x ld
+    float* T128 = nullptr; // ceil(m / 128) blocks of 128 x 128: triangular factors of the outer blocks
 };
 size_t qr_scratch_bytes(int m, int ld);
 QrScratch carve_qr(Arena&, int m, int ld);
@@ -161,6 +167,9 @@ QrScratch carve_qr(Arena&, int m, int ld);
 // writes the orthogonal factor Q with G = Q R.  The caller flips column j of Q where
 // R_jj < 0 (launch_finish_mixing with sign_diag = R) to reach the unique factor.
 int run_householder_qr(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, cudaStream_t);
+struct TcScratch;
+// Same factorisation with 128-column outer blocks whose updates run on the tensor cores in split precision.
+int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, cudaStream_t);
 
 struct LuScratch {
     float* M = nullptr;   // m x ld working copy

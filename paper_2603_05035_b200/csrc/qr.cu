@@ -348,6 +348,47 @@ __global__ void set_identity_kernel(float* __restrict__ Q, int ld, int m)
     }
 }
 
+
+// Triangular factor of an outer block from the factors of its 32-column panels:
+//   (I - V1 T1 V1^T)(I - V2 T2 V2^T) = I - [V1 V2] [[T1, -T1 (V1^T V2) T2], [0, T2]] [V1 V2]^T,
+// applied panel after panel.  S = V^T V of the whole block (128 x 128, stride 128); T32: the panels' factors.
+__global__ void __launch_bounds__(256)
+t_merge_kernel(const float* __restrict__ S, const float* __restrict__ T32, int ob, float* __restrict__ T128)
+{
+    __shared__ float x_s[96][NB + 1];
+    __shared__ float tk_s[NB][NB + 1];
+    const int tid = threadIdx.x;
+    for (int idx = tid; idx < 128 * 128; idx += 256) T128[idx] = 0.0f;
+    __syncthreads();
+    const int nsub = (ob + NB - 1) / NB;
+    for (int k = 0; k < nsub; ++k) {
+        for (int idx = tid; idx < NB * NB; idx += 256) {
+            const int a = idx / NB, b = idx % NB;
+            const float t = T32[(size_t)k * NB * NB + idx];
+            tk_s[a][b] = t;
+            T128[(size_t)(k * NB + a) * 128 + k * NB + b] = t;
+        }
+        __syncthreads();
+        const int rows = k * NB;                    // rows of the already merged part
+        // X = S[0:rows, k*32 : k*32+32] * T_k
+        for (int idx = tid; idx < rows * NB; idx += 256) {
+            const int r = idx / NB, cc = idx % NB;
+            float acc = 0.0f;
+            for (int b = 0; b <= cc; ++b) acc = fmaf(S[(size_t)r * 128 + k * NB + b], tk_s[b][cc], acc);
+            x_s[r][cc] = acc;
+        }
+        __syncthreads();
+        // T128[0:rows, k*32 : k*32+32] = -T128[0:rows, 0:rows] * X   (upper triangular left factor)
+        for (int idx = tid; idx < rows * NB; idx += 256) {
+            const int r = idx / NB, cc = idx % NB;
+            float acc = 0.0f;
+            for (int q = r; q < rows; ++q) acc = fmaf(T128[(size_t)r * 128 + q], x_s[q][cc], acc);
+            T128[(size_t)r * 128 + k * NB + cc] = -acc;
+        }
+        __syncthreads();
+    }
+}
+
 }  // namespace
 
 size_t qr_scratch_bytes(int m, int ld)
@@ -364,6 +405,7 @@ QrScratch carve_qr(Arena& a, int m, int ld)
     s.T = static_cast<float*>(a.take((size_t)ceil_div(m, NB) * NB * NB * sizeof(float)));
     s.Wp = static_cast<float*>(a.take((size_t)kMaxSlabs * NB * ld * sizeof(float)));
     s.W2 = static_cast<float*>(a.take((size_t)NB * ld * sizeof(float)));
+    s.T128 = static_cast<float*>(a.take((size_t)ceil_div(m, 128) * 128 * 128 * sizeof(float)));
     return s;
 }
 
@@ -395,6 +437,75 @@ int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const Q
         // Q[j0:, j0:] <- (I - V T V^T) Q[j0:, j0:]
         GELO_TRY(launch_vtc(ctx, Vp, ld, jb, C, ld, nr, nr, Tp, false, s.Wp, s.W2, ld, st));
         GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, nr, jb, st));
+    }
+    return GELO_OK;
+}
+
+int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const QrScratch& s, const TcScratch& tc,
+                          cudaStream_t st)
+{
+    // reflector entries above a panel's first row are read (as zeros) by the block-level products
+    GELO_CUDA_OK(cudaMemsetAsync(s.V, 0, (size_t)m * ld * sizeof(float), st));
+    const int nblocks = ceil_div(m, kOuter);
+
+    // One outer-block transformation C <- (I - V Top V^T) C on the tensor cores, Top = T^T or T.
+    auto block_apply = [&](int b0, int ob, float* C, int nc, bool transpose_t) -> int {
+        const int nr = m - b0;
+        const int nc8 = (nc + 7) & ~7;
+        const float* Vb = s.V + (size_t)b0 * ld + b0;
+        const float* Tb = s.T128 + (size_t)(b0 / kOuter) * 128 * 128;
+        GELO_TRY(launch_split(ctx, C, ld, nr, nc, tc.big[0], tc.big[1], ld, false, st));
+        GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panA[0], tc.panA[1], kOuter, false, st));
+        GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panAt[0], tc.panAt[1], ld, true, st));
+        GELO_TRY(launch_split(ctx, Tb, 128, ob, ob, tc.tt[0], tc.tt[1], kOuter, transpose_t, st));
+        // W = V^T C
+        GELO_TRY(launch_gemm_tc_split(ctx, ob, nc8, nr, tc.panAt[0], tc.panAt[1], ld, tc.big[0], tc.big[1], ld, nullptr, 0,
+                                      tc.rowB[0], tc.rowB[1], ld, true, st));
+        // W2 = Top W
+        GELO_TRY(launch_gemm_tc_split(ctx, ob, nc8, ob, tc.tt[0], tc.tt[1], kOuter, tc.rowB[0], tc.rowB[1], ld, nullptr, 0,
+                                      tc.rowB2[0], tc.rowB2[1], ld, false, st));
+        // C -= V W2
+        return launch_gemm_tc_split(ctx, nr, nc, ob, tc.panA[0], tc.panA[1], kOuter, tc.rowB2[0], tc.rowB2[1], ld, C, ld,
+                                    nullptr, nullptr, 0, false, st);
+    };
+
+    // ---- factorisation ----
+    for (int blk = 0; blk < nblocks; ++blk) {
+        const int b0 = blk * kOuter;
+        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
+        const int bend = b0 + ob;
+        for (int j0 = b0; j0 < bend; j0 += NB) {
+            const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
+            float* Tp = s.T + (size_t)(j0 / NB) * NB * NB;
+            GELO_TRY(launch_qr_panel(ctx, R, ld, m, j0, jb, s.V, Tp, st));
+            const int ncb = bend - (j0 + jb), nr = m - j0;
+            if (ncb > 0) {
+                float* C = R + (size_t)j0 * ld + j0 + jb;
+                const float* Vp = s.V + (size_t)j0 * ld + j0;
+                GELO_TRY(launch_vtc(ctx, Vp, ld, jb, C, ld, nr, ncb, Tp, true, s.Wp, s.W2, ld, st));
+                GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, ncb, jb, st));
+            }
+        }
+        // block factor: Gram of the block's reflectors, then the merge of the panel factors
+        const float* Vb = s.V + (size_t)b0 * ld + b0;
+        for (int a = 0; a * NB < ob; ++a) {
+            const int jb = (ob - a * NB < NB) ? (ob - a * NB) : NB;
+            GELO_TRY(launch_vtc(ctx, Vb + a * NB, ld, jb, Vb, ld, m - b0, ob, nullptr, false, s.Wp, tc.gram + (size_t)a * NB * 128,
+                                128, st));
+        }
+        float* Tb = s.T128 + (size_t)blk * 128 * 128;
+        t_merge_kernel<<<1, 256, 0, st>>>(tc.gram, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
+        GELO_TRY(after_launch(ctx));
+        const int nc = m - bend;
+        if (nc > 0) GELO_TRY(block_apply(b0, ob, R + (size_t)b0 * ld + bend, nc, true));
+    }
+    // ---- accumulate Q backwards from the identity ----
+    set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
+    GELO_TRY(after_launch(ctx));
+    for (int blk = nblocks - 1; blk >= 0; --blk) {
+        const int b0 = blk * kOuter;
+        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
+        GELO_TRY(block_apply(b0, ob, Q + (size_t)b0 * ld + b0, m - b0, false));
     }
     return GELO_OK;
 }

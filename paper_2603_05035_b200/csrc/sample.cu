@@ -26,10 +26,12 @@ __global__ void philox_words_kernel(uint64_t seed, uint32_t stream_id, uint32_t 
     }
 }
 
-__global__ void gaussian_kernel(int rows, int cols, int ld, uint64_t seed, uint32_t stream_id,
-                                uint32_t attempt, float scale, const float* __restrict__ base,
+__global__ void gaussian_kernel(int rows, int cols, int ld, uint64_t seed_value, const uint64_t* __restrict__ seed_ptr,
+                                uint32_t stream_id, uint32_t attempt, float scale, const float* __restrict__ base,
                                 float* __restrict__ out)
 {
+    // a replayed launch graph cannot change by-value arguments, so the seed may come from device memory
+    const uint64_t seed = seed_ptr ? *seed_ptr : seed_value;
     const uint64_t total = (uint64_t)rows * (uint64_t)cols;
     const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t e0 = q << 2;
@@ -74,14 +76,15 @@ int launch_philox_words(gelo_ctx* ctx, uint64_t seed, uint32_t stream_id, uint32
 }
 
 int launch_gaussian(gelo_ctx* ctx, int rows, int cols, int ld, uint64_t seed, uint32_t stream_id,
-                    uint32_t attempt, float scale, const float* base, float* out, cudaStream_t st)
+                    uint32_t attempt, float scale, const float* base, float* out, cudaStream_t st,
+                    const uint64_t* seed_dev)
 {
     const uint64_t total = (uint64_t)rows * (uint64_t)cols;
     if (total == 0) return GELO_OK;
     const unsigned threads = 256;
     const uint64_t grid = ((total + 3) / 4 + threads - 1) / threads;
     if (grid > 0x7fffffffull) return GELO_ERR_INVALID;
-    gaussian_kernel<<<(unsigned)grid, threads, 0, st>>>(rows, cols, ld, seed, stream_id, attempt, scale, base, out);
+    gaussian_kernel<<<(unsigned)grid, threads, 0, st>>>(rows, cols, ld, seed, seed_dev, stream_id, attempt, scale, base, out);
     return after_launch(ctx);
 }
 

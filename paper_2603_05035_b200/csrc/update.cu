@@ -127,7 +127,7 @@ w_reduce_kernel(const float* __restrict__ Wp, int ldw, int slabs, int nc, const 
     const int l = tid & 31, g = tid >> 5;
     for (int idx = tid; idx < NB * NB; idx += 256) {
         const int a = idx / NB, b = idx % NB;
-        t_s[a][b] = transpose_t ? T[b * NB + a] : T[a * NB + b];
+        t_s[a][b] = !T ? (a == b ? 1.0f : 0.0f) : (transpose_t ? T[b * NB + a] : T[a * NB + b]);   // no T: identity
     }
     const int col = blockIdx.x * 32 + l;
 #pragma unroll

@@ -451,3 +451,24 @@ def test_lu_inverse_tensor_core_blocks(oracle, m):
     assert np.linalg.norm(A64 @ x - np.eye(m)) / np.sqrt(m) <= 1e-3
     assert c.last_status() == binding.OK
     c.close()
+
+
+@pytest.mark.parametrize("m", [100, 130, 257, 512, 1000])
+def test_householder_qr_tensor_core_blocks(oracle, m):
+    c = make_ctx(m, 0, 8, 24, "f32")
+    c.set_level3(2)
+    ld = c.mixing_ld(m)
+    G64 = oracle.gaussian(500 + m, 0, 0, m, m).astype(np.float32).astype(np.float64)
+    G = padded(m, ld, torch.float32); G[:, :m] = dev(G64)
+    Q = padded(m, ld, torch.float32)
+    c.qr_orthogonal(m, G, ld, Q)
+    q = f64(Q[:, :m]); r = np.triu(f64(G[:, :m]))
+    s = np.where(np.diag(r) < 0, -1.0, 1.0)
+    # split-precision products (16 significand bits per operand): defects of a few 1e-5, against 1.6e-3 from
+    # rounding A to bf16 afterwards
+    assert np.linalg.norm(q.T @ q - np.eye(m)) / np.sqrt(m) <= 2e-4
+    assert np.linalg.norm(q @ (r.T * s).T - G64) / np.linalg.norm(G64) <= 2e-4
+    q_ref, _ = oracle.householder_qr(G64)
+    assert np.all(np.sum(q * q_ref, axis=0)[: max(1, m // 2)] > 1 - 2e-3)
+    assert c.last_status() == binding.OK
+    c.close()
