@@ -76,6 +76,7 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
 bool carve_ctx(gelo_ctx* ctx, int n, int k, int d, int p, int dtype, bool host_staging, Layout* out)
 {
     if (!ctx->ws) return false;
+    ctx->chain_valid = false;      // a single call reuses scratch that a later batch must not race with
     Arena a;
     a.base = static_cast<char*>(ctx->ws);
     a.cap = ctx->ws_bytes;
@@ -278,13 +279,20 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     const bool split = K[0] != nullptr;
     const size_t third = (size_t)n * (p / 3) * es;
 
-    GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
-    for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaStreamWaitEvent(ctx->lane_stream[l], ctx->batch_start, 0));
+    // Back-to-back batches of the same shape on the same stream keep the lanes running across the seam: each
+    // lane only waits until the products that read its previous pair are done.  Otherwise the lanes start after
+    // everything already enqueued on the caller's stream.
+    const bool chained = ctx->chain_valid && ctx->chain_stream == st && ctx->chain_key == L[D - 1].G &&
+                         ctx->chain_lanes == D;
+    if (!chained) {
+        GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
+        for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaStreamWaitEvent(ctx->lane_stream[l], ctx->batch_start, 0));
+    }
 
     auto enqueue_sample = [&](int i) -> int {
         const int l = i % D;
         cudaStream_t ls = ctx->lane_stream[l];
-        if (i >= D) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->lane_free[l], 0));
+        if (i >= D || chained) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->lane_free[l], 0));
         GELO_TRY(sample_on_lane(ctx, L[l], l, m, kinds[i], seeds[i], dtype, ls));
         GELO_CUDA_OK(cudaEventRecord(ctx->lane_ready[l], ls));
         return GELO_OK;
@@ -318,6 +326,10 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         }
         if (i + D < calls) GELO_TRY(enqueue_sample(i + D));
     }
+    ctx->chain_valid = calls >= D && !ctx->prof_on;
+    ctx->chain_stream = st;
+    ctx->chain_key = L[D - 1].G;
+    ctx->chain_lanes = D;
     if (host) GELO_CUDA_OK(cudaStreamSynchronize(st));
     return GELO_OK;
 }
@@ -426,6 +438,7 @@ int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes)
     if (!ctx) return GELO_ERR_INVALID;
     if (dev_ws && (reinterpret_cast<uintptr_t>(dev_ws) & 255u)) return GELO_ERR_INVALID;
     drop_graphs(ctx);              // recorded launches point into the old workspace
+    ctx->chain_valid = false;
     ctx->ws = dev_ws;
     ctx->ws_bytes = dev_ws ? bytes : 0;
     return GELO_OK;
@@ -572,6 +585,7 @@ int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, floa
     a.cap = ctx->ws_bytes;
     ShieldScratch sh = carve_shield(a, n);
     if (!a.ok) return GELO_ERR_WORKSPACE;
+    ctx->chain_valid = false;
     return run_shield_rows(ctx, H_dev, n, d, k, scale, seed, dtype, S_dev, sh, as_stream(stream));
 }
 

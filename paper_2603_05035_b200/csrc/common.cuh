@@ -19,7 +19,7 @@ constexpr int kPanel = 32;
 // Device status block (ints).  [0]: first device-side error (gelo_status), sticky until read.
 // [1]: verdict of the last condition-number check (1 = accepted).  [2]: detail word.
 constexpr int kStatusWords = 8;
-constexpr int kMaxLanes = 8;
+constexpr int kMaxLanes = 16;
 
 // Kernel classes that the optional per-launch timing distinguishes.
 enum ProfClass { PROF_RANK_UPDATE = 0, PROF_VTC = 1, PROF_GEMM_TC = 2, PROF_QR_PANEL = 3, PROF_LU_PANEL = 4,
@@ -60,6 +60,12 @@ struct gelo_ctx {
     cudaEvent_t lane_ready[gelo::kMaxLanes] = {};   // A and A^-1 of the lane are complete
     cudaEvent_t lane_free[gelo::kMaxLanes] = {};    // the products that read them have been enqueued and finished
     cudaEvent_t batch_start = nullptr;
+    // a batched call may chain onto the previous one (lanes wait for their own lane_free events only) when
+    // nothing else has touched the workspace in between
+    bool chain_valid = false;
+    cudaStream_t chain_stream = nullptr;
+    const void* chain_key = nullptr;
+    int chain_lanes = 0;
     // replayable launch graphs of the sampling sequence, one per (lane scratch, kind, size, type)
     struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3; cudaGraphExec_t exec; long long launches; };
     std::vector<SampleGraph> graphs;
