@@ -146,6 +146,11 @@ bool gemm_tc_supports(const GemmArgs&);
 int launch_gemm_tc_split(gelo_ctx*, int M, int N, int K, const void* Ahi, const void* Alo, int lda,
                          const void* Bhi, const void* Blo, int ldb, float* sub_from, int ldc, void* emit_hi,
                          void* emit_lo, int lde, bool narrow_tiles, cudaStream_t);
+// Same product with the K range cut into `ksplit` slices whose fp32 partial products go to consecutive planes
+// (plane stride in elements); returns the number of slices used in *used.
+int launch_gemm_tc_split_k(gelo_ctx*, int M, int N, int K, const void* Ahi, const void* Alo, int lda, const void* Bhi,
+                           const void* Blo, int ldb, float* planes, size_t plane, int ldp, int ksplit, int* used,
+                           cudaStream_t);
 
 // ---- factorizations -------------------------------------------------------------------
 
@@ -212,8 +217,12 @@ int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* 
 int launch_split(gelo_ctx*, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
                  bool transpose, cudaStream_t);
 
+int launch_sum_split(gelo_ctx*, const float* planes, size_t plane, int parts, int ld, int rows, int cols, void* hi,
+                     void* lo, int ldo, cudaStream_t);
+
 // Scratch of the tensor-core level-3 updates (outer blocks of kOuter columns).
 constexpr int kOuter = 128;
+constexpr int kMaxKSplit = 16;
 struct TcScratch {
     void* panA[2] = {nullptr, nullptr};    // m x kOuter          block column (V or L), hi / lo
     void* panAt[2] = {nullptr, nullptr};   // kOuter x ld         its transpose
@@ -223,7 +232,7 @@ struct TcScratch {
     void* big[2] = {nullptr, nullptr};     // m x ld              trailing matrix as a pair
     float* t128 = nullptr;                 // kOuter x kOuter fp32
     float* gram = nullptr;                 // kOuter x kOuter fp32
-    float* wf32 = nullptr;                 // kOuter x ld fp32
+    float* wf32 = nullptr;                 // kMaxKSplit planes of kOuter x ld fp32 (split-K partial products)
 };
 TcScratch carve_tc(Arena&, int m, int ld);
 // C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores in split precision

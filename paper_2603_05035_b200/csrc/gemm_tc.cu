@@ -49,6 +49,8 @@ struct TcParams {
     int mode;
     void* C0; void* C1; void* C2;   // STORE_*: column-split outputs; SUB_F32: C0 fp32, C1/C2 optional hi/lo; EMIT_SPLIT: C0 hi, C1 lo
     int ldc, csplit, lde;           // lde: row stride of the hi/lo matrices written next to an fp32 C
+    int ksplit, kb_per_split;       // K slices (TC_STORE_F32 only): slice q covers k-blocks [q*kb_per_split, ...) of every segment
+    long long plane;                // and writes plane q of C0 (stride in elements)
     int* status;
 };
 
@@ -180,7 +182,7 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t&
 // One 8-column group of the epilogue: w[G*8 .. G*8+7] are the fp32 accumulator values of row gm, columns
 // gn..gn+7 (G is a template parameter so that the register array is indexed by constants only).
 template <int G>
-__device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int gn, const uint32_t (&w)[32])
+__device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int gn, const uint32_t (&w)[32], int slice)
 {
     const uint32_t v[8] = {w[G * 8 + 0], w[G * 8 + 1], w[G * 8 + 2], w[G * 8 + 3],
                            w[G * 8 + 4], w[G * 8 + 5], w[G * 8 + 6], w[G * 8 + 7]};
@@ -193,7 +195,7 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
         pk.z = pack_bf16(v[4], v[5]); pk.w = pack_bf16(v[6], v[7]);
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
     } else if (prm.mode == TC_STORE_F32) {
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)gm * prm.ldc + gn);
+        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)slice * prm.plane + (size_t)gm * prm.ldc + gn);
         dst[0] = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
         dst[1] = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
     } else if (prm.mode == TC_EMIT_SPLIT) {
@@ -235,7 +237,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
 
     const int m_tiles = (prm.M + BM - 1) / BM;
     const int n_tiles = (prm.N + BN - 1) / BN;
-    const int total_tiles = m_tiles * n_tiles;
+    const int mn_tiles = m_tiles * n_tiles;
+    const int total_tiles = mn_tiles * prm.ksplit;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -260,15 +263,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int m0 = (tile % m_tiles) * BM;
-                const int n0 = (tile / m_tiles) * BN;
+                const int mn = tile % mn_tiles, slice = tile / mn_tiles;
+                const int m0 = (mn % m_tiles) * BM;
+                const int n0 = (mn / m_tiles) * BN;
 #pragma unroll
                 for (int sg = 0; sg < 3; ++sg) {              // constant indices keep the parameters out of local memory
                     if (sg >= prm.nseg || !ok) break;
                     const TcSegment seg = prm.seg[sg];
                     const CUtensorMap* ma = seg.a_sel ? &map_a1 : &map_a0;
                     const CUtensorMap* mb = seg.b_sel ? &map_b1 : &map_b0;
-                    for (int kb = 0; kb < seg.kb; ++kb, ++it) {
+                    const int kb_lo = slice * prm.kb_per_split;
+                    const int kb_hi = min(seg.kb, kb_lo + prm.kb_per_split);
+                    for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1u;
                         if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
@@ -287,13 +293,18 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            int kb_total = 0;
-#pragma unroll
-            for (int sg = 0; sg < 3; ++sg)
-                if (sg < prm.nseg) kb_total += prm.seg[sg].kb;
             uint32_t it = 0, acc_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
+                const int slice = tile / mn_tiles;
+                int kb_total = 0;
+#pragma unroll
+                for (int sg = 0; sg < 3; ++sg)
+                    if (sg < prm.nseg) {
+                        const int kb_lo = slice * prm.kb_per_split;
+                        const int kb_hi = min(prm.seg[sg].kb, kb_lo + prm.kb_per_split);
+                        kb_total += max(0, kb_hi - kb_lo);
+                    }
                 const int a = acc_it % kAccStages;
                 const uint32_t aph = (acc_it / kAccStages) & 1u;
                 if (!mbar_wait(acc_empty_bar(a), aph ^ 1u, abort_flag)) { ok = false; break; }
@@ -331,8 +342,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
             const int a = acc_it % kAccStages;
             const uint32_t aph = (acc_it / kAccStages) & 1u;
-            const int m0 = (tile % m_tiles) * BM;
-            const int n0 = (tile / m_tiles) * BN;
+            const int mn = tile % mn_tiles, slice = tile / mn_tiles;
+            const int m0 = (mn % m_tiles) * BM;
+            const int n0 = (mn / m_tiles) * BN;
             const int gm = m0 + quarter * 32 + lane;
             const bool row_ok = gm < prm.M;
             if (kStaging && prm.mode == TC_SUB_F32) {
@@ -377,10 +389,10 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     tc_ld_wait();
                     if (row_ok) {
                         const int gn = n0 + c;
-                        if (gn < prm.N) epilogue_group<0>(prm, gm, gn, v);
-                        if (gn + 8 < prm.N) epilogue_group<1>(prm, gm, gn + 8, v);
-                        if (gn + 16 < prm.N) epilogue_group<2>(prm, gm, gn + 16, v);
-                        if (gn + 24 < prm.N) epilogue_group<3>(prm, gm, gn + 24, v);
+                        if (gn < prm.N) epilogue_group<0>(prm, gm, gn, v, slice);
+                        if (gn + 8 < prm.N) epilogue_group<1>(prm, gm, gn + 8, v, slice);
+                        if (gn + 16 < prm.N) epilogue_group<2>(prm, gm, gn + 16, v, slice);
+                        if (gn + 24 < prm.N) epilogue_group<3>(prm, gm, gn + 24, v, slice);
                     }
                 }
             }
@@ -436,7 +448,7 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
                                           (int)Cfg::kSmemBytes));
         attr_done[ctx->device] = true;
     }
-    const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN);
+    const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN) * p.ksplit;
     const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
@@ -499,6 +511,7 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
         p.seg[1] = TcSegment{0, 1, a_k0, a_k0 - g.b_split /* <= 0: rows above S read as zero */,
                              ceil_div(g.K - a_k0, BK)};
     }
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
     p.mode = TC_STORE_BF16;
     p.C0 = g.C[0]; p.C1 = g.C[g.nsplit > 1 ? 1 : 0]; p.C2 = g.C[g.nsplit > 2 ? 2 : 0];
     p.ldc = g.ldc; p.csplit = g.N / g.nsplit; p.lde = 0;
@@ -537,6 +550,7 @@ int launch_gemm_tc_split(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, co
     p.seg[2] = TcSegment{1, 0, 0, 0, kb};
     p.status = ctx->status_dev;
     p.csplit = N;
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
     CUtensorMap mc = a0;
     if (sub_from) {
         if (emit_hi) return GELO_ERR_UNSUPPORTED;
@@ -551,6 +565,42 @@ int launch_gemm_tc_split(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, co
     if (sub_from) return launch_tiles<256, 3, true>(ctx, a0, a1, b0, b1, mc, p, flops, st);
     if (narrow_tiles) return launch_tiles<64, 4, false>(ctx, a0, a1, b0, b1, mc, p, flops, st);
     return launch_tiles<256, 4, false>(ctx, a0, a1, b0, b1, mc, p, flops, st);
+}
+
+
+int launch_gemm_tc_split_k(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, const void* Alo, int lda, const void* Bhi,
+                           const void* Blo, int ldb, float* planes, size_t plane, int ldp, int ksplit, int* used,
+                           cudaStream_t st)
+{
+    if (used) *used = 0;
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if ((lda % 8) || (ldb % 8) || (N % 8) || (ldp % 4) || !aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) ||
+        !aligned16(Blo) || !aligned16(planes) || (plane % 4) || ksplit < 1)
+        return GELO_ERR_INVALID;
+    CUtensorMap a0, a1, b0, b1;
+    if (!make_map(ctx, &a0, Ahi, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM) ||
+        !make_map(ctx, &a1, Alo, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM) ||
+        !make_map(ctx, &b0, Bhi, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 64, BK) ||
+        !make_map(ctx, &b1, Blo, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 64, BK))
+        return GELO_ERR_CUDA;
+    const int kb = ceil_div(K, BK);
+    if (ksplit > kb) ksplit = kb;
+    const int per = ceil_div(kb, ksplit);
+    ksplit = ceil_div(kb, per);                    // no empty slice
+    TcParams p = {};
+    p.M = M; p.N = N;
+    p.nseg = 3;
+    p.seg[0] = TcSegment{0, 0, 0, 0, kb};
+    p.seg[1] = TcSegment{0, 1, 0, 0, kb};
+    p.seg[2] = TcSegment{1, 0, 0, 0, kb};
+    p.status = ctx->status_dev;
+    p.csplit = N;
+    p.mode = TC_STORE_F32;
+    p.C0 = planes; p.ldc = ldp; p.lde = 0;
+    p.ksplit = ksplit; p.kb_per_split = per; p.plane = (long long)plane;
+    if (used) *used = ksplit;
+    return launch_tiles<256, 4, false>(ctx, a0, a1, b0, b1, a0, p, 6.0 * M * (double)N * K, st);
 }
 
 }  // namespace gelo

@@ -53,15 +53,63 @@ __global__ void __launch_bounds__(256) convert_kernel(int m, const TS* __restric
 // hi = bf16(x), lo = bf16(x - hi) for a rows x cols block (fp32, stride lds) -> bf16 pair (stride ldo);
 // with T the pair is written transposed (cols x rows, stride ldo) through a shared-memory tile.
 __global__ void __launch_bounds__(256) split_kernel(const float* __restrict__ src, int lds, int rows, int cols,
-                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int ldo)
+                                                    __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int ldo,
+                                                    int vec)
 {
-    const int c = blockIdx.x * 256 + threadIdx.x;
+    // grid-stride over rows; a thread converts four consecutive columns (16-byte load, two 8-byte stores)
+    const int c4 = (blockIdx.x * 256 + threadIdx.x) * 4;
+    if (c4 >= cols) return;
+    for (int r = blockIdx.y; r < rows; r += gridDim.y) {
+        const float* p = src + (size_t)r * lds + c4;
+        float x[4];
+        if (vec && c4 + 3 < cols) {
+            const float4 t = *reinterpret_cast<const float4*>(p);
+            x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) x[j] = (c4 + j < cols) ? p[j] : 0.0f;
+        }
+        __nv_bfloat16 h[4], l[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            h[j] = __float2bfloat16_rn(x[j]);
+            l[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
+        }
+        __nv_bfloat16* ph = hi + (size_t)r * ldo + c4;
+        __nv_bfloat16* pl = lo + (size_t)r * ldo + c4;
+        if (vec && c4 + 3 < cols) {
+            *reinterpret_cast<uint2*>(ph) = *reinterpret_cast<const uint2*>(h);
+            *reinterpret_cast<uint2*>(pl) = *reinterpret_cast<const uint2*>(l);
+        } else {
+#pragma unroll
+            for (int j = 0; j < 4; ++j)
+                if (c4 + j < cols) { ph[j] = h[j]; pl[j] = l[j]; }
+        }
+    }
+}
+
+// hi/lo pair of the sum of `parts` fp32 planes (fixed order): the second half of a split-K product.
+__global__ void __launch_bounds__(256) sum_split_kernel(const float* __restrict__ planes, size_t plane, int parts,
+                                                        int ld, int rows, int cols, __nv_bfloat16* __restrict__ hi,
+                                                        __nv_bfloat16* __restrict__ lo, int ldo)
+{
+    const int c4 = (blockIdx.x * 256 + threadIdx.x) * 4;
     const int r = blockIdx.y;
-    if (c >= cols) return;
-    const float x = src[(size_t)r * lds + c];
-    const __nv_bfloat16 h = __float2bfloat16_rn(x);
-    hi[(size_t)r * ldo + c] = h;
-    lo[(size_t)r * ldo + c] = __float2bfloat16_rn(x - __bfloat162float(h));
+    if (c4 >= cols) return;                                   // cols is a multiple of 8, rows start 16-byte aligned
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < parts; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(planes + q * plane + (size_t)r * ld + c4);
+        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    }
+    const float x[4] = {acc.x, acc.y, acc.z, acc.w};
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+        h[j] = __float2bfloat16_rn(x[j]);
+        l[j] = __float2bfloat16_rn(x[j] - __bfloat162float(h[j]));
+    }
+    *reinterpret_cast<uint2*>(hi + (size_t)r * ldo + c4) = *reinterpret_cast<const uint2*>(h);
+    *reinterpret_cast<uint2*>(lo + (size_t)r * ldo + c4) = *reinterpret_cast<const uint2*>(l);
 }
 
 __global__ void __launch_bounds__(256) split_transpose_kernel(const float* __restrict__ src, int lds, int rows, int cols,
@@ -97,10 +145,25 @@ int launch_split(gelo_ctx* ctx, const float* src, int lds, int rows, int cols, v
         split_transpose_kernel<<<grid, 256, 0, st>>>(src, lds, rows, cols, static_cast<__nv_bfloat16*>(hi),
                                                      static_cast<__nv_bfloat16*>(lo), ldo);
     } else {
-        dim3 grid(ceil_div(cols, 256), rows);
+        const int vec = ((lds & 3) == 0 && (ldo & 3) == 0 && (reinterpret_cast<uintptr_t>(src) & 15u) == 0 &&
+                         (reinterpret_cast<uintptr_t>(hi) & 7u) == 0 && (reinterpret_cast<uintptr_t>(lo) & 7u) == 0) ? 1 : 0;
+        const int gx = ceil_div(cols, 1024);
+        int gy = ceil_div(8 * ctx->sm_count, gx);
+        if (gy > rows) gy = rows;
+        dim3 grid(gx, gy);
         split_kernel<<<grid, 256, 0, st>>>(src, lds, rows, cols, static_cast<__nv_bfloat16*>(hi),
-                                           static_cast<__nv_bfloat16*>(lo), ldo);
+                                           static_cast<__nv_bfloat16*>(lo), ldo, vec);
     }
+    return after_launch(ctx);
+}
+
+int launch_sum_split(gelo_ctx* ctx, const float* planes, size_t plane, int parts, int ld, int rows, int cols, void* hi,
+                     void* lo, int ldo, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return GELO_OK;
+    dim3 grid(ceil_div(cols, 1024), rows);
+    sum_split_kernel<<<grid, 256, 0, st>>>(planes, plane, parts, ld, rows, cols, static_cast<__nv_bfloat16*>(hi),
+                                           static_cast<__nv_bfloat16*>(lo), ldo);
     return after_launch(ctx);
 }
 

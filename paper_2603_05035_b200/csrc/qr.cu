@@ -458,9 +458,16 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
         GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panA[0], tc.panA[1], kOuter, false, st));
         GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panAt[0], tc.panAt[1], ld, true, st));
         GELO_TRY(launch_split(ctx, Tb, 128, ob, ob, tc.tt[0], tc.tt[1], kOuter, transpose_t, st));
-        // W = V^T C
-        GELO_TRY(launch_gemm_tc_split(ctx, ob, nc8, nr, tc.panAt[0], tc.panAt[1], ld, tc.big[0], tc.big[1], ld, nullptr, 0,
-                                      tc.rowB[0], tc.rowB[1], ld, true, st));
+        // W = V^T C: a long, thin product, so the rows are cut into slices whose partial products are summed in a
+        // fixed order by the kernel that also forms the (high, low) pair
+        const int n_tiles = ceil_div(nc8, 256);
+        int want = ceil_div(2 * ctx->sm_count, n_tiles);
+        if (want > kMaxKSplit) want = kMaxKSplit;
+        int used = 0;
+        const size_t plane = (size_t)kOuter * ld;
+        GELO_TRY(launch_gemm_tc_split_k(ctx, ob, nc8, nr, tc.panAt[0], tc.panAt[1], ld, tc.big[0], tc.big[1], ld, tc.wf32,
+                                        plane, ld, want, &used, st));
+        GELO_TRY(launch_sum_split(ctx, tc.wf32, plane, used, ld, ob, nc8, tc.rowB[0], tc.rowB[1], ld, st));
         // W2 = Top W
         GELO_TRY(launch_gemm_tc_split(ctx, ob, nc8, ob, tc.tt[0], tc.tt[1], kOuter, tc.rowB[0], tc.rowB[1], ld, nullptr, 0,
                                       tc.rowB2[0], tc.rowB2[1], ld, false, st));

@@ -271,7 +271,7 @@ TcScratch carve_tc(Arena& a, int m, int ld)
     }
     t.t128 = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
     t.gram = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
-    t.wf32 = static_cast<float*>(a.take((size_t)kOuter * ld * 4));
+    t.wf32 = static_cast<float*>(a.take((size_t)kMaxKSplit * kOuter * ld * 4));
     return t;
 }
 
