@@ -185,6 +185,7 @@ def run_ours(args):
 
     ctx = gelo.Context(local_rank)
     ctx.set_lanes(args.lanes)
+    ctx.set_level3(args.level3)
     ctx.ensure_batch_workspace(n, k, d, p, w.dtype, args.lanes)
     # replicas draw different inputs and mixing seeds
     base = rank * 1000
@@ -378,6 +379,8 @@ def main():
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--lanes", type=int, default=16, help="concurrent sampling lanes of the batched call (1..16)")
+    ap.add_argument("--level3", type=int, default=0, choices=[0, 1, 2],
+                    help="factorisation updates: 0 auto (tensor cores for bf16), 1 fp32 FMA, 2 tensor cores")
     ap.add_argument("--calls", type=int, default=0, help="projection calls per step (default: the workload's 32)")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed sweeps (for profiler launch lists)")

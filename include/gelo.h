@@ -245,7 +245,7 @@ int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_h
                                 void* const* Q_host, void* const* K_host, void* const* V_host,
                                 void* stream);
 
-/* Number of concurrent sampling lanes of the batched calls (1..16, default 4) and the workspace
+/* Number of concurrent sampling lanes of the batched calls (1..32, default 4) and the workspace
  * they need.  0 bytes if an argument is invalid. */
 int gelo_set_lanes(gelo_ctx* ctx, int lanes);
 size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lanes);

@@ -19,7 +19,7 @@ constexpr int kPanel = 32;
 // Device status block (ints).  [0]: first device-side error (gelo_status), sticky until read.
 // [1]: verdict of the last condition-number check (1 = accepted).  [2]: detail word.
 constexpr int kStatusWords = 8;
-constexpr int kMaxLanes = 16;
+constexpr int kMaxLanes = 32;
 
 // Kernel classes that the optional per-launch timing distinguishes.
 enum ProfClass { PROF_RANK_UPDATE = 0, PROF_VTC = 1, PROF_GEMM_TC = 2, PROF_QR_PANEL = 3, PROF_LU_PANEL = 4,
