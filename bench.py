@@ -33,9 +33,9 @@ if ROOT not in sys.path:
 METRIC = "obfuscated-QKV tokens/s at Llama-2-7B shapes"
 UNIT = "tokens/s"
 WORKLOAD = "prefill_bf16"
-# DRAM bytes per launch of a kernel class (dram__bytes_read.sum + dram__bytes_write.sum from one ncu capture,
-# see profiles/); None until counters have been taken for the current kernel.
-TRAFFIC = {}
+# DRAM bytes over algorithmic bytes of the panel kernels, from one ncu capture (profiles/qr_panel_cluster_kernel_*):
+# the capture ran a panel of 3300 rows; traffic scales with the rows, so other panel heights use the same ratio.
+PANEL_TRAFFIC_RATIO = 0.49
 
 
 def _peaks():
@@ -323,17 +323,37 @@ def run_ours(args):
     if rank == 0:
         es = 2 if w.dtype == "bf16" else 4
         dk = kernels[dominant]
-        if dk["unit"] == "TFLOP/s":
-            peak, bound, src = peaks["bf16_tflops"], "tensor", peaks["source"] + " (burst bf16 GEMM)"
+        # FP32 FMA peak of the whole GPU: 148 SMs x 128 lanes x 2 flop x 1.965 GHz (max SM clock)
+        alu_peak = 148 * 128 * 2 * 1.965e9 / 1e12
+        descr = {"rank_update": "rank_update_kernel: C -= A B inside the QR / LU outer blocks",
+                 "vtc": "vtc_partial_kernel: V^T C inside the QR outer blocks",
+                 "gemm_tc": "gemm_tc_kernel: tcgen05 GEMM (mix / project / unmix and the level-3 QR / LU updates)",
+                 "qr_panel": "qr_panel_cluster_kernel: 32-column Householder panel in registers across a cluster of <= 8 CTAs",
+                 "lu_panel": "lu_panel_cluster_kernel: 32-column pivoted LU panel in registers across a cluster of <= 8 CTAs"}
+        roofline = {"kernel": descr[dominant], "achieved": dk["achieved"], "unit": dk["unit"],
+                    "avg_launch_us": dk["avg_us"], "launches_timed": dk["launches"], "traffic": None}
+        if dominant in ("qr_panel", "lu_panel"):
+            per_flop = 2.0 if dominant == "qr_panel" else 1.0
+            avg_rows = prof[dominant]["work"] / prof[dominant]["launches"] / (per_flop * 32 * 32)
+            roofline.update({"bound": "alu", "peak": alu_peak, "frac": dk["achieved"] / alu_peak,
+                             "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz",
+                             "sms_used": 8, "frac_of_sms_used": dk["achieved"] / (alu_peak * 8 / 148),
+                             "note": "latency-bound by design: 33 dependent column steps per launch on one cluster; "
+                                     "other lanes' kernels use the remaining SMs concurrently",
+                             # ncu: 0.41 MB DRAM per launch against 0.85 MB algorithmic (8 B x rows x 32) at rows = 3300
+                             "traffic": PANEL_TRAFFIC_RATIO * 8.0 * avg_rows * 32})
+        elif dk["unit"] == "TFLOP/s":
+            roofline.update({"bound": "tensor", "peak": peaks["bf16_tflops"], "frac": dk["achieved"] / peaks["bf16_tflops"],
+                             "peak_source": peaks["source"] + " (burst bf16 GEMM)"})
         else:
-            peak, bound, src = peaks["hbm_gbs"], "hbm", peaks["source"] + " (copy bandwidth)"
-        descr = {"rank_update": "rank_update_kernel: C -= A B with 32-column panels in the QR / LU trailing updates",
-                 "vtc": "vtc_partial_kernel: V^T C of the QR trailing updates",
-                 "gemm_tc": "gemm_tc_kernel: tcgen05 bf16 GEMM of mix / project / unmix",
-                 "qr_panel": "qr_panel_cluster_kernel", "lu_panel": "lu_panel_cluster_kernel"}[dominant]
-        roofline = {"kernel": descr, "bound": bound, "achieved": dk["achieved"], "peak": peak, "unit": dk["unit"],
-                    "frac": dk["achieved"] / peak, "peak_source": src, "avg_launch_us": dk["avg_us"],
-                    "launches_timed": dk["launches"], "traffic": TRAFFIC.get(dominant)}
+            roofline.update({"bound": "hbm", "peak": peaks["hbm_gbs"], "frac": dk["achieved"] / peaks["hbm_gbs"],
+                             "peak_source": peaks["source"] + " (copy bandwidth)"})
+        # the projection GEMM on its own (one launch per call), the contraction the paper offloads (Eq. 2)
+        proj_tflops = 2.0 * m * d * p / (stage_ms["project"] * 1e-3) / 1e12
+        projection = {"kernel": "gemm_tc_kernel, Y' = U W", "bound": "tensor", "achieved": proj_tflops,
+                      "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": proj_tflops / peaks["bf16_tflops"],
+                      # ncu: dram read 157.1 MB + write 85.9 MB per launch (algorithmic 241.6 MB)
+                      "traffic": 243.0e6}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
@@ -348,6 +368,7 @@ def run_ours(args):
                     "d2h_bytes_per_step": calls * n * p * es, "calls_timed": e2e_calls},
             "gpu_launches": launches,
             "roofline": roofline,
+            "roofline_projection_gemm": projection,
             "kernels": kernels,
             "stage_ms": {k_: round(v, 4) for k_, v in stage_ms.items()},
             "chain": {"ms": chain_ms, "tflops": chain_flops / (chain_ms * 1e-3) / 1e12,

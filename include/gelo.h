@@ -256,7 +256,7 @@ size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lan
  * bracketed by CUDA events on its own stream.  gelo_profile_stop waits for `stream` and the lane
  * streams and fills out[3 * c + {0, 1, 2}] = {launches, summed milliseconds, summed algorithmic
  * work} for class c: 0 rank-32 update (bytes), 1 V^T C product (bytes), 2 tensor-core GEMM
- * (flops), 3 QR panel (bytes), 4 LU panel (bytes).  `out` holds 15 doubles.  Timing mode creates
+ * (flops), 3 QR panel (flops), 4 LU panel (flops).  `out` holds 15 doubles.  Timing mode creates
  * events per launch; keep it out of measured regions. */
 int gelo_profile_start(gelo_ctx* ctx);
 int gelo_profile_stop(gelo_ctx* ctx, void* stream, double* out);

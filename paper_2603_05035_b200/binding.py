@@ -185,7 +185,7 @@ class Context:
         return need
 
     PROFILE_CLASSES = ("rank_update", "vtc", "gemm_tc", "qr_panel", "lu_panel")
-    PROFILE_UNITS = ("bytes", "bytes", "flops", "bytes", "bytes")
+    PROFILE_UNITS = ("bytes", "bytes", "flops", "flops", "flops")
 
     def profile_start(self):
         self._check(self._lib.gelo_profile_start(self._h), "gelo_profile_start")

@@ -252,7 +252,7 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
     int* sd = ctx->status_dev;
-    ProfScope ps(ctx, PROF_LU_PANEL, 8.0 * rows * (double)jb, st);
+    ProfScope ps(ctx, PROF_LU_PANEL, 1.0 * rows * (double)jb * jb, st);   // flops of the eliminations
     cudaError_t e;
     if (rpt <= 2) e = launch_cluster_lu_panel<2>(cs, st, M, ld, m, j0, jb, ipiv, sd);
     else if (rpt <= 3) e = launch_cluster_lu_panel<3>(cs, st, M, ld, m, j0, jb, ipiv, sd);

@@ -323,7 +323,7 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
     int cs = 1;
     while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
-    ProfScope ps(ctx, PROF_QR_PANEL, 8.0 * rows * (double)jb, st);
+    ProfScope ps(ctx, PROF_QR_PANEL, 2.0 * rows * (double)jb * jb, st);   // flops of the column dots and updates
     cudaError_t e;
     if (rpt <= 2) e = launch_cluster_panel<2>(cs, st, R, ld, m, j0, jb, V, T);
     else if (rpt <= 3) e = launch_cluster_panel<3>(cs, st, R, ld, m, j0, jb, V, T);
