@@ -185,6 +185,9 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
     __shared__ float gram[NB][NB + 1];
     __shared__ float tau_s[NB];
     __shared__ float t_s[NB][NB + 1];
+    __shared__ float coef_s[NB];
+    __shared__ float tw_s[NB];
+    __shared__ float scal_s[2];
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -229,42 +232,50 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
         }
         if (CS > 1) cluster.sync(); else __syncthreads();
 
-        float d_own = 0.0f, d_c = 0.0f;
-        for (int r = 0; r < CS; ++r) { d_own += slot[par][r][lane]; d_c += slot[par][r][csrc]; }
-        if (c > 0 && warp == 0 && lane < c - 1) gram[lane][c - 1] = d_own;
-        if (c == jb) break;
-
-        const float alpha = rowbuf[par][c];
-        const float rj = rowbuf[par][lane];
-        const float sigma = d_c;
-        float beta = alpha, tau = 0.0f, scale = 0.0f;
-        if (sigma > 0.0f) {
-            beta = -copysignf(sqrtf(fmaf(alpha, alpha, sigma)), alpha);
-            tau = (beta - alpha) / beta;
-            scale = 1.0f / (alpha - beta);
+        // ---- warp 0 turns the sums into this column's reflector; everybody else only reads the result ----
+        if (warp == 0) {
+            float d_own = 0.0f;
+            for (int r = 0; r < CS; ++r) d_own += slot[par][r][lane];
+            if (c > 0 && lane < c - 1) gram[lane][c - 1] = d_own;
+            if (c < jb) {
+                const float sigma = __shfl_sync(full, d_own, c);
+                const float alpha = rowbuf[par][c];
+                const float rj = rowbuf[par][lane];
+                float beta = alpha, tau = 0.0f, scale = 0.0f;
+                if (sigma > 0.0f) {
+                    beta = -copysignf(sqrtf(fmaf(alpha, alpha, sigma)), alpha);
+                    tau = (beta - alpha) / beta;
+                    scale = 1.0f / (alpha - beta);
+                }
+                const float wv = (lane > c && col_ok) ? fmaf(scale, d_own, rj) : 0.0f;
+                const float tw = tau * wv;
+                tw_s[lane] = tw;
+                // x <- coef * x_c + (lane == c ? 0 : x):  -tw v for later columns, v itself in column c, nothing before
+                coef_s[lane] = (lane > c) ? -tw * scale : ((lane == c) ? scale : 0.0f);
+                if (lane == 0) { scal_s[0] = scale; scal_s[1] = beta; tau_s[c] = tau; }
+            }
         }
-        const float wv = (lane > c && col_ok) ? fmaf(scale, d_own, rj) : 0.0f;
-        const float tw = tau * wv;
-        if (threadIdx.x == 0) tau_s[c] = tau;
-        // ---- apply H_c; lanes < c gather v_c^T v_lane for T ----
-        g = 0.0f;
+        if (c == jb) break;
+        __syncthreads();
+        const float coef = coef_s[lane];
+        const float scale = scal_s[0];
+        // ---- apply H_c; every lane also gathers x_c^T x_lane (only lanes < c use it: v_c^T v_lane for T) ----
+        float graw = 0.0f;
 #pragma unroll
         for (int i = 1; i < RPT; ++i) {
-            const float v = xc[i] * scale;
-            if (lane > c) x[i] = fmaf(-tw, v, x[i]);
-            else if (lane == c) x[i] = v;
-            else g = fmaf(v, x[i], g);
+            graw = fmaf(xc[i], x[i], graw);
+            x[i] = fmaf(coef, xc[i], (lane == c) ? 0.0f : x[i]);
         }
+        g = 0.0f;
         if (gw > c) {
-            const float v = xc[0] * scale;
-            if (lane > c) x[0] = fmaf(-tw, v, x[0]);
-            else if (lane == c) x[0] = v;
-            else g = fmaf(v, x[0], g);
+            graw = fmaf(xc[0], x[0], graw);
+            x[0] = fmaf(coef, xc[0], (lane == c) ? 0.0f : x[0]);
         } else if (gw == c) {                               // row j itself: v_c(j) = 1
-            if (lane > c) x[0] -= tw;
-            else if (lane == c) x[0] = beta;
-            else g += x[0];
+            g = x[0];
+            if (lane > c) x[0] -= tw_s[lane];
+            else if (lane == c) x[0] = scal_s[1];
         }
+        g = fmaf(scale, graw, g);
     }
 
     // ---- write back: R above / on the diagonal, reflectors below it ----
