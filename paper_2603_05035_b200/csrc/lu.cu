@@ -267,21 +267,54 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     return after_launch(ctx);
 }
 
-// Applies the panel's interchanges (rows j0+c <-> ipiv[j0+c], c = 0..jb-1, in order) to
-// columns [c_lo, c_hi) of X, skipping columns [skip_lo, skip_hi).
-__global__ void swap_rows_kernel(float* __restrict__ X, int ld, int j0, int jb, const int* __restrict__ ipiv,
-                                 int c_lo, int c_hi, int skip_lo, int skip_hi)
+// Applies the interchanges rows j0+c <-> ipiv[j0+c], c = 0 .. jb-1 (in order, jb <= 128) to columns
+// [c_lo, c_hi) of X, skipping columns [skip_lo, skip_hi).  Every CTA first composes the interchanges into a
+// row permutation of the (at most 2 jb) rows they touch -- one warp, table in shared memory -- and then moves
+// 32 columns of those rows through a shared-memory tile: gather from the source rows, scatter to the targets.
+constexpr int kSwapMaxRows = 256;
+
+__global__ void __launch_bounds__(256)
+swap_rows_kernel(float* __restrict__ X, int ld, int j0, int jb, const int* __restrict__ ipiv,
+                 int c_lo, int c_hi, int skip_lo, int skip_hi)
 {
-    const int col = c_lo + blockIdx.x * blockDim.x + threadIdx.x;
-    if (col >= c_hi || (col >= skip_lo && col < skip_hi)) return;
-    for (int c = 0; c < jb; ++c) {
-        const int a = j0 + c, b = ipiv[a];
-        if (a != b) {
-            const float t = X[(size_t)a * ld + col];
-            X[(size_t)a * ld + col] = X[(size_t)b * ld + col];
-            X[(size_t)b * ld + col] = t;
+    __shared__ int pos_s[kSwapMaxRows];       // row that receives ...
+    __shared__ int src_s[kSwapMaxRows];       // ... the content this row had before the interchanges
+    __shared__ int count_s;
+    __shared__ float tile[kSwapMaxRows][33];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    if (warp == 0) {
+        int count = 0;
+        for (int c = 0; c < jb; ++c) {
+            const int a = j0 + c, b = ipiv[a];
+            if (a == b) continue;
+            // table slots of rows a and b (insert identity entries when they are new)
+            int ia = -1, ib = -1;
+            for (int base = 0; base < count; base += 32) {
+                const int e = base + lane;
+                const int p = (e < count) ? pos_s[e] : -1;
+                const unsigned ma = __ballot_sync(0xffffffffu, p == a);
+                const unsigned mb = __ballot_sync(0xffffffffu, p == b);
+                if (ma) ia = base + __ffs(ma) - 1;
+                if (mb) ib = base + __ffs(mb) - 1;
+            }
+            if (ia < 0) { ia = count; if (lane == 0) { pos_s[count] = a; src_s[count] = a; } ++count; }
+            if (ib < 0) { ib = count; if (lane == 0) { pos_s[count] = b; src_s[count] = b; } ++count; }
+            __syncwarp();
+            if (lane == 0) { const int t = src_s[ia]; src_s[ia] = src_s[ib]; src_s[ib] = t; }
+            __syncwarp();
         }
+        if (lane == 0) count_s = count;
     }
+    __syncthreads();
+    const int count = count_s;
+    int col = c_lo + blockIdx.x * 32 + lane;
+    if (col >= skip_lo && col < skip_hi) col = c_hi;          // inactive lane
+    const bool ok = col < c_hi;
+    for (int e = warp; e < count; e += 8)
+        if (ok) tile[e][lane] = X[(size_t)src_s[e] * ld + col];
+    __syncthreads();
+    for (int e = warp; e < count; e += 8)
+        if (ok && src_s[e] != pos_s[e]) X[(size_t)pos_s[e] * ld + col] = tile[e][lane];
 }
 
 // X[i0:i0+ib, c_lo:c_hi) <- L_ii^-1 X (unit lower, forward) or U_ii^-1 X (upper, backward);
@@ -324,6 +357,87 @@ tri_solve_block_kernel(const float* M, int ldm, float* X, int ldx,
 #pragma unroll
     for (int i = 0; i < NB; ++i)
         if (i < ib) X[(size_t)(i0 + i) * ldx + col] = x[i];
+}
+
+// The same solve for a whole outer block (ob <= 128 rows) in one launch: the block's triangle sits transposed in
+// shared memory, every thread owns one column of X (its 128 entries in a shared-memory tile) and works through
+// the four 32-row sub-blocks with the sub-block in registers: first the contributions of the rows already solved
+// (32 independent FMAs per shared-memory value), then the 32 x 32 substitution.
+constexpr int kTri128LtStride = 132;
+constexpr int kTri128SmemBytes = (128 * kTri128LtStride + 128 * 129) * 4;
+
+template <bool UPPER>
+__global__ void __launch_bounds__(128)
+tri_solve128_kernel(const float* M, int ldm, float* X, int ldx, int b0, int ob, int c_lo, int c_hi)
+{
+    extern __shared__ __align__(16) float tsm[];
+    float (*Lt)[kTri128LtStride] = reinterpret_cast<float (*)[kTri128LtStride]>(tsm);   // Lt[t][i] = L[i][t]
+    float (*tile)[129] = reinterpret_cast<float (*)[129]>(tsm + 128 * kTri128LtStride);
+    const int tid = threadIdx.x;
+    const int col = c_lo + blockIdx.x * 128 + tid;
+    const bool ok = col < c_hi;
+    for (int idx = tid; idx < 128 * 128; idx += 128) {
+        const int i = idx >> 7, t = idx & 127;
+        Lt[t][i] = (i < ob && t < ob) ? M[(size_t)(b0 + i) * ldm + b0 + t] : 0.0f;
+    }
+    for (int t = 0; t < 128; ++t) tile[t][tid] = (ok && t < ob) ? X[(size_t)(b0 + t) * ldx + col] : 0.0f;
+    __syncthreads();
+    const int nsub = (ob + NB - 1) / NB;
+    for (int q = 0; q < nsub; ++q) {
+        const int sidx = UPPER ? (nsub - 1 - q) : q;
+        const int r0 = sidx * NB;
+        float x[NB];
+#pragma unroll
+        for (int i = 0; i < NB; ++i) x[i] = tile[r0 + i][tid];
+        const int t_lo = UPPER ? r0 + NB : 0;
+        const int t_hi = UPPER ? nsub * NB : r0;
+        for (int t = t_lo; t < t_hi; ++t) {
+            const float xt = tile[t][tid];
+            const float4* lp = reinterpret_cast<const float4*>(&Lt[t][r0]);
+#pragma unroll
+            for (int i4 = 0; i4 < NB / 4; ++i4) {
+                const float4 l = lp[i4];
+                x[4 * i4 + 0] = fmaf(-l.x, xt, x[4 * i4 + 0]);
+                x[4 * i4 + 1] = fmaf(-l.y, xt, x[4 * i4 + 1]);
+                x[4 * i4 + 2] = fmaf(-l.z, xt, x[4 * i4 + 2]);
+                x[4 * i4 + 3] = fmaf(-l.w, xt, x[4 * i4 + 3]);
+            }
+        }
+        if (!UPPER) {
+#pragma unroll
+            for (int i = 1; i < NB; ++i) {
+                float sacc = x[i];
+#pragma unroll
+                for (int t = 0; t < i; ++t) sacc = fmaf(-Lt[r0 + t][r0 + i], x[t], sacc);
+                x[i] = sacc;
+            }
+        } else {
+#pragma unroll
+            for (int i = NB - 1; i >= 0; --i) {
+                if (r0 + i < ob) {
+                    float sacc = x[i];
+#pragma unroll
+                    for (int t = i + 1; t < NB; ++t) sacc = fmaf(-Lt[r0 + t][r0 + i], x[t], sacc);
+                    x[i] = sacc / Lt[r0 + i][r0 + i];
+                }
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < NB; ++i) tile[r0 + i][tid] = x[i];
+    }
+    if (ok)
+        for (int t = 0; t < ob; ++t) X[(size_t)(b0 + t) * ldx + col] = tile[t][tid];
+}
+
+template <bool UPPER>
+int launch_tri_solve128(gelo_ctx* ctx, const float* M, int ldm, float* X, int ldx, int b0, int ob, int c_lo, int c_hi,
+                        cudaStream_t st)
+{
+    if (c_hi <= c_lo) return GELO_OK;
+    GELO_CUDA_OK(cudaFuncSetAttribute(tri_solve128_kernel<UPPER>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kTri128SmemBytes));
+    tri_solve128_kernel<UPPER><<<ceil_div(c_hi - c_lo, 128), 128, kTri128SmemBytes, st>>>(M, ldm, X, ldx, b0, ob, c_lo, c_hi);
+    return after_launch(ctx);
 }
 
 // perm = the row order produced by the interchanges; X = P (X[i, perm[i]] = 1).
@@ -378,7 +492,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
             const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
             GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
             if (ob > jb) {       // interchanges on the other columns of this block
-                swap_rows_kernel<<<ceil_div(ob, 256), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, b0, bend, j0, j0 + jb);
+                swap_rows_kernel<<<ceil_div(ob, 32), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, b0, bend, j0, j0 + jb);
                 GELO_TRY(after_launch(ctx));
             }
             const int ncb = bend - (j0 + jb);
@@ -390,21 +504,13 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
             }
         }
         if (m > ob) {            // the block's interchanges on everything left and right of it
-            swap_rows_kernel<<<ceil_div(m, 256), 256, 0, st>>>(M, ld, b0, ob, s.ipiv, 0, m, b0, bend);
+            swap_rows_kernel<<<ceil_div(m, 32), 256, 0, st>>>(M, ld, b0, ob, s.ipiv, 0, m, b0, bend);
             GELO_TRY(after_launch(ctx));
         }
         const int nc = m - bend;
         if (nc <= 0) continue;
         // U12 = L11^-1 A12 on the block's row strip
-        for (int i0 = b0; i0 < bend; i0 += NB) {
-            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
-            tri_solve_block_kernel<false><<<ceil_div(nc, 256), 256, 0, st>>>(M, ld, M, ld, i0, ib, bend, m);
-            GELO_TRY(after_launch(ctx));
-            const int rem = bend - (i0 + ib);
-            if (rem > 0)
-                GELO_TRY(launch_rank_update(ctx, M + (size_t)(i0 + ib) * ld + i0, ld, M + (size_t)i0 * ld + bend, ld,
-                                            M + (size_t)(i0 + ib) * ld + bend, ld, rem, nc, ib, st));
-        }
+        GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, M, ld, b0, ob, bend, m, st));
         // A22 -= L21 U12
         GELO_TRY(tc_update_f32(ctx, tc, nc, nc, ob, M + (size_t)bend * ld + b0, ld, M + (size_t)b0 * ld + bend, ld,
                                M + (size_t)bend * ld + bend, ld, st));
@@ -420,15 +526,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
     for (int b0 = 0; b0 < m; b0 += kOuter) {
         const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
         const int bend = b0 + ob;
-        for (int i0 = b0; i0 < bend; i0 += NB) {
-            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
-            tri_solve_block_kernel<false><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);
-            GELO_TRY(after_launch(ctx));
-            const int rem = bend - (i0 + ib);
-            if (rem > 0)
-                GELO_TRY(launch_rank_update(ctx, M + (size_t)(i0 + ib) * ld + i0, ld, X + (size_t)i0 * ld, ld,
-                                            X + (size_t)(i0 + ib) * ld, ld, rem, m, ib, st));
-        }
+        GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
         if (m - bend > 0)
             GELO_TRY(tc_update_f32(ctx, tc, m - bend, m, ob, M + (size_t)bend * ld + b0, ld, X + (size_t)b0 * ld, ld,
                                    X + (size_t)bend * ld, ld, st));
@@ -438,17 +536,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         const int b0 = blk * kOuter;
         const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
         const int bend = b0 + ob;
-        const int nsub = ceil_div(ob, NB);
-        for (int sb = nsub - 1; sb >= 0; --sb) {
-            const int i0 = b0 + sb * NB;
-            const int ib = (bend - i0 < NB) ? (bend - i0) : NB;
-            tri_solve_block_kernel<true><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);
-            GELO_TRY(after_launch(ctx));
-            const int above = i0 - b0;
-            if (above > 0)
-                GELO_TRY(launch_rank_update(ctx, M + (size_t)b0 * ld + i0, ld, X + (size_t)i0 * ld, ld,
-                                            X + (size_t)b0 * ld, ld, above, m, ib, st));
-        }
+        GELO_TRY(launch_tri_solve128<true>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
         if (b0 > 0)
             GELO_TRY(tc_update_f32(ctx, tc, b0, m, ob, M + b0, ld, X + (size_t)b0 * ld, ld, X, ld, st));
     }
@@ -465,7 +553,7 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
         const int j0 = pnl * NB, jb = (m - j0 < NB) ? (m - j0) : NB;
         GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
         if (m > jb) {
-            swap_rows_kernel<<<ceil_div(m, 256), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, 0, m, j0, j0 + jb);
+            swap_rows_kernel<<<ceil_div(m, 32), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, 0, m, j0, j0 + jb);
             GELO_TRY(after_launch(ctx));
         }
         const int nc = m - j0 - jb;

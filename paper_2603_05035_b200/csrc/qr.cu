@@ -360,44 +360,119 @@ __global__ void set_identity_kernel(float* __restrict__ Q, int ld, int m)
 }
 
 
-// Triangular factor of an outer block from the factors of its 32-column panels:
-//   (I - V1 T1 V1^T)(I - V2 T2 V2^T) = I - [V1 V2] [[T1, -T1 (V1^T V2) T2], [0, T2]] [V1 V2]^T,
-// applied panel after panel.  S = V^T V of the whole block (128 x 128, stride 128); T32: the panels' factors.
+// Gram matrix of an outer block's reflectors, S = V^T V (V: nr x ob, ob <= 128), as per-slab partial sums:
+// CTA s accumulates rows [s * kGramRows, ...) in 32-row chunks staged in shared memory (256 threads, 8 x 8
+// outputs each) and writes its 128 x 128 partial to part[s].
+constexpr int kGramRows = 256;
+
 __global__ void __launch_bounds__(256)
-t_merge_kernel(const float* __restrict__ S, const float* __restrict__ T32, int ob, float* __restrict__ T128)
+gram128_kernel(const float* __restrict__ V, int ld, int nr, int ob, float* __restrict__ part)
 {
-    __shared__ float x_s[96][NB + 1];
-    __shared__ float tk_s[NB][NB + 1];
+    __shared__ __align__(16) float vs[32][128 + 4];
     const int tid = threadIdx.x;
-    for (int idx = tid; idx < 128 * 128; idx += 256) T128[idx] = 0.0f;
-    __syncthreads();
-    const int nsub = (ob + NB - 1) / NB;
-    for (int k = 0; k < nsub; ++k) {
-        for (int idx = tid; idx < NB * NB; idx += 256) {
-            const int a = idx / NB, b = idx % NB;
-            const float t = T32[(size_t)k * NB * NB + idx];
-            tk_s[a][b] = t;
-            T128[(size_t)(k * NB + a) * 128 + k * NB + b] = t;
+    const int ty = tid >> 4, tx = tid & 15;
+    const int r0 = blockIdx.x * kGramRows;
+    const int r1 = min(nr, r0 + kGramRows);
+    float acc[8][8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[i][j] = 0.0f;
+    for (int rb = r0; rb < r1; rb += 32) {
+        // 32 rows x 128 columns: thread loads 4 float4 (row = tid / 32 + 8 i, column group = tid % 32)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int rr = (tid >> 5) + 8 * i, c4 = (tid & 31) * 4;
+            const int row = rb + rr;
+            float4 t = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (row < r1) {
+                const float* p = V + (size_t)row * ld + c4;
+                if (c4 + 3 < ob) t = *reinterpret_cast<const float4*>(p);
+                else {
+                    if (c4 + 0 < ob) t.x = p[0];
+                    if (c4 + 1 < ob) t.y = p[1];
+                    if (c4 + 2 < ob) t.z = p[2];
+                }
+            }
+            *reinterpret_cast<float4*>(&vs[rr][c4]) = t;
         }
         __syncthreads();
-        const int rows = k * NB;                    // rows of the already merged part
-        // X = S[0:rows, k*32 : k*32+32] * T_k
-        for (int idx = tid; idx < rows * NB; idx += 256) {
-            const int r = idx / NB, cc = idx % NB;
-            float acc = 0.0f;
-            for (int b = 0; b <= cc; ++b) acc = fmaf(S[(size_t)r * 128 + k * NB + b], tk_s[b][cc], acc);
-            x_s[r][cc] = acc;
-        }
-        __syncthreads();
-        // T128[0:rows, k*32 : k*32+32] = -T128[0:rows, 0:rows] * X   (upper triangular left factor)
-        for (int idx = tid; idx < rows * NB; idx += 256) {
-            const int r = idx / NB, cc = idx % NB;
-            float acc = 0.0f;
-            for (int q = r; q < rows; ++q) acc = fmaf(T128[(size_t)r * 128 + q], x_s[q][cc], acc);
-            T128[(size_t)r * 128 + k * NB + cc] = -acc;
+#pragma unroll 8
+        for (int k = 0; k < 32; ++k) {
+            const float4 a0 = *reinterpret_cast<const float4*>(&vs[k][ty * 4]);
+            const float4 a1 = *reinterpret_cast<const float4*>(&vs[k][ty * 4 + 64]);
+            const float4 b0 = *reinterpret_cast<const float4*>(&vs[k][tx * 4]);
+            const float4 b1 = *reinterpret_cast<const float4*>(&vs[k][tx * 4 + 64]);
+            const float a[8] = {a0.x, a0.y, a0.z, a0.w, a1.x, a1.y, a1.z, a1.w};
+            const float b[8] = {b0.x, b0.y, b0.z, b0.w, b1.x, b1.y, b1.z, b1.w};
+#pragma unroll
+            for (int i = 0; i < 8; ++i)
+#pragma unroll
+                for (int j = 0; j < 8; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
         }
         __syncthreads();
     }
+    float* out = part + (size_t)blockIdx.x * 128 * 128;
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+        const int r = ty * 4 + (i >> 2) * 64 + (i & 3);
+#pragma unroll
+        for (int h = 0; h < 2; ++h)
+            *reinterpret_cast<float4*>(out + (size_t)r * 128 + tx * 4 + h * 64) =
+                make_float4(acc[i][4 * h + 0], acc[i][4 * h + 1], acc[i][4 * h + 2], acc[i][4 * h + 3]);
+    }
+}
+
+// Triangular factor of an outer block from the factors of its 32-column panels:
+//   (I - V1 T1 V1^T)(I - V2 T2 V2^T) = I - [V1 V2] [[T1, -T1 (V1^T V2) T2], [0, T2]] [V1 V2]^T,
+// applied panel after panel.  part: `slabs` partial Gram matrices (summed here in slab order); T32: the panels'
+// factors.  One CTA, everything in shared memory.
+constexpr int kMergeSmemBytes = (2 * 128 * 129 + 96 * 33 + 32 * 33) * 4;
+
+__global__ void __launch_bounds__(1024)
+t_merge_kernel(const float* __restrict__ part, int slabs, const float* __restrict__ T32, int ob, float* __restrict__ T128)
+{
+    extern __shared__ float msm[];
+    float (*S)[129] = reinterpret_cast<float (*)[129]>(msm);
+    float (*Tm)[129] = reinterpret_cast<float (*)[129]>(msm + 128 * 129);
+    float (*x_s)[33] = reinterpret_cast<float (*)[33]>(msm + 2 * 128 * 129);
+    float (*tk_s)[33] = reinterpret_cast<float (*)[33]>(msm + 2 * 128 * 129 + 96 * 33);
+    const int tid = threadIdx.x;
+    for (int idx = tid; idx < 128 * 128; idx += 1024) {
+        float acc = 0.0f;
+        for (int q = 0; q < slabs; ++q) acc += part[(size_t)q * 128 * 128 + idx];
+        S[idx >> 7][idx & 127] = acc;
+        Tm[idx >> 7][idx & 127] = 0.0f;
+    }
+    __syncthreads();
+    const int nsub = (ob + NB - 1) / NB;
+    for (int k = 0; k < nsub; ++k) {
+        {
+            const int a = tid >> 5, b = tid & 31;                   // 1024 threads = one 32 x 32 factor
+            const float t = T32[(size_t)k * NB * NB + tid];
+            tk_s[a][b] = t;
+            Tm[k * NB + a][k * NB + b] = t;
+        }
+        __syncthreads();
+        const int rows = k * NB;                                    // rows of the already merged part
+        // X = S[0:rows, k*32 : k*32+32] * T_k
+        for (int idx = tid; idx < rows * NB; idx += 1024) {
+            const int r = idx >> 5, cc = idx & 31;
+            float acc = 0.0f;
+            for (int b = 0; b <= cc; ++b) acc = fmaf(S[r][k * NB + b], tk_s[b][cc], acc);
+            x_s[r][cc] = acc;
+        }
+        __syncthreads();
+        // T[0:rows, k*32 : k*32+32] = -T[0:rows, 0:rows] * X   (upper triangular left factor)
+        for (int idx = tid; idx < rows * NB; idx += 1024) {
+            const int r = idx >> 5, cc = idx & 31;
+            float acc = 0.0f;
+            for (int q = r; q < rows; ++q) acc = fmaf(Tm[r][q], x_s[q][cc], acc);
+            Tm[r][k * NB + cc] = -acc;
+        }
+        __syncthreads();
+    }
+    for (int idx = tid; idx < 128 * 128; idx += 1024) T128[idx] = Tm[idx >> 7][idx & 127];
 }
 
 }  // namespace
@@ -457,6 +532,7 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
 {
     // reflector entries above a panel's first row are read (as zeros) by the block-level products
     GELO_CUDA_OK(cudaMemsetAsync(s.V, 0, (size_t)m * ld * sizeof(float), st));
+    GELO_CUDA_OK(cudaFuncSetAttribute(t_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemBytes));
     const int nblocks = ceil_div(m, kOuter);
 
     // One outer-block transformation C <- (I - V Top V^T) C on the tensor cores, Top = T^T or T.
@@ -504,15 +580,13 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
                 GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, ncb, jb, st));
             }
         }
-        // block factor: Gram of the block's reflectors, then the merge of the panel factors
+        // block factor: Gram of the block's reflectors (row slabs, summed in order), then the merge of the panel factors
         const float* Vb = s.V + (size_t)b0 * ld + b0;
-        for (int a = 0; a * NB < ob; ++a) {
-            const int jb = (ob - a * NB < NB) ? (ob - a * NB) : NB;
-            GELO_TRY(launch_vtc(ctx, Vb + a * NB, ld, jb, Vb, ld, m - b0, ob, nullptr, false, s.Wp, tc.gram + (size_t)a * NB * 128,
-                                128, st));
-        }
+        const int slabs = ceil_div(m - b0, kGramRows);
+        gram128_kernel<<<slabs, 256, 0, st>>>(Vb, ld, m - b0, ob, tc.gram);
+        GELO_TRY(after_launch(ctx));
         float* Tb = s.T128 + (size_t)blk * 128 * 128;
-        t_merge_kernel<<<1, 256, 0, st>>>(tc.gram, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
+        t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.gram, slabs, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
         GELO_TRY(after_launch(ctx));
         const int nc = m - bend;
         if (nc > 0) GELO_TRY(block_apply(b0, ob, R + (size_t)b0 * ld + bend, nc, true));

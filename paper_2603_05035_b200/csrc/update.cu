@@ -270,7 +270,7 @@ TcScratch carve_tc(Arena& a, int m, int ld)
         t.big[h] = a.take((size_t)m * ld * 2);
     }
     t.t128 = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
-    t.gram = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
+    t.gram = static_cast<float*>(a.take((size_t)(m / 256 + 2) * kOuter * kOuter * 4));   // one partial Gram per 256-row slab
     t.wf32 = static_cast<float*>(a.take((size_t)kMaxKSplit * kOuter * ld * 4));
     return t;
 }
