@@ -632,6 +632,14 @@ int gelo_qkv_offload(gelo_ctx* ctx, const void* H_dev, const void* W_dev, int n,
         return GELO_ERR_INVALID;
     GELO_TRY(check_split(p, Q_dev, K_dev, V_dev));
     DeviceGuard guard(ctx->device);
+    if (kind == GELO_ORTHOGONAL && !ctx->prof_on) {
+        // nothing to verify: run it as a batch of one, which replays the recorded sampling graph on a lane stream
+        const void* H1[1] = { H_dev }; const void* W1[1] = { W_dev };
+        void* Q1[1] = { Q_dev }; void* K1[1] = { K_dev }; void* V1[1] = { V_dev };
+        const int kind1[1] = { kind }; const uint64_t seed1[1] = { seed };
+        return offload_batch_impl(ctx, 1, H1, W1, n, k, d, p, kind1, seed1, shield_scale, dtype, Q1, K1, V1,
+                                  as_stream(stream), false);
+    }
     Layout L;
     if (!carve_ctx(ctx, n, k, d, p, dtype, false, &L)) return GELO_ERR_WORKSPACE;
     return offload_impl(ctx, L, H_dev, W_dev, n, k, d, p, kind, seed, shield_scale, dtype, Q_dev, K_dev, V_dev,

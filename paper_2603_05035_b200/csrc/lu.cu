@@ -376,10 +376,10 @@ tri_solve128_kernel(const float* M, int ldm, float* X, int ldx, int b0, int ob, 
     const int tid = threadIdx.x;
     const int col = c_lo + blockIdx.x * 128 + tid;
     const bool ok = col < c_hi;
-    for (int idx = tid; idx < 128 * 128; idx += 128) {
-        const int i = idx >> 7, t = idx & 127;
-        Lt[t][i] = (i < ob && t < ob) ? M[(size_t)(b0 + i) * ldm + b0 + t] : 0.0f;
-    }
+    // many independent loads in flight: these two fills and the write-back are pure latency otherwise
+#pragma unroll 16
+    for (int i = 0; i < 128; ++i) Lt[tid][i] = (i < ob && tid < ob) ? M[(size_t)(b0 + i) * ldm + b0 + tid] : 0.0f;
+#pragma unroll 16
     for (int t = 0; t < 128; ++t) tile[t][tid] = (ok && t < ob) ? X[(size_t)(b0 + t) * ldx + col] : 0.0f;
     __syncthreads();
     const int nsub = (ob + NB - 1) / NB;
@@ -425,8 +425,11 @@ tri_solve128_kernel(const float* M, int ldm, float* X, int ldx, int b0, int ob, 
 #pragma unroll
         for (int i = 0; i < NB; ++i) tile[r0 + i][tid] = x[i];
     }
-    if (ok)
-        for (int t = 0; t < ob; ++t) X[(size_t)(b0 + t) * ldx + col] = tile[t][tid];
+    if (ok) {
+#pragma unroll 16
+        for (int t = 0; t < 128; ++t)
+            if (t < ob) X[(size_t)(b0 + t) * ldx + col] = tile[t][tid];
+    }
 }
 
 template <bool UPPER>
