@@ -49,6 +49,25 @@ def _peaks():
     return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "source": "fallback"}
 
 
+def max_over_ranks(values, dist=None, device="cpu"):
+    """Element-wise maximum of a list of floats over all ranks (identity without a process group)."""
+    import torch
+    t = torch.tensor([float(v) for v in values], device=device, dtype=torch.float64)
+    if dist is not None and dist.is_initialized() and dist.get_world_size() > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(x) for x in t]
+
+
+def whole_job_rate(units_per_rank: float, world: int, slowest_ms: float) -> float:
+    """Units all ranks processed divided by the slowest rank's time (replicas: weak scaling)."""
+    return units_per_rank * world / (slowest_ms * 1e-3)
+
+
+def replica_seed_base(rank: int) -> int:
+    """Replicas draw different inputs and mixing seeds."""
+    return rank * 1000
+
+
 class ClockSampler:
     """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
     QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
@@ -135,7 +154,7 @@ def run_reference(args):
         return 0
     oracle.build()
     w = inputs.WORKLOADS[WORKLOAD]
-    n_s, k_s = 128, 6
+    n_s, k_s = 512, 26
     for i in range(args.warmup):
         oracle_sample_step(w, 16, 1, i)
     times = [oracle_sample_step(w, n_s, k_s, i) for i in range(args.steps)]
@@ -188,7 +207,7 @@ def run_ours(args):
     ctx.set_level3(args.level3)
     ctx.ensure_batch_workspace(n, k, d, p, w.dtype, args.lanes)
     # replicas draw different inputs and mixing seeds
-    base = rank * 1000
+    base = replica_seed_base(rank)
     Hs, Ws, seeds = [], [], []
     for c in range(calls):
         h = inputs.make_hidden(n, d, w.dtype, w.seed + base + c, w.rms_norm, dev)
@@ -293,13 +312,9 @@ def run_ours(args):
     e2e_s = (time.perf_counter() - t0) / args.steps
     checksum += Qh.float().abs().mean().to(dev)
 
-    t_ms = torch.tensor([ms, e2e_s * 1e3], device=dev, dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(t_ms, op=dist.ReduceOp.MAX)
-    ms_max, e2e_ms_max = float(t_ms[0]), float(t_ms[1])
-    tokens = float(n) * calls * args.steps * world
-    value = tokens / (ms_max * 1e-3)
-    e2e_value = float(n) * e2e_calls * world / (e2e_ms_max * 1e-3)
+    ms_max, e2e_ms_max = max_over_ranks([ms, e2e_s * 1e3], dist, dev)
+    value = whole_job_rate(float(n) * calls * args.steps, world, ms_max)
+    e2e_value = whole_job_rate(float(n) * e2e_calls, world, e2e_ms_max)
 
     # ---- per-launch device times of the main kernel classes (CUDA events on the launching stream):
     #      one orthogonal and one non-orthogonal call, sampling lanes off so that launches do not overlap ----
@@ -380,7 +395,7 @@ def run_ours(args):
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
-            n_s, k_s = 128, 6
+            n_s, k_s = 512, 26
             dt_s = oracle_sample_step(w, n_s, k_s, 0)
             line["cpu_baseline"] = {"value": n_s / dt_s, "unit": UNIT, "cores": oracle.num_threads(),
                                     "kind": "oracle", "sample": oracle_sample_desc(n_s, k_s, w)}
