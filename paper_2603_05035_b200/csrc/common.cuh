@@ -186,6 +186,7 @@ struct LuScratch {
     float* M = nullptr;   // m x ld working copy
     int* ipiv = nullptr;  // m
     int* perm = nullptr;  // m
+    int* swap_table = nullptr;  // composed interchanges of one panel / block: count, then (target, source) pairs
 };
 LuScratch carve_lu(Arena&, int m, int ld);
 int run_lu_inverse(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, cudaStream_t);

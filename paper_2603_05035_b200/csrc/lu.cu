@@ -267,54 +267,71 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     return after_launch(ctx);
 }
 
-// Applies the interchanges rows j0+c <-> ipiv[j0+c], c = 0 .. jb-1 (in order, jb <= 128) to columns
-// [c_lo, c_hi) of X, skipping columns [skip_lo, skip_hi).  Every CTA first composes the interchanges into a
-// row permutation of the (at most 2 jb) rows they touch -- one warp, table in shared memory -- and then moves
-// 32 columns of those rows through a shared-memory tile: gather from the source rows, scatter to the targets.
+// Row interchanges of a panel or an outer block, in two launches:
+//   compose_swaps_kernel (one warp): turns rows j0+c <-> ipiv[j0+c], c = 0 .. jb-1 (in order, jb <= 128) into a
+//       row permutation of the at most 2 jb rows they touch: table[0] = count, then (target row, source row) pairs;
+//   swap_rows_kernel: every CTA moves 32 columns of those rows through a shared-memory tile (gather from the
+//       source rows, scatter to the targets) for columns [c_lo, c_hi) minus [skip_lo, skip_hi).
 constexpr int kSwapMaxRows = 256;
 
-__global__ void __launch_bounds__(256)
-swap_rows_kernel(float* __restrict__ X, int ld, int j0, int jb, const int* __restrict__ ipiv,
-                 int c_lo, int c_hi, int skip_lo, int skip_hi)
+__global__ void __launch_bounds__(32)
+compose_swaps_kernel(int j0, int jb, const int* __restrict__ ipiv, int* __restrict__ table)
 {
     __shared__ int pos_s[kSwapMaxRows];       // row that receives ...
     __shared__ int src_s[kSwapMaxRows];       // ... the content this row had before the interchanges
-    __shared__ int count_s;
+    const int lane = threadIdx.x;
+    int count = 0;
+    for (int c = 0; c < jb; ++c) {
+        const int a = j0 + c, b = ipiv[a];
+        if (a == b) continue;
+        int ia = -1, ib = -1;
+        for (int base = 0; base < count; base += 32) {
+            const int e = base + lane;
+            const int p = (e < count) ? pos_s[e] : -1;
+            const unsigned ma = __ballot_sync(0xffffffffu, p == a);
+            const unsigned mb = __ballot_sync(0xffffffffu, p == b);
+            if (ma) ia = base + __ffs(ma) - 1;
+            if (mb) ib = base + __ffs(mb) - 1;
+        }
+        if (ia < 0) { ia = count; if (lane == 0) { pos_s[count] = a; src_s[count] = a; } ++count; }
+        if (ib < 0) { ib = count; if (lane == 0) { pos_s[count] = b; src_s[count] = b; } ++count; }
+        __syncwarp();
+        if (lane == 0) { const int t = src_s[ia]; src_s[ia] = src_s[ib]; src_s[ib] = t; }
+        __syncwarp();
+    }
+    if (lane == 0) table[0] = count;
+    for (int e = lane; e < count; e += 32) { table[1 + 2 * e] = pos_s[e]; table[2 + 2 * e] = src_s[e]; }
+}
+
+__global__ void __launch_bounds__(256)
+swap_rows_kernel(float* __restrict__ X, int ld, const int* __restrict__ table, int c_lo, int c_hi, int skip_lo,
+                 int skip_hi)
+{
     __shared__ float tile[kSwapMaxRows][33];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    if (warp == 0) {
-        int count = 0;
-        for (int c = 0; c < jb; ++c) {
-            const int a = j0 + c, b = ipiv[a];
-            if (a == b) continue;
-            // table slots of rows a and b (insert identity entries when they are new)
-            int ia = -1, ib = -1;
-            for (int base = 0; base < count; base += 32) {
-                const int e = base + lane;
-                const int p = (e < count) ? pos_s[e] : -1;
-                const unsigned ma = __ballot_sync(0xffffffffu, p == a);
-                const unsigned mb = __ballot_sync(0xffffffffu, p == b);
-                if (ma) ia = base + __ffs(ma) - 1;
-                if (mb) ib = base + __ffs(mb) - 1;
-            }
-            if (ia < 0) { ia = count; if (lane == 0) { pos_s[count] = a; src_s[count] = a; } ++count; }
-            if (ib < 0) { ib = count; if (lane == 0) { pos_s[count] = b; src_s[count] = b; } ++count; }
-            __syncwarp();
-            if (lane == 0) { const int t = src_s[ia]; src_s[ia] = src_s[ib]; src_s[ib] = t; }
-            __syncwarp();
-        }
-        if (lane == 0) count_s = count;
-    }
-    __syncthreads();
-    const int count = count_s;
+    const int count = table[0];
     int col = c_lo + blockIdx.x * 32 + lane;
     if (col >= skip_lo && col < skip_hi) col = c_hi;          // inactive lane
     const bool ok = col < c_hi;
     for (int e = warp; e < count; e += 8)
-        if (ok) tile[e][lane] = X[(size_t)src_s[e] * ld + col];
+        if (ok) tile[e][lane] = X[(size_t)table[2 + 2 * e] * ld + col];
     __syncthreads();
-    for (int e = warp; e < count; e += 8)
-        if (ok && src_s[e] != pos_s[e]) X[(size_t)pos_s[e] * ld + col] = tile[e][lane];
+    for (int e = warp; e < count; e += 8) {
+        const int pos = table[1 + 2 * e], src = table[2 + 2 * e];
+        if (ok && src != pos) X[(size_t)pos * ld + col] = tile[e][lane];
+    }
+}
+
+int launch_swaps(gelo_ctx* ctx, float* X, int ld, int j0, int jb, const int* ipiv, int* table, bool compose,
+                 int c_lo, int c_hi, int skip_lo, int skip_hi, cudaStream_t st)
+{
+    if (compose) {
+        compose_swaps_kernel<<<1, 32, 0, st>>>(j0, jb, ipiv, table);
+        GELO_TRY(after_launch(ctx));
+    }
+    if (c_hi <= c_lo) return GELO_OK;
+    swap_rows_kernel<<<ceil_div(c_hi - c_lo, 32), 256, 0, st>>>(X, ld, table, c_lo, c_hi, skip_lo, skip_hi);
+    return after_launch(ctx);
 }
 
 // X[i0:i0+ib, c_lo:c_hi) <- L_ii^-1 X (unit lower, forward) or U_ii^-1 X (upper, backward);
@@ -477,6 +494,7 @@ LuScratch carve_lu(Arena& a, int m, int ld)
     s.M = static_cast<float*>(a.take((size_t)m * ld * sizeof(float)));
     s.ipiv = static_cast<int*>(a.take((size_t)m * sizeof(int)));
     s.perm = static_cast<int*>(a.take((size_t)m * sizeof(int)));
+    s.swap_table = static_cast<int*>(a.take((size_t)(2 * 256 + 4) * sizeof(int)));
     return s;
 }
 
@@ -495,8 +513,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
             const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
             GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
             if (ob > jb) {       // interchanges on the other columns of this block
-                swap_rows_kernel<<<ceil_div(ob, 32), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, b0, bend, j0, j0 + jb);
-                GELO_TRY(after_launch(ctx));
+                GELO_TRY(launch_swaps(ctx, M, ld, j0, jb, s.ipiv, s.swap_table, true, b0, bend, j0, j0 + jb, st));
             }
             const int ncb = bend - (j0 + jb);
             if (ncb > 0) {
@@ -507,8 +524,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
             }
         }
         if (m > ob) {            // the block's interchanges on everything left and right of it
-            swap_rows_kernel<<<ceil_div(m, 32), 256, 0, st>>>(M, ld, b0, ob, s.ipiv, 0, m, b0, bend);
-            GELO_TRY(after_launch(ctx));
+            GELO_TRY(launch_swaps(ctx, M, ld, b0, ob, s.ipiv, s.swap_table, true, 0, m, b0, bend, st));
         }
         const int nc = m - bend;
         if (nc <= 0) continue;
@@ -556,8 +572,7 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
         const int j0 = pnl * NB, jb = (m - j0 < NB) ? (m - j0) : NB;
         GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
         if (m > jb) {
-            swap_rows_kernel<<<ceil_div(m, 32), 256, 0, st>>>(M, ld, j0, jb, s.ipiv, 0, m, j0, j0 + jb);
-            GELO_TRY(after_launch(ctx));
+            GELO_TRY(launch_swaps(ctx, M, ld, j0, jb, s.ipiv, s.swap_table, true, 0, m, j0, j0 + jb, st));
         }
         const int nc = m - j0 - jb;
         if (nc <= 0) continue;

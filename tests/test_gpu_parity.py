@@ -472,3 +472,20 @@ def test_householder_qr_tensor_core_blocks(oracle, m):
     assert np.all(np.sum(q * q_ref, axis=0)[: max(1, m // 2)] > 1 - 2e-3)
     assert c.last_status() == binding.OK
     c.close()
+
+
+# ------------------------------------------------------------------------- attention output projection
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("kind", [ORTHOGONAL, NONORTHOGONAL])
+def test_output_projection_unsplit(ctx, oracle, dt, kind):
+    """The same procedure on the attention output projection O: a d x d weight, one unsplit result."""
+    n, k, d = 320, 16, 512
+    p = d
+    ctx.ensure_workspace(n, k, d, p, dt)
+    H = inputs.make_hidden(n, d, dt, 41, True, "cuda")
+    W = inputs.make_weight(d, p, dt, 41, "cuda")
+    Y = torch.full((n, p), float("nan"), device="cuda", dtype=TDT[dt])
+    ctx.qkv_offload(H, W, n, k, d, p, kind, 4242, 10.0, dt, Y)
+    torch.cuda.synchronize()
+    assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL[dt]
