@@ -248,6 +248,10 @@ int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_h
 /* Number of concurrent sampling lanes of the batched calls (1..32, default 4) and the workspace
  * they need.  0 bytes if an argument is invalid. */
 int gelo_set_lanes(gelo_ctx* ctx, int lanes);
+/* In batches with at least `share` lanes every tensor-core update of the factorisations runs on 1/share of
+ * the SMs (default 4; 1 = always all SMs), so that the updates of different lanes overlap instead of queueing
+ * behind each other's launch and drain phases. */
+int gelo_set_lane_share(gelo_ctx* ctx, int share);
 size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lanes);
 
 /* ---- per-launch timing (measurement aid; no counterpart in the paper) ----------------------- */

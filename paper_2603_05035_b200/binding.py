@@ -58,6 +58,7 @@ EXPORTS = {
     "gelo_qkv_offload_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_lanes": (_i, [_vp, _i]),
+    "gelo_set_lane_share": (_i, [_vp, _i]),
     "gelo_batch_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "gelo_profile_start": (_i, [_vp]),
     "gelo_profile_stop": (_i, [_vp, _vp, _vp]),
@@ -173,6 +174,9 @@ class Context:
     def set_lanes(self, lanes: int):
         self._check(self._lib.gelo_set_lanes(self._h, lanes), "gelo_set_lanes")
         self.lanes = int(lanes)
+
+    def set_lane_share(self, share: int):
+        self._check(self._lib.gelo_set_lane_share(self._h, share), "gelo_set_lane_share")
 
     def ensure_batch_workspace(self, n, k, d, p, dtype, lanes=None):
         """Workspace for the batched entry points with `lanes` concurrent sampling lanes."""

@@ -227,7 +227,8 @@ int sample_on_lane(gelo_ctx* ctx, const Layout& L, int lane, int m, int kind, ui
     if (ctx->prof_on)      // per-launch timing needs real launches
         return sample_attempt(ctx, L, m, kind, seed, 0u, dtype, L.A, L.Ainv, L.ldi, nullptr, ls, true, slot);
     for (auto& g : ctx->graphs) {
-        if (g.key_ptr == L.G && g.m == m && g.kind == kind && g.dtype == dtype && g.level3 == ctx->level3) {
+        if (g.key_ptr == L.G && g.m == m && g.kind == kind && g.dtype == dtype && g.level3 == ctx->level3 &&
+            g.tc_ctas == ctx->tc_update_ctas) {
             GELO_CUDA_OK(cudaGraphLaunch(g.exec, ls));
             ctx->launches += g.launches;
             return GELO_OK;
@@ -243,7 +244,7 @@ int sample_on_lane(gelo_ctx* ctx, const Layout& L, int lane, int m, int kind, ui
         return rc != GELO_OK ? rc : GELO_ERR_CUDA;
     }
     gelo_ctx::SampleGraph g;
-    g.key_ptr = L.G; g.m = m; g.kind = kind; g.dtype = dtype; g.level3 = ctx->level3;
+    g.key_ptr = L.G; g.m = m; g.kind = kind; g.dtype = dtype; g.level3 = ctx->level3; g.tc_ctas = ctx->tc_update_ctas;
     g.launches = ctx->launches - before;
     g.exec = nullptr;
     const cudaError_t ie = cudaGraphInstantiate(&g.exec, graph, 0);
@@ -278,6 +279,8 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     const size_t es = elem_size(dtype);
     const bool split = K[0] != nullptr;
     const size_t third = (size_t)n * (p / 3) * es;
+    // with several lanes in flight each level-3 update takes a share of the SMs (ctx->lane_tc_share-th of them)
+    ctx->tc_update_ctas = (D >= ctx->lane_tc_share && ctx->lane_tc_share > 1) ? ctx->sm_count / ctx->lane_tc_share : 0;
 
     // Back-to-back batches of the same shape on the same stream keep the lanes running across the seam: each
     // lane only waits until the products that read its previous pair are done.  Otherwise the lanes start after
@@ -326,6 +329,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         }
         if (i + D < calls) GELO_TRY(enqueue_sample(i + D));
     }
+    ctx->tc_update_ctas = 0;
     ctx->chain_valid = calls >= D && !ctx->prof_on;
     ctx->chain_stream = st;
     ctx->chain_key = L[D - 1].G;
@@ -758,6 +762,13 @@ int gelo_set_level3(gelo_ctx* ctx, int mode)
 {
     if (!ctx || mode < 0 || mode > 2) return GELO_ERR_INVALID;
     ctx->level3 = mode;
+    return GELO_OK;
+}
+
+int gelo_set_lane_share(gelo_ctx* ctx, int share)
+{
+    if (!ctx || share < 1 || share > 16) return GELO_ERR_INVALID;
+    ctx->lane_tc_share = share;
     return GELO_OK;
 }
 

@@ -51,6 +51,9 @@ struct gelo_ctx {
     float gamma = 0.5f;
     float cond_bound = 100.0f;
     int max_attempts = 8;
+    int lane_tc_share = 4;        // batches with at least this many lanes give each level-3 update 1/share of the SMs
+    int tc_update_ctas = 0;       // CTAs of a level-3 tensor-core launch (0: one per SM); batches with many lanes use fewer,
+                                  // so that the updates of several lanes run side by side instead of queueing
     int level3 = 0;               // 0: tensor cores for bf16 calls with m >= 256; 1: always fp32 FMA; 2: always tensor cores
     long long launches = 0;
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
@@ -67,7 +70,7 @@ struct gelo_ctx {
     const void* chain_key = nullptr;
     int chain_lanes = 0;
     // replayable launch graphs of the sampling sequence, one per (lane scratch, kind, size, type)
-    struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3; cudaGraphExec_t exec; long long launches; };
+    struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3, tc_ctas; cudaGraphExec_t exec; long long launches; };
     std::vector<SampleGraph> graphs;
     uint64_t* lane_seed_dev = nullptr;              // one seed slot per lane
     // optional per-launch timing (gelo_profile_start / gelo_profile_stop)

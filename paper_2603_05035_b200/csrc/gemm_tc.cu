@@ -449,7 +449,8 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
         attr_done[ctx->device] = true;
     }
     const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN) * p.ksplit;
-    const int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
+    if (p.mode != TC_STORE_BF16 && ctx->tc_update_ctas > 0 && grid > ctx->tc_update_ctas) grid = ctx->tc_update_ctas;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
         gemm_tc_kernel<BN, kStages, kStaging><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, p);
