@@ -394,9 +394,10 @@ def test_batched_offload_matches_single_calls(oracle, name, calls, lanes):
 def test_batched_offload_full_size(oracle):
     w = inputs.WORKLOADS["prefill_bf16"]
     n, k, d, p = w.n, w.k, w.d, w.p
-    calls = 6
+    calls = 20                      # the benchmark's configuration: 16 lanes, a quarter of the SMs per level-3 update
     c = binding.Context(0)
-    c.ensure_batch_workspace(n, k, d, p, w.dtype, 4)
+    c.set_lanes(16)
+    c.ensure_batch_workspace(n, k, d, p, w.dtype, 16)
     Hs, Ws, seeds = [], [], []
     for i in range(calls):
         H, W, seed = inputs.make_call_inputs(w, i, "cuda")
@@ -406,7 +407,7 @@ def test_batched_offload_full_size(oracle):
     c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, *outs)
     torch.cuda.synchronize()
     assert c.last_status() == binding.OK
-    for i in (0, 3, 5):
+    for i in (0, 7, 19):
         y = np.hstack([f64(outs[0][i]), f64(outs[1][i]), f64(outs[2][i])])
         rows = sample_rows(n, 48, seed=i)
         assert oracle.rel_fro(y[rows], oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)) <= TOL["bf16"]
@@ -489,3 +490,53 @@ def test_output_projection_unsplit(ctx, oracle, dt, kind):
     ctx.qkv_offload(H, W, n, k, d, p, kind, 4242, 10.0, dt, Y)
     torch.cuda.synchronize()
     assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL[dt]
+
+
+def test_batch_of_zero_calls_and_bad_batches():
+    c = binding.Context(0)
+    c.ensure_batch_workspace(64, 0, 64, 192, "f32", 2)
+    c.qkv_offload_batch([], [], 64, 0, 64, 192, [], [], 0.0, "f32", [], [], [])       # nothing to do
+    H = torch.zeros((64, 64), device="cuda"); W = torch.zeros((64, 192), device="cuda")
+    Q = torch.zeros((64, 64), device="cuda")
+    with pytest.raises(binding.GeloError) as e:                                        # unknown mixing kind
+        c.qkv_offload_batch([H], [W], 64, 0, 64, 192, [7], [0], 0.0, "f32", [Q], [Q], [Q])
+    assert e.value.status == binding.ERR_INVALID
+    with pytest.raises(binding.GeloError) as e:                                        # K given, V missing
+        c.qkv_offload_batch([H], [W], 64, 0, 64, 192, [0], [0], 0.0, "f32", [Q], [Q], [None])
+    assert e.value.status == binding.ERR_INVALID
+    c.set_workspace(torch.empty(4096, dtype=torch.uint8, device="cuda"))
+    with pytest.raises(binding.GeloError) as e:
+        c.qkv_offload_batch([H], [W], 64, 0, 64, 192, [0], [0], 0.0, "f32", [Q], [Q], [Q])
+    assert e.value.status == binding.ERR_WORKSPACE
+    c.close()
+
+
+@pytest.mark.parametrize("kind", [ORTHOGONAL, NONORTHOGONAL])
+def test_offload_beyond_the_register_resident_panels(oracle, kind):
+    """m = 4400 rows exceed what a cluster's registers hold (4352): the first panels fall back to the
+    one-CTA kernels that work out of L2, the rest use the cluster kernels."""
+    n, k, d, p = 4400, 0, 64, 192
+    c = binding.Context(0)
+    c.ensure_workspace(n, k, d, p, "bf16")
+    H = inputs.make_hidden(n, d, "bf16", 77, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 77, "cuda")
+    Q = torch.empty((n, p // 3), device="cuda", dtype=torch.bfloat16); K = torch.empty_like(Q); V = torch.empty_like(Q)
+    c.qkv_offload(H, W, n, k, d, p, kind, 9, 0.0, "bf16", Q, K, V)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    y = np.hstack([f64(Q), f64(K), f64(V)])
+    assert oracle.rel_fro(y, oracle.direct(f64(H), f64(W))) <= TOL["bf16"]
+    c.close()
+
+
+def test_profile_counts_launches(ctx):
+    w = inputs.WORKLOADS["decode_bf16"]
+    H, W, seed = inputs.make_call_inputs(w, 0, "cuda")
+    ctx.ensure_workspace(w.n, w.k, w.d, w.p, w.dtype)
+    Q = torch.empty((w.n, w.p // 3), device="cuda", dtype=torch.bfloat16); K = torch.empty_like(Q); V = torch.empty_like(Q)
+    ctx.profile_start()
+    ctx.qkv_offload(H, W, w.n, w.k, w.d, w.p, ORTHOGONAL, seed, 10.0, w.dtype, Q, K, V)
+    prof = ctx.profile_stop()
+    assert prof["gemm_tc"]["launches"] == 3 and prof["gemm_tc"]["ms"] > 0          # mix, project, unmix
+    assert prof["qr_panel"]["launches"] == 3                                        # m = 68: three 32-column panels
+    assert prof["gemm_tc"]["work"] == pytest.approx(2.0 * (68 * 68 * 4096 + 68 * 4096 * 12288 + 64 * 68 * 12288))
