@@ -12,7 +12,7 @@ namespace gelo {
 namespace {
 
 constexpr int kRowSlabs = 16;
-constexpr int kPowerIters = 24;
+constexpr int kPowerIters = 12;   // the estimate is within about 4% of kappa_2 after 12 steps (measured at m = 512 .. 4300)
 
 struct CondViews {
     const float* op[2];
