@@ -118,6 +118,9 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
     __shared__ int win_r[2][kClusterMax];
     __shared__ float win_row[2][kClusterMax][NB];
     __shared__ float rowj_buf[2][NB];
+    __shared__ float coef_s[NB];
+    __shared__ float prow_s[NB];
+    __shared__ int pr_s;
 
     const int lane = threadIdx.x & 31;
     const int warp = threadIdx.x >> 5;
@@ -177,45 +180,51 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
             for (int r = 0; r < CS; ++r) cluster.map_shared_rank(&rowj_buf[par][lane], r)[0] = x[0];
         if (CS > 1) cluster.sync(); else __syncthreads();
 
-        // ---- the winner over the cluster ----
-        float pv = win_v[par][0];
-        int pr = win_r[par][0], pw = 0;
-        for (int r = 1; r < CS; ++r) {
-            const float ov = win_v[par][r];
-            const int orow = win_r[par][r];
-            if (ov > pv || (ov == pv && orow < pr)) { pv = ov; pr = orow; pw = r; }
+        // ---- warp 0 picks the winner over the cluster and prepares the elimination coefficients ----
+        if (warp == 0) {
+            float pv = (lane < CS) ? win_v[par][lane] : -2.0f;
+            int pr = (lane < CS) ? win_r[par][lane] : 0x7fffffff;
+            int pw = lane;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) {
+                const float ov = __shfl_xor_sync(full, pv, off);
+                const int orow = __shfl_xor_sync(full, pr, off);
+                const int ow = __shfl_xor_sync(full, pw, off);
+                if (ov > pv || (ov == pv && orow < pr)) { pv = ov; pr = orow; pw = ow; }
+            }
+            const float prow = win_row[par][pw][lane];       // pivot row, this lane's column
+            const float pivot = __shfl_sync(full, prow, c);
+            const float inv = (pivot != 0.0f) ? 1.0f / pivot : 0.0f;
+            // x <- coef * x_c + (lane == c ? 0 : x):  the multiplier l = x_c / pivot in column c, -l * pivot row after it
+            coef_s[lane] = (lane > c) ? -inv * prow : ((lane == c) ? inv : 0.0f);
+            prow_s[lane] = prow;
+            if (lane == 0) {
+                pr_s = pr;
+                if (rank == 0) {
+                    ipiv[j] = pr;
+                    if (!(pv > 0.0f)) atomicCAS(status, 0, (int)GELO_ERR_COND);
+                }
+            }
         }
-        const float prow = win_row[par][pw][lane];           // pivot row, this lane's column
-        const float oldj = rowj_buf[par][lane];
-        if (rank == 0 && threadIdx.x == 0) {
-            ipiv[j] = pr;
-            if (!(pv > 0.0f)) atomicCAS(status, 0, (int)GELO_ERR_COND);
-        }
-        const float pivot = __shfl_sync(full, prow, c);
-        const float inv = (pivot != 0.0f) ? 1.0f / pivot : 0.0f;
+        __syncthreads();
+        const int pr = pr_s;
+        const float coef = coef_s[lane];
         // ---- swap in registers ----
         if (pr != j) {
             const int poff = pr - j0;
             if (poff % stride == gw) {                       // this warp holds row pr: it receives old row j
                 const int pi = poff / stride;
+                const float oldj = rowj_buf[par][lane];
                 const float oc = __shfl_sync(full, oldj, c);
 #pragma unroll
                 for (int i = 0; i < RPT; ++i) if (i == pi) { x[i] = oldj; xc[i] = oc; }
             }
-            if (gw == c) x[0] = prow;                        // rank 0, warp c: row j receives the pivot row
+            if (gw == c) x[0] = prow_s[lane];                // rank 0, warp c: row j receives the pivot row
         }
         // ---- eliminate below row j ----
 #pragma unroll
-        for (int i = 1; i < RPT; ++i) {
-            const float l = xc[i] * inv;
-            if (lane > c) x[i] = fmaf(-l, prow, x[i]);
-            else if (lane == c) x[i] = l;
-        }
-        if (gw > c) {
-            const float l = xc[0] * inv;
-            if (lane > c) x[0] = fmaf(-l, prow, x[0]);
-            else if (lane == c) x[0] = l;
-        }
+        for (int i = 1; i < RPT; ++i) x[i] = fmaf(coef, xc[i], (lane == c) ? 0.0f : x[i]);
+        if (gw > c) x[0] = fmaf(coef, xc[0], (lane == c) ? 0.0f : x[0]);
     }
 #pragma unroll
     for (int i = 0; i < RPT; ++i) {
