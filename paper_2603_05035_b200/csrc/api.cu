@@ -13,12 +13,18 @@ inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
 inline int round_up(int x, int to) { return (x + to - 1) / to * to; }
 constexpr int kTcMinRows = 256;   // below this the factorisations are latency-bound anyway
 
-// Whether the factorisations of an m x m sample stored as `dtype` use the split-precision tensor-core updates.
-inline bool use_level3_tc(const gelo_ctx* ctx, int m, int dtype)
+// How a factorisation of an m x m sample stored as `dtype` runs its level-3 updates: 0 = fp32 FMA kernels,
+// 2 = tensor cores with three bf16 products of split operands, 3 = tensor cores with one tf32 product.
+// By default bf16 calls run the QR on tf32: its errors only perturb the orthogonality of a matrix that is rounded to
+// bf16 (8 significant bits against tf32's 11) right afterwards, and its trailing matrix is itself an operand, which
+// the split products would have to convert block after block.  The LU keeps the split products: the two triangular
+// solves behind A^-1 amplify update errors by the conditioning of L and U, and its operands are thin panels only.
+inline int level3_kind(const gelo_ctx* ctx, int m, int dtype, bool qr)
 {
-    if (ctx->level3 == 1) return false;
-    if (ctx->level3 == 2) return m > gelo::kPanel;
-    return dtype == GELO_BF16 && m >= kTcMinRows;
+    if (ctx->level3 == 1) return 0;
+    if (ctx->level3 == 2 || ctx->level3 == 3) return m > gelo::kPanel ? ctx->level3 : 0;
+    if (dtype != GELO_BF16 || m < kTcMinRows) return 0;
+    return qr ? 3 : 2;
 }
 
 // Every scratch buffer of one call with sizes (n, k, d, p, dtype); carved in a fixed order so
@@ -113,9 +119,13 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
 {
     const int ldi = L.ldi;
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st, seed_dev));
-    if (use_level3_tc(ctx, m, dtype)) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, st));
+    const int l3 = level3_kind(ctx, m, dtype, true);
+    if (l3) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, l3 == 3, st));
     else GELO_TRY(run_householder_qr(ctx, m, L.G, ldi, L.Qraw, L.qr, st));
     if (kind == GELO_ORTHOGONAL) {
+        // tf32 updates: polish Q (A32 and X32 are free for this kind).  The non-orthogonal kind skips it: there Q0 only
+        // has to keep A = Q0 + gamma G1 well conditioned, and A^-1 comes from the LU of the stored A.
+        if (l3 == 3) GELO_TRY(polish_orthogonal_tf32(ctx, m, L.Qraw, ldi, L.X32, L.A32, st));
         GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, dtype, A_out, Ainv_out, lda, st));
         if (cond_dev) {
             set_scalar_kernel<<<1, 1, 0, st>>>(cond_dev, 1.0f);
@@ -129,8 +139,9 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st, seed_dev));
     GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st));
     if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
-    // split-precision tensor-core updates (about 1e-5 relative) serve the bf16 path; the fp32 path stays exact
-    if (use_level3_tc(ctx, m, dtype)) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, ldi, L.X32, L.lu, L.tc, st));
+    // tensor-core updates serve the bf16 path; the fp32 path stays exact
+    const int l3lu = level3_kind(ctx, m, dtype, false);
+    if (l3lu) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, ldi, L.X32, L.lu, L.tc, l3lu == 3, st));
     else GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
     GELO_TRY(launch_narrow(ctx, m, L.X32, ldi, dtype, Ainv_out, lda, st));
     return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st,
@@ -520,16 +531,18 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
     Layout L;
     if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
-    const bool tcp = use_level3_tc(ctx, m, GELO_F32);
+    const int tcp = level3_kind(ctx, m, GELO_F32, true);
     if (ld == L.ldi) {
-        if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, st));
+        if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, tcp == 3, st));
         else GELO_TRY(run_householder_qr(ctx, m, G_dev, ld, L.Qraw, L.qr, st));
+        if (tcp == 3) GELO_TRY(polish_orthogonal_tf32(ctx, m, L.Qraw, ld, L.X32, L.A32, st));
         return launch_finish_mixing(ctx, m, L.Qraw, ld, G_dev, ld, GELO_F32, Q_dev, Qt_dev, ld, st);
     }
     GELO_CUDA_OK(cudaMemcpy2DAsync(L.G, (size_t)L.ldi * 4, G_dev, (size_t)ld * 4, (size_t)m * 4, m,
                                    cudaMemcpyDeviceToDevice, st));
-    if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, st));
+    if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, tcp == 3, st));
     else GELO_TRY(run_householder_qr(ctx, m, L.G, L.ldi, L.Qraw, L.qr, st));
+    if (tcp == 3) GELO_TRY(polish_orthogonal_tf32(ctx, m, L.Qraw, L.ldi, L.X32, L.A32, st));
     GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, L.ldi, L.G, L.ldi, GELO_F32, Q_dev, Qt_dev, ld, st));
     return cudaMemcpy2DAsync(G_dev, (size_t)ld * 4, L.G, (size_t)L.ldi * 4, (size_t)m * 4, m,
                              cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
@@ -542,12 +555,12 @@ int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ain
     Layout L;
     if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
     cudaStream_t st = as_stream(stream);
-    const bool tcp = use_level3_tc(ctx, m, GELO_F32);
-    if (ld == L.ldi) return tcp ? run_lu_inverse_tc(ctx, m, A_dev, ld, Ainv_dev, L.lu, L.tc, st)
+    const int tcp = level3_kind(ctx, m, GELO_F32, false);
+    if (ld == L.ldi) return tcp ? run_lu_inverse_tc(ctx, m, A_dev, ld, Ainv_dev, L.lu, L.tc, tcp == 3, st)
                                 : run_lu_inverse(ctx, m, A_dev, ld, Ainv_dev, L.lu, st);
     GELO_CUDA_OK(cudaMemcpy2DAsync(L.A32, (size_t)L.ldi * 4, A_dev, (size_t)ld * 4, (size_t)m * 4, m,
                                    cudaMemcpyDeviceToDevice, st));
-    if (tcp) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, L.ldi, L.X32, L.lu, L.tc, st));
+    if (tcp) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, L.ldi, L.X32, L.lu, L.tc, tcp == 3, st));
     else GELO_TRY(run_lu_inverse(ctx, m, L.A32, L.ldi, L.X32, L.lu, st));
     return cudaMemcpy2DAsync(Ainv_dev, (size_t)ld * 4, L.X32, (size_t)L.ldi * 4, (size_t)m * 4, m,
                              cudaMemcpyDeviceToDevice, st) == cudaSuccess ? GELO_OK : GELO_ERR_CUDA;
@@ -755,12 +768,12 @@ int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int 
     DeviceGuard guard(ctx->device);
     Layout L;
     if (!carve_ctx(ctx, M > N ? M : N, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
-    return tc_update_f32(ctx, L.tc, M, N, K, A_dev, lda, B_dev, ldb, C_dev, ldc, as_stream(stream));
+    return tc_update_f32(ctx, L.tc, ctx->level3 == 3, M, N, K, A_dev, lda, B_dev, ldb, C_dev, ldc, as_stream(stream));
 }
 
 int gelo_set_level3(gelo_ctx* ctx, int mode)
 {
-    if (!ctx || mode < 0 || mode > 2) return GELO_ERR_INVALID;
+    if (!ctx || mode < 0 || mode > 3) return GELO_ERR_INVALID;
     ctx->level3 = mode;
     return GELO_OK;
 }

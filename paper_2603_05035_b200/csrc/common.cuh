@@ -54,7 +54,8 @@ struct gelo_ctx {
     int lane_tc_share = 4;        // batches with at least this many lanes give each level-3 update 1/share of the SMs
     int tc_update_ctas = 0;       // CTAs of a level-3 tensor-core launch (0: one per SM); batches with many lanes use fewer,
                                   // so that the updates of several lanes run side by side instead of queueing
-    int level3 = 0;               // 0: tensor cores for bf16 calls with m >= 256; 1: always fp32 FMA; 2: always tensor cores
+    int level3 = 0;               // 0: tf32 tensor-core updates for bf16 calls with m >= 256; 1: always fp32 FMA;
+                                  // 2: always tensor cores, three bf16 products of split operands; 3: always tensor cores, tf32
     long long launches = 0;
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
     // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
@@ -155,6 +156,18 @@ int launch_gemm_tc_split_k(gelo_ctx*, int M, int N, int K, const void* Ahi, cons
                            const void* Blo, int ldb, float* planes, size_t plane, int ldp, int ksplit, int* used,
                            cudaStream_t);
 
+// One-product tf32 GEMM straight from fp32 matrices (see gemm_tc.cu): C -= op(A) B in place, or C = op(A) B
+// (optionally rounded to tf32, optionally as split-K planes).
+int launch_gemm_tf32(gelo_ctx*, int M, int N, int K, const float* A, int lda, bool a_mn, const float* B, int ldb,
+                     bool subtract, float* C, int ldc, bool round_out, float out_scale, int ksplit, size_t plane, int* used,
+                     cudaStream_t, float diag_sub = 0.0f, float post_scale = 1.0f);
+// The tensor core drops the 13 low mantissa bits of an fp32 operand instead of rounding them.  For values whose
+// mantissas are spread log-uniformly that loses 2^-11 / (2 ln 2) of the magnitude on average, coherently over all
+// terms of a product; a result whose operand was truncated is scaled back by 1 + kTf32TruncLoss per such operand,
+// which leaves a zero-mean error of about 3e-4 per term.  Operands that a kernel of this library rounded to tf32
+// when it stored them pass through the tensor core unchanged and need no correction.
+constexpr float kTf32TruncLoss = 3.5224e-4f;
+
 // ---- factorizations -------------------------------------------------------------------
 
 // ---- rank-32 updates of the factorisations (HBM streamers) ---------------------------------
@@ -183,7 +196,11 @@ QrScratch carve_qr(Arena&, int m, int ld);
 int run_householder_qr(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, cudaStream_t);
 struct TcScratch;
 // Same factorisation with 128-column outer blocks whose updates run on the tensor cores in split precision.
-int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, cudaStream_t);
+int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, bool tf32,
+                          cudaStream_t);
+// One Newton-Schulz step Q <- Q - Q (Q^T Q - I) / 2 on the tensor cores in tf32: squares the orthogonality defect
+// that tf32 updates leave in Q.  D and Qold are m x ld scratch matrices.
+int polish_orthogonal_tf32(gelo_ctx*, int m, float* Q, int ld, float* D, float* Qold, cudaStream_t);
 
 struct LuScratch {
     float* M = nullptr;   // m x ld working copy
@@ -195,7 +212,7 @@ LuScratch carve_lu(Arena&, int m, int ld);
 int run_lu_inverse(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, cudaStream_t);
 struct TcScratch;
 int run_lu_inverse_tc(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, const TcScratch&,
-                      cudaStream_t);
+                      bool tf32, cudaStream_t);
 
 struct CondScratch {
     float* vec = nullptr;     // iterate, image and row-slab partial sums for both operators
@@ -223,6 +240,9 @@ int launch_split(gelo_ctx*, const float* src, int lds, int rows, int cols, void*
 
 int launch_sum_split(gelo_ctx*, const float* planes, size_t plane, int parts, int ld, int rows, int cols, void* hi,
                      void* lo, int ldo, cudaStream_t);
+// out = scale * (sum of `parts` fp32 planes in plane order), rounded to tf32 (cols a multiple of 4)
+int launch_sum_planes(gelo_ctx*, const float* planes, size_t plane, int parts, int ld, int rows, int cols, float scale,
+                      float* out, int ldo, cudaStream_t);
 
 // Scratch of the tensor-core level-3 updates (outer blocks of kOuter columns).
 constexpr int kOuter = 128;
@@ -237,11 +257,13 @@ struct TcScratch {
     float* t128 = nullptr;                 // kOuter x kOuter fp32
     float* gram = nullptr;                 // kOuter x kOuter fp32
     float* wf32 = nullptr;                 // kMaxKSplit planes of kOuter x ld fp32 (split-K partial products)
+    float* w32[2] = {nullptr, nullptr};    // kOuter x ld fp32    block rows W and T W of the tf32 updates
 };
 TcScratch carve_tc(Arena&, int m, int ld);
-// C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores in split precision
-int tc_update_f32(gelo_ctx*, const TcScratch&, int M, int N, int K, const float* A, int lda, const float* B, int ldb,
-                  float* C, int ldc, cudaStream_t);
+// C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores: three bf16 products of
+// (high, low) operand pairs, or (tf32) one tf32 product straight from the fp32 operands
+int tc_update_f32(gelo_ctx*, const TcScratch&, bool tf32, int M, int N, int K, const float* A, int lda, const float* B,
+                  int ldb, float* C, int ldc, cudaStream_t);
 
 // ---- shields ---------------------------------------------------------------------------------
 

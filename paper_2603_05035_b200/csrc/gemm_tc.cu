@@ -5,7 +5,10 @@
 //   * the level-3 updates of the blocked QR / LU behind the sampling of A: fp32 matrices are held
 //     as a bf16 (high, low) pair and the product is accumulated as hi*hi + hi*lo + lo*hi in fp32,
 //     with an epilogue that either subtracts the result from an fp32 matrix in place or writes it
-//     as a new (high, low) pair.
+//     as a new (high, low) pair;
+//   * the same level-3 updates in one product of kind::tf32 straight from the fp32 matrices (no operand
+//     conversion passes at all): the A operand is either K-major (a row-major M x K matrix) or MN-major
+//     (the transpose of a row-major K x M matrix, which is how V^T C reads the reflectors).
 //
 //   C (M x N)  (+)=  sum over segments s of  A_s (M x K_s, row-major)  *  B_s (K_s x N, row-major)
 //
@@ -51,6 +54,10 @@ struct TcParams {
     int ldc, csplit, lde;           // lde: row stride of the hi/lo matrices written next to an fp32 C
     int ksplit, kb_per_split;       // K slices (TC_STORE_F32 only): slice q covers k-blocks [q*kb_per_split, ...) of every segment
     long long plane;                // and writes plane q of C0 (stride in elements)
+    int round_tf32;                 // TC_STORE_F32: round the stored values to tf32 (they feed a later tf32 product)
+    float out_scale;                // TC_STORE_F32 with round_tf32: factor applied before the rounding
+    float diag_sub;                 // TC_STORE_F32 with round_tf32: subtracted from the scaled diagonal entries
+    float post_scale;               //   ... and the factor applied after that: out = post_scale * (out_scale * acc - diag_sub [row == col])
     int* status;
 };
 
@@ -115,6 +122,23 @@ __device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, ui
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+__device__ __forceinline__ void tc_mma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
+                                            uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+__device__ __forceinline__ float round_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
 __device__ __forceinline__ void tc_ld_32cols(uint32_t taddr, uint32_t v[32])
 {
     asm volatile(
@@ -131,14 +155,16 @@ __device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sy
 
 // Shared-memory matrix descriptor (sm_100 format): start address, leading and stride byte
 // offsets in 16-byte units, descriptor version 1, 128-byte swizzle.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+// Layout type 2: 128-byte swizzle of 16-byte chunks (8-row atoms).  Layout type 1: 128-byte swizzle of 32-byte
+// chunks (4-row atoms), the only layout that 32-bit operands may use when they are not K-major.
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout = 2)
 {
     uint64_t d = 0;
     d |= (uint64_t)((addr >> 4) & 0x3FFF);
     d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
     d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
     d |= (uint64_t)1 << 46;       // version
-    d |= (uint64_t)2 << 61;       // SWIZZLE_128B
+    d |= (uint64_t)layout << 61;
     return d;
 }
 
@@ -148,15 +174,31 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
 constexpr uint32_t kStageBoxBytes = 32 * 32 * 4;
 constexpr uint32_t kStagingBytes = kEpiWarps * 2 * kStageBoxBytes;
 
-template <int BN, int kStages, bool kStaging>
+// A stage holds 128 bytes of k per A row (64 bf16 or 32 tf32 values) and the matching B rows, so both kinds share
+// the shared-memory geometry: kTf32 only changes the element count per k-block, the box width of the N-major B tile
+// (128 bytes = 64 bf16 or 32 fp32 columns) and the instruction.  kAMn (tf32 only): the A tile arrives as four
+// boxes of 32 m-columns x 32 k-rows, i.e. laid out exactly like a 128-column B tile.
+template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false>
 struct TcCfg {
     static constexpr uint32_t kStagingUsed = kStaging ? kStagingBytes : 0u;
-    static constexpr uint32_t kBBytes = (BN / 64) * kBBoxBytes;
+    static constexpr int kBKE = kTf32 ? 32 : 64;                           // elements of k per stage
+    static constexpr int kBoxCols = kTf32 ? 32 : 64;                       // columns of one N-major box (128 bytes)
+    static constexpr uint32_t kBoxBytes = (uint32_t)kBKE * 128u;           // one N-major box: kBKE rows of 128 bytes
+    static constexpr uint32_t kBBytes = (BN / kBoxCols) * kBoxBytes;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kStagingUsed + 1024 /*alignment slack*/ + 256 /*barriers*/;
-    // Instruction descriptor: fp32 accumulate, bf16 x bf16, A K-major, B N-major, M = 128, N = BN.
-    static constexpr uint32_t kInstrDesc = (1u << 4) | (1u << 7) | (1u << 10) | (0u << 15) | (1u << 16) |
+    // k advance per instruction inside an N-major (or MN-major A) tile: 16 bf16 rows or 8 tf32 rows of 128 bytes
+    static constexpr uint32_t kMnStep = kTf32 ? 1024u : 2048u;
+    // N-major tiles: bf16 in the 16-byte-chunk swizzle (atoms of 8 k-rows, 1024 bytes), fp32 in the 32-byte-chunk
+    // swizzle (atoms of 4 k-rows, 512 bytes)
+    static constexpr uint32_t kMnLayout = kTf32 ? 1u : 2u;
+    static constexpr uint32_t kMnSbo = kTf32 ? 512u : 1024u;
+    // Instruction descriptor: fp32 accumulate, operand formats (1 = bf16, 2 = tf32), A K-major or MN-major,
+    // B N-major, M = 128, N = BN.
+    static constexpr uint32_t kFmt = kTf32 ? 2u : 1u;
+    static constexpr uint32_t kInstrDesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((kAMn ? 1u : 0u) << 15) | (1u << 16) |
                                            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
+    static_assert(!kAMn || kTf32, "MN-major A is only wired up for the tf32 kind");
 };
 
 __device__ __forceinline__ uint32_t pack_bf16(uint32_t a, uint32_t b)
@@ -196,8 +238,14 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
     } else if (prm.mode == TC_STORE_F32) {
         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)slice * prm.plane + (size_t)gm * prm.ldc + gn);
-        dst[0] = make_float4(__uint_as_float(v[0]), __uint_as_float(v[1]), __uint_as_float(v[2]), __uint_as_float(v[3]));
-        dst[1] = make_float4(__uint_as_float(v[4]), __uint_as_float(v[5]), __uint_as_float(v[6]), __uint_as_float(v[7]));
+        float f[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const float a = __uint_as_float(v[j]);
+            f[j] = prm.round_tf32 ? round_tf32(prm.post_scale * (prm.out_scale * a - ((gm == gn + j) ? prm.diag_sub : 0.0f))) : a;
+        }
+        dst[0] = make_float4(f[0], f[1], f[2], f[3]);
+        dst[1] = make_float4(f[4], f[5], f[6], f[7]);
     } else if (prm.mode == TC_EMIT_SPLIT) {
         uint4 hi, lo;
         split2(__uint_as_float(v[0]), __uint_as_float(v[1]), hi.x, lo.x);
@@ -210,13 +258,13 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
     }
 }
 
-template <int BN, int kStages, bool kStaging>
+template <int BN, int kStages, bool kStaging, bool kTf32, bool kAMn>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_c, const TcParams prm)
 {
-    using Cfg = TcCfg<BN, kStages, kStaging>;
+    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-byte alignment
@@ -281,10 +329,16 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                         const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                         const uint32_t sb = sa + kABytes;
                         mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
-                        tma_load_2d(sa, ma, seg.a_k0 + kb * BK, m0, full_bar(s));
+                        if (kAMn) {
 #pragma unroll
-                        for (int j = 0; j < BN / 64; ++j)
-                            tma_load_2d(sb + j * kBBoxBytes, mb, n0 + j * 64, seg.b_row0 + kb * BK, full_bar(s));
+                            for (int j = 0; j < BM / Cfg::kBoxCols; ++j)
+                                tma_load_2d(sa + j * Cfg::kBoxBytes, ma, m0 + j * Cfg::kBoxCols, seg.a_k0 + kb * Cfg::kBKE, full_bar(s));
+                        } else {
+                            tma_load_2d(sa, ma, seg.a_k0 + kb * Cfg::kBKE, m0, full_bar(s));
+                        }
+#pragma unroll
+                        for (int j = 0; j < BN / Cfg::kBoxCols; ++j)
+                            tma_load_2d(sb + j * Cfg::kBoxBytes, mb, n0 + j * Cfg::kBoxCols, seg.b_row0 + kb * Cfg::kBKE, full_bar(s));
                     }
                 }
             }
@@ -318,12 +372,14 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                     const uint32_t sb = sa + kABytes;
 #pragma unroll
-                    for (int ks = 0; ks < BK / 16; ++ks) {
-                        // A: K-major, 8-row groups 1024 bytes apart, 32 bytes per 16-wide k step
-                        const uint64_t da = smem_desc(sa + ks * 32, 16, 1024);
-                        // B: N-major, 64-column boxes 8192 bytes apart, 8-row k groups 1024 bytes apart
-                        const uint64_t db = smem_desc(sb + ks * 2048, kBBoxBytes, 1024);
-                        tc_mma_bf16(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
+                    for (int ks = 0; ks < 4; ++ks) {          // four instructions of 32 bytes of k (16 bf16 / 8 tf32) per stage
+                        // A K-major: 8-row groups 1024 bytes apart, 32 bytes per k step.  A MN-major: like B below.
+                        const uint64_t da = kAMn ? smem_desc(sa + ks * Cfg::kMnStep, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout)
+                                                 : smem_desc(sa + ks * 32, 16, 1024);
+                        // B: N-major, 128-byte-wide boxes kBoxBytes apart, k-row atoms kMnSbo bytes apart
+                        const uint64_t db = smem_desc(sb + ks * Cfg::kMnStep, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout);
+                        if (kTf32) tc_mma_tf32(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
                     }
                     tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
                 }
@@ -436,15 +492,15 @@ bool make_map(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, u
 
 bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
-template <int BN, int kStages, bool kStaging>
+template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false>
 int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
                  const CUtensorMap& b1, const CUtensorMap& c, const TcParams& p, double flops, cudaStream_t st)
 {
-    using Cfg = TcCfg<BN, kStages, kStaging>;
+    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn>;
     static_assert(Cfg::kSmemBytes <= 227 * 1024, "shared memory budget");
     static bool attr_done[64] = {};
     if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
-        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN, kStages, kStaging>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)Cfg::kSmemBytes));
         attr_done[ctx->device] = true;
     }
@@ -453,22 +509,25 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
     if (p.mode != TC_STORE_BF16 && ctx->tc_update_ctas > 0 && grid > ctx->tc_update_ctas) grid = ctx->tc_update_ctas;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
-        gemm_tc_kernel<BN, kStages, kStaging><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, p);
+        gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, p);
     }
     return after_launch(ctx);
 }
 
 // fp32 tensor map of the matrix that the subtracting epilogue reduces into: 32 x 32 boxes, 128-byte swizzle.
-bool make_map_f32_box(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, uint64_t rows, uint64_t ld)
+bool make_map_f32_box(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, uint64_t rows, uint64_t ld,
+                      uint32_t box_rows = 32, bool chunk32 = false)
 {
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
     if (!enc) return false;
     const cuuint64_t dims[2] = { cols, rows };
     const cuuint64_t strides[1] = { ld * 4 };
-    const cuuint32_t box[2] = { 32, 32 };
+    const cuuint32_t box[2] = { 32, box_rows };
     const cuuint32_t estr[2] = { 1, 1 };
+    // chunk32: the 128-byte swizzle that moves 32-byte chunks, which the MMA wants for fp32 tiles that are not K-major
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(ptr), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, chunk32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B,
+               CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -602,6 +661,58 @@ int launch_gemm_tc_split_k(gelo_ctx* ctx, int M, int N, int K, const void* Ahi, 
     p.ksplit = ksplit; p.kb_per_split = per; p.plane = (long long)plane;
     if (used) *used = ksplit;
     return launch_tiles<256, 4, false>(ctx, a0, a1, b0, b1, a0, p, 6.0 * M * (double)N * K, st);
+}
+
+// One-product tf32 GEMM on fp32 matrices, fp32 accumulation:  P = op(A) (M x K) * B (K x N, row-major, stride ldb).
+//   a_mn = false : A is row-major M x K (stride lda);  a_mn = true : A points at a row-major K x M matrix (stride lda)
+//                  and the product uses its transpose.
+//   mode TC_SUB_F32   : C (fp32, stride ldc) -= P, in place, by TMA reduce-add
+//   mode TC_STORE_F32 : C = P, or with round_out C = post_scale * (out_scale * P - diag_sub * I) rounded to tf32, or
+//                       with ksplit > 1 the partial products of the K slices
+//                       go to consecutive planes of C (plane stride in elements); *used = slices written
+int launch_gemm_tf32(gelo_ctx* ctx, int M, int N, int K, const float* A, int lda, bool a_mn, const float* B, int ldb,
+                     bool subtract, float* C, int ldc, bool round_out, float out_scale, int ksplit, size_t plane, int* used,
+                     cudaStream_t st, float diag_sub, float post_scale)
+{
+    if (used) *used = 0;
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if ((lda % 4) || (ldb % 4) || (ldc % 4) || !aligned16(A) || !aligned16(B) || !aligned16(C) || !C) return GELO_ERR_INVALID;
+    if (!subtract && (N % 8)) return GELO_ERR_INVALID;
+    if (subtract && ksplit > 1) return GELO_ERR_INVALID;
+    CUtensorMap ma, mb, mc;
+    const bool a_ok = a_mn ? make_map_f32_box(ctx, &ma, A, (uint64_t)M, (uint64_t)K, (uint64_t)lda, 32, true)
+                           : make_map_f32_box(ctx, &ma, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM);
+    if (!a_ok || !make_map_f32_box(ctx, &mb, B, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, true)) return GELO_ERR_CUDA;
+    mc = ma;
+    TcParams p = {};
+    p.M = M; p.N = N;
+    const int kb = ceil_div(K, 32);
+    p.nseg = 1;
+    p.seg[0] = TcSegment{0, 0, 0, 0, kb};
+    p.status = ctx->status_dev;
+    p.csplit = N;
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
+    p.round_tf32 = round_out ? 1 : 0;
+    p.out_scale = out_scale; p.diag_sub = diag_sub; p.post_scale = post_scale;
+    p.C0 = C; p.ldc = ldc;
+    const double flops = 2.0 * M * (double)N * K;
+    if (subtract) {
+        if (!make_map_f32_box(ctx, &mc, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc, 32)) return GELO_ERR_CUDA;
+        p.mode = TC_SUB_F32;
+        return a_mn ? launch_tiles<256, 3, true, true, true>(ctx, ma, ma, mb, mb, mc, p, flops, st)
+                    : launch_tiles<256, 3, true, true, false>(ctx, ma, ma, mb, mb, mc, p, flops, st);
+    }
+    p.mode = TC_STORE_F32;
+    if (ksplit > 1) {
+        if (ksplit > kb) ksplit = kb;
+        const int per = ceil_div(kb, ksplit);
+        ksplit = ceil_div(kb, per);                // no empty slice
+        p.ksplit = ksplit; p.kb_per_split = per; p.plane = (long long)plane;
+    }
+    if (used) *used = p.ksplit;
+    return a_mn ? launch_tiles<256, 4, false, true, true>(ctx, ma, ma, mb, mb, mc, p, flops, st)
+                : launch_tiles<256, 4, false, true, false>(ctx, ma, ma, mb, mb, mc, p, flops, st);
 }
 
 }  // namespace gelo

@@ -112,6 +112,28 @@ __global__ void __launch_bounds__(256) sum_split_kernel(const float* __restrict_
     *reinterpret_cast<uint2*>(lo + (size_t)r * ldo + c4) = *reinterpret_cast<const uint2*>(l);
 }
 
+// Sum of `parts` fp32 planes (fixed order), rounded to tf32: the second half of a split-K tf32 product whose
+// result feeds the next tf32 product.
+__global__ void __launch_bounds__(256) sum_planes_kernel(const float* __restrict__ planes, size_t plane, int parts,
+                                                         int ld, int rows, int cols, float scale, float* __restrict__ out,
+                                                         int ldo)
+{
+    const int c4 = (blockIdx.x * 256 + threadIdx.x) * 4;
+    const int r = blockIdx.y;
+    if (c4 >= cols) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < parts; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(planes + q * plane + (size_t)r * ld + c4);
+        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    }
+    uint32_t o[4];
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o[0]) : "f"(scale * acc.x));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o[1]) : "f"(scale * acc.y));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o[2]) : "f"(scale * acc.z));
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(o[3]) : "f"(scale * acc.w));
+    *reinterpret_cast<uint4*>(out + (size_t)r * ldo + c4) = make_uint4(o[0], o[1], o[2], o[3]);
+}
+
 __global__ void __launch_bounds__(256) split_transpose_kernel(const float* __restrict__ src, int lds, int rows, int cols,
                                                               __nv_bfloat16* __restrict__ hi, __nv_bfloat16* __restrict__ lo, int ldo)
 {
@@ -164,6 +186,15 @@ int launch_sum_split(gelo_ctx* ctx, const float* planes, size_t plane, int parts
     dim3 grid(ceil_div(cols, 1024), rows);
     sum_split_kernel<<<grid, 256, 0, st>>>(planes, plane, parts, ld, rows, cols, static_cast<__nv_bfloat16*>(hi),
                                            static_cast<__nv_bfloat16*>(lo), ldo);
+    return after_launch(ctx);
+}
+
+int launch_sum_planes(gelo_ctx* ctx, const float* planes, size_t plane, int parts, int ld, int rows, int cols, float scale,
+                      float* out, int ldo, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return GELO_OK;
+    dim3 grid(ceil_div(cols, 1024), rows);
+    sum_planes_kernel<<<grid, 256, 0, st>>>(planes, plane, parts, ld, rows, cols, scale, out, ldo);
     return after_launch(ctx);
 }
 

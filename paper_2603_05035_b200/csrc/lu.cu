@@ -511,7 +511,7 @@ LuScratch carve_lu(Arena& a, int m, int ld)
 // updates above run on the block only; everything outside the block is updated once per block by a
 // split-precision tensor-core product (K = kOuter), which cuts the passes over the big matrices by four.
 int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const LuScratch& s, const TcScratch& tc,
-                      cudaStream_t st)
+                      bool tf32, cudaStream_t st)
 {
     float* M = s.M;
     GELO_CUDA_OK(cudaMemcpyAsync(M, A, (size_t)m * ld * sizeof(float), cudaMemcpyDeviceToDevice, st));
@@ -540,7 +540,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         // U12 = L11^-1 A12 on the block's row strip
         GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, M, ld, b0, ob, bend, m, st));
         // A22 -= L21 U12
-        GELO_TRY(tc_update_f32(ctx, tc, nc, nc, ob, M + (size_t)bend * ld + b0, ld, M + (size_t)b0 * ld + bend, ld,
+        GELO_TRY(tc_update_f32(ctx, tc, tf32, nc, nc, ob, M + (size_t)bend * ld + b0, ld, M + (size_t)b0 * ld + bend, ld,
                                M + (size_t)bend * ld + bend, ld, st));
     }
     // ---- X = P, then L Y = P, then U X = Y ----
@@ -556,7 +556,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         const int bend = b0 + ob;
         GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
         if (m - bend > 0)
-            GELO_TRY(tc_update_f32(ctx, tc, m - bend, m, ob, M + (size_t)bend * ld + b0, ld, X + (size_t)b0 * ld, ld,
+            GELO_TRY(tc_update_f32(ctx, tc, tf32, m - bend, m, ob, M + (size_t)bend * ld + b0, ld, X + (size_t)b0 * ld, ld,
                                    X + (size_t)bend * ld, ld, st));
     }
     const int nblocks = ceil_div(m, kOuter);
@@ -566,7 +566,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         const int bend = b0 + ob;
         GELO_TRY(launch_tri_solve128<true>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
         if (b0 > 0)
-            GELO_TRY(tc_update_f32(ctx, tc, b0, m, ob, M + b0, ld, X + (size_t)b0 * ld, ld, X, ld, st));
+            GELO_TRY(tc_update_f32(ctx, tc, tf32, b0, m, ob, M + b0, ld, X + (size_t)b0 * ld, ld, X, ld, st));
     }
     return GELO_OK;
 }

@@ -272,14 +272,16 @@ TcScratch carve_tc(Arena& a, int m, int ld)
     t.t128 = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
     t.gram = static_cast<float*>(a.take((size_t)(m / 256 + 2) * kOuter * kOuter * 4));   // one partial Gram per 256-row slab
     t.wf32 = static_cast<float*>(a.take((size_t)kMaxKSplit * kOuter * ld * 4));
+    for (int h = 0; h < 2; ++h) t.w32[h] = static_cast<float*>(a.take((size_t)kOuter * ld * 4));
     return t;
 }
 
-int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, int M, int N, int K, const float* A, int lda, const float* B,
-                  int ldb, float* C, int ldc, cudaStream_t st)
+int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, bool tf32, int M, int N, int K, const float* A, int lda,
+                  const float* B, int ldb, float* C, int ldc, cudaStream_t st)
 {
     if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
     if (K > kOuter) return GELO_ERR_INVALID;
+    if (tf32) return launch_gemm_tf32(ctx, M, N, K, A, lda, false, B, ldb, true, C, ldc, false, 1.0f, 1, 0, nullptr, st);
     const int ldn = (N + 7) & ~7;
     GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], kOuter, false, st));
     GELO_TRY(launch_split(ctx, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, false, st));

@@ -475,6 +475,78 @@ def test_householder_qr_tensor_core_blocks(oracle, m):
     c.close()
 
 
+# ------------------------------------------------------------------------- tf32 tensor-core updates
+
+@pytest.mark.parametrize("M,N,K", [(128, 256, 128), (300, 520, 128), (1000, 776, 96), (4300, 4172, 128), (64, 8, 32),
+                                    (130, 4, 8)])
+def test_tensor_core_update_tf32(ctx, oracle, M, N, K):
+    """C -= A B as one tf32 product straight from the fp32 operands (no operand conversion passes)."""
+    rng = np.random.default_rng(M + N + K)
+    lda = (K + 3) // 4 * 4
+    ldb = (N + 63) // 64 * 64
+    A0 = rng.standard_normal((M, K)).astype(np.float32)
+    B0 = rng.standard_normal((K, N)).astype(np.float32)
+    C0 = rng.standard_normal((M, N)).astype(np.float32)
+    A = torch.zeros((M, lda), device="cuda"); A[:, :K] = dev(A0)
+    B = padded(K, ldb, torch.float32); B[:, :N] = dev(B0)
+    C = padded(M, ldb, torch.float32); C[:, :N] = dev(C0)
+    ctx.set_level3(3)
+    try:
+        ctx.update_f32(M, N, K, A, lda, B, ldb, C, ldb)
+    finally:
+        ctx.set_level3(0)
+    a64, b64 = A0.astype(np.float64), B0.astype(np.float64)
+    prod = oracle.matmul(a64, b64) if M * N * K < 3e8 else a64 @ b64
+    got = f64(C[:, :N])
+    err = got - (C0.astype(np.float64) - prod)
+    # the tensor core keeps 10 fraction bits of each operand and drops the rest: every term loses up to 2^-10 per
+    # operand, 2^-11 / (2 ln 2) on average for log-uniformly spread mantissas, i.e. 7.0e-4 for the product
+    assert np.linalg.norm(err) / np.linalg.norm(prod) <= 1.2e-3
+    loss = -np.sum(err * prod) / np.sum(prod * prod)
+    if M * N >= 128 * 256:
+        assert abs(loss - 2 * 3.5224e-4) <= 5e-5
+    assert torch.isnan(C[:, N:]).all()                     # padding columns are never written
+
+
+@pytest.mark.parametrize("m", [100, 130, 257, 512, 1000])
+def test_householder_qr_tf32_blocks(oracle, m):
+    """QR with tf32 level-3 updates and the Newton-Schulz polish, as the bf16 path runs it."""
+    c = make_ctx(m, 0, 8, 24, "f32")
+    c.set_level3(3)
+    ld = c.mixing_ld(m)
+    G64 = oracle.gaussian(500 + m, 0, 0, m, m).astype(np.float32).astype(np.float64)
+    G = padded(m, ld, torch.float32); G[:, :m] = dev(G64)
+    Q = padded(m, ld, torch.float32)
+    c.qr_orthogonal(m, G, ld, Q)
+    q = f64(Q[:, :m]); r = np.triu(f64(G[:, :m]))
+    s = np.where(np.diag(r) < 0, -1.0, 1.0)
+    d = q.T @ q - np.eye(m)
+    # polished: what is left is the zero-mean tf32 noise of Q^T Q (about 3e-4), far below the 1.6e-3 that rounding A
+    # to bf16 adds afterwards; the trace shows that no coherent shrinkage survives
+    assert np.linalg.norm(d) / np.sqrt(m) <= 6e-4
+    assert abs(np.trace(d)) / m <= 1e-4
+    # the factorisation itself is tf32-grade
+    assert np.linalg.norm(q @ (r.T * s).T - G64) / np.linalg.norm(G64) <= 5e-3
+    q_ref, _ = oracle.householder_qr(G64)
+    assert np.all(np.sum(q * q_ref, axis=0)[: max(1, m // 2)] > 1 - 5e-3)
+    assert c.last_status() == binding.OK
+    c.close()
+
+
+def test_orthogonal_sample_bf16_benchmark_size(ctx):
+    """Orthogonal A at the benchmark size on the default (tf32 + polish) route: A^T A = I up to bf16 rounding."""
+    m = 4300
+    lda = ctx.mixing_ld(m)
+    A = padded(m, lda, torch.bfloat16); X = padded(m, lda, torch.bfloat16)
+    ctx.sample_mixing(m, ORTHOGONAL, 31337, "bf16", A, X, lda)
+    a = A[:, :m].double()
+    assert torch.equal(X[:, :m], A[:, :m].t())
+    d = a.t() @ a - torch.eye(m, device="cuda", dtype=torch.float64)
+    # bf16 rounding alone gives 2^-9 / sqrt(3) per entry pair, about 1.6e-3 here
+    assert d.norm().item() / np.sqrt(m) <= 2.0e-3
+    assert abs(torch.trace(d).item()) / m <= 2e-4
+
+
 # ------------------------------------------------------------------------- attention output projection
 
 @pytest.mark.parametrize("dt", ["f32", "bf16"])
