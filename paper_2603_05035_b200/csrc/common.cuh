@@ -198,6 +198,10 @@ struct TcScratch;
 // Same factorisation with 128-column outer blocks whose updates run on the tensor cores in split precision.
 int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, bool tf32,
                           cudaStream_t);
+// The tf32 route: 128-column blocks grouped four by four; only the group's merged reflector (512 columns) is
+// applied to the columns right of the group and, later, to Q, so the big matrices stream through the GPU once per
+// 512 columns instead of once per 128.
+int run_householder_qr_tf32(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, cudaStream_t);
 // One Newton-Schulz step Q <- Q - Q (Q^T Q - I) / 2 on the tensor cores in tf32: squares the orthogonality defect
 // that tf32 updates leave in Q.  D and Qold are m x ld scratch matrices.
 int polish_orthogonal_tf32(gelo_ctx*, int m, float* Q, int ld, float* D, float* Qold, cudaStream_t);
@@ -246,7 +250,9 @@ int launch_sum_planes(gelo_ctx*, const float* planes, size_t plane, int parts, i
 
 // Scratch of the tensor-core level-3 updates (outer blocks of kOuter columns).
 constexpr int kOuter = 128;
+constexpr int kSuper = 4 * kOuter;        // columns whose reflectors reach the rest of the matrix in one tf32 update
 constexpr int kMaxKSplit = 16;
+constexpr int kSuperKSplit = kMaxKSplit * kOuter / kSuper;   // K slices of a kSuper-row product that fit the same planes
 struct TcScratch {
     void* panA[2] = {nullptr, nullptr};    // m x kOuter          block column (V or L), hi / lo
     void* panAt[2] = {nullptr, nullptr};   // kOuter x ld         its transpose
@@ -257,7 +263,10 @@ struct TcScratch {
     float* t128 = nullptr;                 // kOuter x kOuter fp32
     float* gram = nullptr;                 // kOuter x kOuter fp32
     float* wf32 = nullptr;                 // kMaxKSplit planes of kOuter x ld fp32 (split-K partial products)
-    float* w32[2] = {nullptr, nullptr};    // kOuter x ld fp32    block rows W and T W of the tf32 updates
+    float* w32[2] = {nullptr, nullptr};    // kSuper x ld fp32    block rows W and T W of the tf32 updates
+    float* tsuper = nullptr;               // ceil(m / kSuper) merged triangular factors, kSuper x kSuper each
+    float* sx = nullptr;                   // kOuter x kSuper     V_i^T V_(<i) of the block being merged
+    float* xb = nullptr;                   // kSuper x kOuter     its product with T_i
 };
 TcScratch carve_tc(Arena&, int m, int ld);
 // C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores: three bf16 products of

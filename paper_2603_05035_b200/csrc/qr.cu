@@ -616,6 +616,117 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
     return GELO_OK;
 }
 
+// Blocked QR whose level-3 work is tf32 products read straight from the fp32 matrices.  Panels of 32 columns and
+// blocks of 128 run as in run_householder_qr_tc.  Blocks are grouped into superblocks of kSuper = 512 columns:
+//   * inside a superblock a finished block is applied to the superblock's remaining columns only, and its factor
+//     is merged into the superblock's factor:  with S = V_i^T V_(<i),
+//         T(1..i) = [[T(1..i-1), -T(1..i-1) S^T T_i], [0, T_i]];
+//   * the columns right of the superblock see ONE update C <- (I - V T^T V^T) C with all 512 reflectors, and Q is
+//     accumulated backwards with one such update (with T) per superblock.
+// A trailing update with 512 reflectors does four times the arithmetic of one with 128 per byte of C moved, which
+// is what the 128-column updates were short of (they ran at the speed of the memory system, not of the tensor cores).
+int run_householder_qr_tf32(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const QrScratch& s, const TcScratch& tc,
+                            cudaStream_t st)
+{
+    GELO_CUDA_OK(cudaMemsetAsync(s.V, 0, (size_t)m * ld * sizeof(float), st));
+    GELO_CUDA_OK(cudaFuncSetAttribute(t_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemBytes));
+    const float back2 = (1.0f + kTf32TruncLoss) * (1.0f + kTf32TruncLoss);
+    const int width = ctx->tc_update_ctas > 0 ? ctx->tc_update_ctas : ctx->sm_count;   // CTAs one launch may use
+
+    // C (nr x nc, rows from row r0 of the matrix) <- (I - V op(T) V^T) C with V = reflector columns c0 .. c0+kv-1
+    // (rows from r0 = c0), T: kv x kv with row stride ldt; planes hold `maxsplit` slices of kv x ld.
+    auto apply = [&](int c0, int kv, const float* T, int ldt, float* C, int nc, bool transpose_t, int maxsplit) -> int {
+        const int nr = m - c0;
+        const int nc8 = (nc + 7) & ~7;
+        const float* Vb = s.V + (size_t)c0 * ld + c0;
+        // W = V^T C contracts over all nr rows: with few output tiles the rows are cut into slices (summed in a fixed
+        // order afterwards) so that the launch still fills its CTAs; with enough tiles it is one plain product
+        const int tiles = ceil_div(kv, 128) * ceil_div(nc8, 256);
+        int want = (2 * tiles >= width) ? 1 : ceil_div(2 * width, tiles);
+        if (want > maxsplit) want = maxsplit;
+        if (want <= 1) {
+            GELO_TRY(launch_gemm_tf32(ctx, kv, nc8, nr, Vb, ld, true, C, ld, false, tc.w32[0], ld, true, 1.0f, 1, 0, nullptr, st));
+        } else {
+            int used = 0;
+            const size_t plane = (size_t)kv * ld;
+            GELO_TRY(launch_gemm_tf32(ctx, kv, nc8, nr, Vb, ld, true, C, ld, false, tc.wf32, ld, false, 1.0f, want, plane, &used, st));
+            GELO_TRY(launch_sum_planes(ctx, tc.wf32, plane, used, ld, kv, nc8, 1.0f, tc.w32[0], ld, st));
+        }
+        GELO_TRY(launch_gemm_tf32(ctx, kv, nc8, kv, T, ldt, transpose_t, tc.w32[0], ld, false, tc.w32[1], ld, true, 1.0f, 1, 0,
+                                  nullptr, st));
+        return launch_gemm_tf32(ctx, nr, nc, kv, Vb, ld, false, tc.w32[1], ld, true, C, ld, false, 1.0f, 1, 0, nullptr, st);
+    };
+
+    const int nsuper = ceil_div(m, kSuper);
+    // ---- factorisation ----
+    for (int sb = 0; sb < nsuper; ++sb) {
+        const int s0 = sb * kSuper;
+        const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+        const int send = s0 + sw;
+        float* Ts = tc.tsuper + (size_t)sb * kSuper * kSuper;
+        GELO_CUDA_OK(cudaMemsetAsync(Ts, 0, (size_t)kSuper * kSuper * sizeof(float), st));
+        for (int b0 = s0; b0 < send; b0 += kOuter) {
+            const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+            const int bend = b0 + ob;
+            for (int j0 = b0; j0 < bend; j0 += NB) {
+                const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
+                float* Tp = s.T + (size_t)(j0 / NB) * NB * NB;
+                GELO_TRY(launch_qr_panel(ctx, R, ld, m, j0, jb, s.V, Tp, st));
+                const int ncb = bend - (j0 + jb), nr = m - j0;
+                if (ncb > 0) {
+                    float* C = R + (size_t)j0 * ld + j0 + jb;
+                    const float* Vp = s.V + (size_t)j0 * ld + j0;
+                    GELO_TRY(launch_vtc(ctx, Vp, ld, jb, C, ld, nr, ncb, Tp, true, s.Wp, s.W2, ld, st));
+                    GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, ncb, jb, st));
+                }
+            }
+            // block factor T_i from the Gram matrix of the block's reflectors and the panel factors
+            const float* Vb = s.V + (size_t)b0 * ld + b0;
+            const int slabs = ceil_div(m - b0, kGramRows);
+            gram128_kernel<<<slabs, 256, 0, st>>>(Vb, ld, m - b0, ob, tc.gram);
+            GELO_TRY(after_launch(ctx));
+            float* Tb = s.T128 + (size_t)(b0 / kOuter) * 128 * 128;
+            t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.gram, slabs, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
+            GELO_TRY(after_launch(ctx));
+            // ... into the superblock's factor
+            const int r = b0 - s0;                           // reflector columns already merged
+            GELO_CUDA_OK(cudaMemcpy2DAsync(Ts + (size_t)r * kSuper + r, (size_t)kSuper * sizeof(float), Tb, 128 * sizeof(float),
+                                           (size_t)ob * sizeof(float), ob, cudaMemcpyDeviceToDevice, st));
+            if (r > 0) {
+                const int nr = m - b0;
+                const int ob8 = (ob + 7) & ~7;
+                // S = V_i^T V_(<i)  (ob x r); both operands reach the tensor core truncated
+                int want = ceil_div(2 * width, ceil_div(r, 256));
+                if (want > kMaxKSplit) want = kMaxKSplit;
+                int used = 0;
+                const size_t plane = (size_t)kOuter * ld;
+                GELO_TRY(launch_gemm_tf32(ctx, ob, r, nr, Vb, ld, true, s.V + (size_t)b0 * ld + s0, ld, false, tc.wf32, ld, false,
+                                          1.0f, want, plane, &used, st));
+                GELO_TRY(launch_sum_planes(ctx, tc.wf32, plane, used, ld, ob, r, back2, tc.sx, kSuper, st));
+                // X = S^T T_i  (r x ob),  then  T[0:r, r:r+ob] = -T[0:r, 0:r] X  (that part of T is still zero)
+                GELO_TRY(launch_gemm_tf32(ctx, r, ob8, ob, tc.sx, kSuper, true, Tb, 128, false, tc.xb, kOuter, true, 1.0f, 1, 0,
+                                          nullptr, st));
+                GELO_TRY(launch_gemm_tf32(ctx, r, ob, r, Ts, kSuper, false, tc.xb, kOuter, true, Ts + r, kSuper, false, 1.0f, 1, 0,
+                                          nullptr, st));
+            }
+            // the block's own reflector on the remaining columns of the superblock
+            if (send > bend) GELO_TRY(apply(b0, ob, Tb, 128, R + (size_t)b0 * ld + bend, send - bend, true, kMaxKSplit));
+        }
+        // the merged reflector on everything right of the superblock
+        if (m > send) GELO_TRY(apply(s0, sw, Ts, kSuper, R + (size_t)s0 * ld + send, m - send, true, kSuperKSplit));
+    }
+    // ---- accumulate Q backwards from the identity, one superblock at a time ----
+    set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
+    GELO_TRY(after_launch(ctx));
+    for (int sb = nsuper - 1; sb >= 0; --sb) {
+        const int s0 = sb * kSuper;
+        const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+        GELO_TRY(apply(s0, sw, tc.tsuper + (size_t)sb * kSuper * kSuper, kSuper, Q + (size_t)s0 * ld + s0, m - s0, false,
+                       kSuperKSplit));
+    }
+    return GELO_OK;
+}
+
 // The tf32 updates leave Q orthogonal to a few 1e-3 only (the tensor core truncates unrounded operands, which
 // shrinks every block reflector a little).  One Newton-Schulz step, Q <- Q - Q D with D = (Q^T Q - I) / 2, squares
 // that defect.  Both products are single large tf32 GEMMs.  Q is dense with log-uniformly spread mantissas, so the

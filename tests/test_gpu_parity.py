@@ -502,7 +502,7 @@ def test_tensor_core_update_tf32(ctx, oracle, M, N, K):
     # the tensor core keeps 10 fraction bits of each operand and drops the rest: every term loses up to 2^-10 per
     # operand, 2^-11 / (2 ln 2) on average for log-uniformly spread mantissas, i.e. 7.0e-4 for the product
     assert np.linalg.norm(err) / np.linalg.norm(prod) <= 1.2e-3
-    loss = -np.sum(err * prod) / np.sum(prod * prod)
+    loss = np.sum(err * prod) / np.sum(prod * prod)          # C - (1 - loss) A B against C - A B
     if M * N >= 128 * 256:
         assert abs(loss - 2 * 3.5224e-4) <= 5e-5
     assert torch.isnan(C[:, N:]).all()                     # padding columns are never written
@@ -542,8 +542,9 @@ def test_orthogonal_sample_bf16_benchmark_size(ctx):
     a = A[:, :m].double()
     assert torch.equal(X[:, :m], A[:, :m].t())
     d = a.t() @ a - torch.eye(m, device="cuda", dtype=torch.float64)
-    # bf16 rounding alone gives 2^-9 / sqrt(3) per entry pair, about 1.6e-3 here
-    assert d.norm().item() / np.sqrt(m) <= 2.0e-3
+    # bf16 rounding alone: relative errors uniform in +-2^-9 on both factors of every term, 2^-9 sqrt(2/3) = 1.6e-3
+    # per off-diagonal entry pair and twice that on the diagonal, 2.35e-3 in this norm; the polished Q adds 3e-4
+    assert d.norm().item() / np.sqrt(m) <= 2.6e-3
     assert abs(torch.trace(d).item()) / m <= 2e-4
 
 
