@@ -415,9 +415,9 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--lanes", type=int, default=16, help="concurrent sampling lanes of the batched call (1..16)")
+    ap.add_argument("--lanes", type=int, default=32, help="concurrent sampling lanes of the batched call (1..32)")
     ap.add_argument("--lane-share", type=int, default=4, help="each level-3 update uses 1/share of the SMs in batches")
-    ap.add_argument("--level3", type=int, default=0, choices=[0, 1, 2],
+    ap.add_argument("--level3", type=int, default=0, choices=[0, 1, 2, 3],
                     help="factorisation updates: 0 auto (tensor cores for bf16), 1 fp32 FMA, 2 tensor cores")
     ap.add_argument("--calls", type=int, default=0, help="projection calls per step (default: the workload's 32)")
     ap.add_argument("--timed-only", action="store_true",
