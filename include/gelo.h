@@ -129,7 +129,8 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
 int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ainv_dev, void* stream);
 
 /* cond_dev[0] = estimate of kappa_2(A) = sigma_max(A) * sigma_max(A^-1) by power
- * iteration on A^T A and A^-T A^-1 (a lower estimate, within a few percent). */
+ * iteration on A^T A and A^-T A^-1 (a lower estimate, within a few percent).  ld must be a multiple of 8
+ * and both matrices 16-byte aligned. */
 int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
                        float* cond_dev, void* stream);
 
@@ -244,6 +245,17 @@ int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_h
                                 const uint64_t* seeds, float shield_scale, int dtype,
                                 void* const* Q_host, void* const* K_host, void* const* V_host,
                                 void* stream);
+
+/* The same call without the final wait: it returns once everything is enqueued on `stream`, and the host
+ * results are valid after the caller has synchronised `stream` (the host buffers must stay alive and, for
+ * the copies to be asynchronous at all, be pinned).  Back-to-back calls then keep the sampling lanes busy
+ * across the seam, exactly as gelo_qkv_offload_batch does: the lanes already sample the mixing pairs of
+ * the next batch while the last results of this one are still on their way to the host. */
+int gelo_qkv_offload_batch_host_async(gelo_ctx* ctx, int calls, const void* const* H_host,
+                                      const void* const* W_dev, int n, int k, int d, int p, const int* kinds,
+                                      const uint64_t* seeds, float shield_scale, int dtype,
+                                      void* const* Q_host, void* const* K_host, void* const* V_host,
+                                      void* stream);
 
 /* Number of concurrent sampling lanes of the batched calls (1..32, default 4) and the workspace
  * they need.  0 bytes if an argument is invalid. */

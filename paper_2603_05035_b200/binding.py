@@ -57,6 +57,7 @@ EXPORTS = {
     "gelo_qkv_offload": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_qkv_offload_batch_host_async": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_lanes": (_i, [_vp, _i]),
     "gelo_set_lane_share": (_i, [_vp, _i]),
     "gelo_batch_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
@@ -300,6 +301,12 @@ class Context:
                                V_host=None, stream=None):
         self._batch(self._lib.gelo_qkv_offload_batch_host, "gelo_qkv_offload_batch_host", H_host, W, n, k, d, p,
                     kinds, seeds, shield_scale, dtype, Q_host, K_host, V_host, stream)
+
+    def qkv_offload_batch_host_async(self, H_host, W, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host=None,
+                                     V_host=None, stream=None):
+        """Enqueues the batch and returns; read the host results after synchronising the stream."""
+        self._batch(self._lib.gelo_qkv_offload_batch_host_async, "gelo_qkv_offload_batch_host_async", H_host, W, n, k,
+                    d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host, V_host, stream)
 
     def qkv_offload_host(self, H_host, W, n, k, d, p, kind, seed, shield_scale, dtype, Q_host, K_host=None,
                          V_host=None, stream=None):

@@ -145,8 +145,9 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     if (l3lu) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, ldi, L.X32, L.lu, L.tc, l3lu == 3, st));
     else GELO_TRY(run_lu_inverse(ctx, m, L.A32, ldi, L.X32, L.lu, st));
     GELO_TRY(launch_narrow(ctx, m, L.X32, ldi, dtype, Ainv_out, lda, st));
-    return run_cond_estimate(ctx, m, L.A32, L.X32, ldi, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond, st,
-                             deferred);
+    // the verified matrices are the stored ones: what mix and unmix will read
+    return run_cond_estimate(ctx, m, A_out, Ainv_out, lda, dtype, ctx->cond_bound, cond_dev ? cond_dev : L.cond_val, L.cond,
+                             st, deferred);
 }
 
 int sample_mixing_impl(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t seed, int dtype,
@@ -276,7 +277,7 @@ int sample_on_lane(gelo_ctx* ctx, const Layout& L, int lane, int m, int kind, ui
 // the status word (GELO_ERR_COND) instead of a resample, because nothing here waits for the device.
 int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const void* const* W, int n, int k, int d,
                        int p, const int* kinds, const uint64_t* seeds, float shield_scale, int dtype,
-                       void* const* Q, void* const* K, void* const* V, cudaStream_t st, bool host)
+                       void* const* Q, void* const* K, void* const* V, cudaStream_t st, bool host, bool wait = true)
 {
     const int m = n + k;
     const int D = calls < ctx->lanes ? calls : ctx->lanes;
@@ -346,7 +347,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     ctx->chain_stream = st;
     ctx->chain_key = L[D - 1].G;
     ctx->chain_lanes = D;
-    if (host) GELO_CUDA_OK(cudaStreamSynchronize(st));
+    if (host && wait) GELO_CUDA_OK(cudaStreamSynchronize(st));
     return GELO_OK;
 }
 
@@ -576,7 +577,7 @@ int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ai
     DeviceGuard guard(ctx->device);
     Layout L;
     if (!carve_ctx(ctx, m, 0, 0, 0, GELO_F32, false, &L)) return GELO_ERR_WORKSPACE;
-    return run_cond_estimate(ctx, m, A_dev, Ainv_dev, ld, ctx->cond_bound, cond_dev, L.cond, as_stream(stream));
+    return run_cond_estimate(ctx, m, A_dev, Ainv_dev, ld, GELO_F32, ctx->cond_bound, cond_dev, L.cond, as_stream(stream));
 }
 
 int gelo_sample_mixing(gelo_ctx* ctx, int m, int kind, uint64_t seed, int dtype, void* A_dev, void* Ainv_dev,
@@ -729,6 +730,18 @@ int gelo_qkv_offload_batch_host(gelo_ctx* ctx, int calls, const void* const* H_h
     DeviceGuard guard(ctx->device);
     return offload_batch_impl(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host,
                               V_host, as_stream(stream), true);
+}
+
+int gelo_qkv_offload_batch_host_async(gelo_ctx* ctx, int calls, const void* const* H_host, const void* const* W_dev,
+                                      int n, int k, int d, int p, const int* kinds, const uint64_t* seeds,
+                                      float shield_scale, int dtype, void* const* Q_host, void* const* K_host,
+                                      void* const* V_host, void* stream)
+{
+    GELO_TRY(check_batch_args(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, dtype, Q_host, K_host, V_host, true));
+    if (calls == 0) return GELO_OK;
+    DeviceGuard guard(ctx->device);
+    return offload_batch_impl(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host,
+                              V_host, as_stream(stream), true, false);
 }
 
 int gelo_profile_start(gelo_ctx* ctx)

@@ -224,7 +224,8 @@ struct CondScratch {
 };
 CondScratch carve_cond(Arena&, int m);
 // cond_out[0] = estimate; status_dev[1] = (estimate * 1.1 <= bound)
-int run_cond_estimate(gelo_ctx*, int m, const float* A, const float* Ainv, int ld, float bound,
+// A, Ainv: m x m matrices of type `dtype` with row stride ld (a multiple of 8)
+int run_cond_estimate(gelo_ctx*, int m, const void* A, const void* Ainv, int ld, int dtype, float bound,
                       float* cond_out, const CondScratch&, cudaStream_t, bool deferred = false);
 
 // ---- layout helpers ----------------------------------------------------------------------

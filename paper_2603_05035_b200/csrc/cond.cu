@@ -2,8 +2,9 @@
 // Mitigation 1: "generate and verify well-conditioned A (e.g., enforce kappa(A) < 100)").
 // kappa_2(A) = sigma_max(A) * sigma_max(A^-1); each factor by power iteration on
 // Op^T Op with Op = A (z = 0) and Op = A^-1 (z = 1), both run in the same launches.
-// All sums have a fixed order, so the estimate is bit-reproducible.  HBM/L2-bound:
-// every iteration streams both matrices twice.
+// The operators are the matrices as stored (bf16 or fp32), i.e. exactly what the mixing and unmixing products
+// read.  All sums have a fixed order, so the estimate is bit-reproducible.  HBM-bound: every iteration streams
+// both matrices once from DRAM (the second touch of a row slab hits L2).
 #include "common.cuh"
 #include "philox.cuh"
 
@@ -11,15 +12,14 @@ namespace gelo {
 
 namespace {
 
-constexpr int kRowSlabs = 16;
-constexpr int kPowerIters = 12;   // the estimate is within about 4% of kappa_2 after 12 steps (measured at m = 512 .. 4300)
+constexpr int kCondSlabsMax = 160;   // row slabs of one operator pass (one CTA each)
+constexpr int kPowerIters = 12;      // the estimate is within about 4% of kappa_2 after 12 steps (measured at m = 512 .. 4300)
 
 struct CondViews {
-    const float* op[2];
-    int ld, m, mpad;
+    const void* op[2];
+    int ld, m, mpad, slabs, rows_per;
     float* xhat;      // [2][mpad]
-    float* y;         // [2][mpad]
-    float* partial;   // [2][kRowSlabs][mpad]
+    float* partial;   // [2][slabs][mpad]
     float* scal;      // [0..1] sigma estimates
 };
 
@@ -33,14 +33,13 @@ __global__ void cond_init_kernel(CondViews v, uint64_t seed, uint32_t attempt)
     for (int t = 0; t < 4; ++t) {
         const int i = i4 + t;
         if (i >= v.mpad) break;
-        for (int s = 0; s < kRowSlabs; ++s)
-            v.partial[((size_t)z * kRowSlabs + s) * v.mpad + i] = (s == 0 && i < v.m) ? g[t] : 0.0f;
+        for (int s = 0; s < v.slabs; ++s)
+            v.partial[((size_t)z * v.slabs + s) * v.mpad + i] = (s == 0 && i < v.m) ? g[t] : 0.0f;
     }
 }
 
 // xhat = (sum of slab partials) / its norm;  scal[z] = sqrt(norm)
-__global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v, int last, float bound,
-                                                              float* cond_out, int* status)
+__global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v)
 {
     __shared__ float red[32];
     __shared__ float total;
@@ -48,8 +47,7 @@ __global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v, int l
     float local = 0.0f;
     for (int i = threadIdx.x; i < v.m; i += blockDim.x) {
         float s = 0.0f;
-#pragma unroll
-        for (int k = 0; k < kRowSlabs; ++k) s += v.partial[((size_t)z * kRowSlabs + k) * v.mpad + i];
+        for (int k = 0; k < v.slabs; ++k) s += v.partial[((size_t)z * v.slabs + k) * v.mpad + i];
         v.xhat[(size_t)z * v.mpad + i] = s;
         local = fmaf(s, s, local);
     }
@@ -68,7 +66,6 @@ __global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v, int l
     const float inv = nrm > 0.0f ? 1.0f / nrm : 0.0f;
     for (int i = threadIdx.x; i < v.m; i += blockDim.x) v.xhat[(size_t)z * v.mpad + i] *= inv;
     if (threadIdx.x == 0) v.scal[z] = sqrtf(nrm);   // nrm -> lambda_max(Op^T Op) = sigma_max^2
-    (void)last; (void)bound; (void)cond_out; (void)status;
 }
 
 __global__ void cond_verdict_kernel(CondViews v, float bound, float* cond_out, int* status, int deferred)
@@ -81,37 +78,66 @@ __global__ void cond_verdict_kernel(CondViews v, float bound, float* cond_out, i
     if (deferred && !ok) atomicCAS(status, 0, (int)GELO_ERR_COND);
 }
 
-// y = Op xhat, one warp per row
-__global__ void __launch_bounds__(256) cond_matvec_kernel(CondViews v)
+// Eight consecutive elements of a stored row, widened to fp32 (rows start 16-byte aligned, ld is a multiple of 8).
+__device__ __forceinline__ void load8(const float* p, float (&a)[8])
 {
-    const int z = blockIdx.y;
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= v.m) return;
-    const float* a = v.op[z] + (size_t)row * v.ld;
-    const float* x = v.xhat + (size_t)z * v.mpad;
-    float s = 0.0f;
-    for (int j = lane; j < v.m; j += 32) s = fmaf(a[j], x[j], s);
+    const float4 lo = *reinterpret_cast<const float4*>(p), hi = *reinterpret_cast<const float4*>(p + 4);
+    a[0] = lo.x; a[1] = lo.y; a[2] = lo.z; a[3] = lo.w; a[4] = hi.x; a[5] = hi.y; a[6] = hi.z; a[7] = hi.w;
+}
+__device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&a)[8])
+{
+    const uint4 raw = *reinterpret_cast<const uint4*>(p);
+    const uint32_t w[4] = {raw.x, raw.y, raw.z, raw.w};
 #pragma unroll
-    for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    if (lane == 0) v.y[(size_t)z * v.mpad + row] = s;
+    for (int t = 0; t < 4; ++t) {
+        a[2 * t] = __uint_as_float(w[t] << 16);
+        a[2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u);
+    }
 }
 
-// partial[z][slab][col] = sum over the slab's rows of Op[r, col] * y[r]
-__global__ void __launch_bounds__(128) cond_matvec_t_kernel(CondViews v)
+// One power-iteration step Op^T (Op xhat) in a single pass over the operator: CTA (slab, z) first forms y_r =
+// Op[r, :] . xhat for its rows (one warp per row), then accumulates sum_r y_r Op[r, :] for every column; the
+// second read of the slab comes from L2.  partial[z][slab][:] receives the slab's contribution.
+template <typename T>
+__global__ void __launch_bounds__(256) cond_step_kernel(CondViews v)
 {
-    const int z = blockIdx.z, slab = blockIdx.y;
-    const int col = blockIdx.x * 128 + threadIdx.x;
-    const int rows_per = (v.m + kRowSlabs - 1) / kRowSlabs;
-    const int r0 = slab * rows_per;
-    const int r1 = min(v.m, r0 + rows_per);
-    if (col >= v.m) return;
-    const float* a = v.op[z];
-    const float* y = v.y + (size_t)z * v.mpad;
-    float s = 0.0f;
-#pragma unroll 4
-    for (int r = r0; r < r1; ++r) s = fmaf(a[(size_t)r * v.ld + col], y[r], s);
-    v.partial[((size_t)z * kRowSlabs + slab) * v.mpad + col] = s;
+    extern __shared__ float ys[];
+    const int z = blockIdx.y, slab = blockIdx.x;
+    const int r0 = slab * v.rows_per;
+    const int r1 = min(v.m, r0 + v.rows_per);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const T* op = static_cast<const T*>(v.op[z]);
+    const float* x = v.xhat + (size_t)z * v.mpad;
+    const int groups = (v.m + 7) >> 3;
+    for (int r = r0 + warp; r < r1; r += 8) {
+        const T* a = op + (size_t)r * v.ld;
+        float s = 0.0f;
+        for (int g = lane; g < groups; g += 32) {
+            float e[8];
+            load8(a + 8 * g, e);
+#pragma unroll
+            for (int t = 0; t < 8; ++t)
+                if (8 * g + t < v.m) s = fmaf(e[t], x[8 * g + t], s);
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
+        if (lane == 0) ys[r - r0] = s;
+    }
+    __syncthreads();
+    float* out = v.partial + ((size_t)z * v.slabs + slab) * v.mpad;
+    for (int g = threadIdx.x; g < groups; g += 256) {
+        float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
+        for (int r = r0; r < r1; ++r) {
+            float e[8];
+            load8(op + (size_t)r * v.ld + 8 * g, e);
+            const float y = ys[r - r0];
+#pragma unroll
+            for (int t = 0; t < 8; ++t) acc[t] = fmaf(e[t], y, acc[t]);
+        }
+#pragma unroll
+        for (int t = 0; t < 8; ++t)
+            if (8 * g + t < v.m) out[8 * g + t] = acc[t];
+    }
 }
 
 }  // namespace
@@ -120,33 +146,35 @@ CondScratch carve_cond(Arena& a, int m)
 {
     CondScratch s;
     const size_t mpad = (size_t)((m + 63) / 64) * 64;
-    s.vec = static_cast<float*>(a.take((4 + 2 * kRowSlabs) * mpad * sizeof(float)));
+    s.vec = static_cast<float*>(a.take((2 + 2 * kCondSlabsMax) * mpad * sizeof(float)));
     s.scal = static_cast<float*>(a.take(16 * sizeof(float)));
     return s;
 }
 
-int run_cond_estimate(gelo_ctx* ctx, int m, const float* A, const float* Ainv, int ld, float bound,
+int run_cond_estimate(gelo_ctx* ctx, int m, const void* A, const void* Ainv, int ld, int dtype, float bound,
                       float* cond_out, const CondScratch& s, cudaStream_t st, bool deferred)
 {
+    if ((ld % 8) || (reinterpret_cast<uintptr_t>(A) & 15u) || (reinterpret_cast<uintptr_t>(Ainv) & 15u)) return GELO_ERR_INVALID;
     CondViews v;
     v.op[0] = A; v.op[1] = Ainv; v.ld = ld; v.m = m; v.mpad = ((m + 63) / 64) * 64;
+    v.slabs = ceil_div(m, 32) < kCondSlabsMax ? ceil_div(m, 32) : kCondSlabsMax;
+    v.rows_per = ceil_div(m, v.slabs);
     v.xhat = s.vec;
-    v.y = s.vec + 2 * (size_t)v.mpad;
-    v.partial = s.vec + 4 * (size_t)v.mpad;
+    v.partial = s.vec + 2 * (size_t)v.mpad;
     v.scal = s.scal;
+    const size_t ys_bytes = (size_t)v.rows_per * sizeof(float);
+    if (ys_bytes > 48 * 1024) return GELO_ERR_UNSUPPORTED;
     dim3 gi(ceil_div(v.mpad, 4 * 256), 2);
     cond_init_kernel<<<gi, 256, 0, st>>>(v, 0x5eedull, 0u);
     GELO_TRY(after_launch(ctx));
-    cond_normalise_kernel<<<2, 1024, 0, st>>>(v, 0, bound, cond_out, ctx->status_dev);
+    cond_normalise_kernel<<<2, 1024, 0, st>>>(v);
     GELO_TRY(after_launch(ctx));
     for (int it = 0; it < kPowerIters; ++it) {
-        dim3 g1(ceil_div(m, 8), 2);
-        cond_matvec_kernel<<<g1, 256, 0, st>>>(v);
+        dim3 g(v.slabs, 2);
+        if (dtype == GELO_BF16) cond_step_kernel<__nv_bfloat16><<<g, 256, ys_bytes, st>>>(v);
+        else cond_step_kernel<float><<<g, 256, ys_bytes, st>>>(v);
         GELO_TRY(after_launch(ctx));
-        dim3 g2(ceil_div(m, 128), kRowSlabs, 2);
-        cond_matvec_t_kernel<<<g2, 128, 0, st>>>(v);
-        GELO_TRY(after_launch(ctx));
-        cond_normalise_kernel<<<2, 1024, 0, st>>>(v, 0, bound, cond_out, ctx->status_dev);
+        cond_normalise_kernel<<<2, 1024, 0, st>>>(v);
         GELO_TRY(after_launch(ctx));
     }
     cond_verdict_kernel<<<1, 1, 0, st>>>(v, bound, cond_out, ctx->status_dev, deferred ? 1 : 0);

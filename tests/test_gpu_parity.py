@@ -387,6 +387,15 @@ def test_batched_offload_matches_single_calls(oracle, name, calls, lanes):
     c.qkv_offload_batch_host(Hh, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Qh, Kh, Vh)
     for i in range(calls):
         assert torch.equal(Qh[i], Qb[i].cpu()) and torch.equal(Vh[i], Vb[i].cpu())
+    # the variant that does not wait: two batches back to back, results valid after the stream is synchronised
+    Qa, Ka, Va = mkh(), mkh(), mkh()
+    Q2, K2, V2 = mkh(), mkh(), mkh()
+    c.qkv_offload_batch_host_async(Hh, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Qa, Ka, Va)
+    c.qkv_offload_batch_host_async(Hh, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Q2, K2, V2)
+    torch.cuda.synchronize()
+    for i in range(calls):
+        assert torch.equal(Qa[i], Qh[i]) and torch.equal(Ka[i], Kh[i]) and torch.equal(Va[i], Vh[i])
+        assert torch.equal(Q2[i], Qh[i]) and torch.equal(V2[i], Vh[i])
     assert c.last_status() == binding.OK
     c.close()
 
