@@ -255,9 +255,9 @@ constexpr int kSuper = 4 * kOuter;        // columns whose reflectors reach the 
 constexpr int kMaxKSplit = 16;
 constexpr int kSuperKSplit = kMaxKSplit * kOuter / kSuper;   // K slices of a kSuper-row product that fit the same planes
 struct TcScratch {
-    void* panA[2] = {nullptr, nullptr};    // m x kOuter          block column (V or L), hi / lo
+    void* panA[2] = {nullptr, nullptr};    // m x kSuper          block column (V or L), hi / lo
     void* panAt[2] = {nullptr, nullptr};   // kOuter x ld         its transpose
-    void* rowB[2] = {nullptr, nullptr};    // kOuter x ld         block row (W, U12 or X rows)
+    void* rowB[2] = {nullptr, nullptr};    // kSuper x ld         block row (W, U12 or X rows)
     void* rowB2[2] = {nullptr, nullptr};   // kOuter x ld
     void* tt[2] = {nullptr, nullptr};      // kOuter x kOuter     triangular factor (transposed or not)
     void* big[2] = {nullptr, nullptr};     // m x ld              trailing matrix as a pair
@@ -270,7 +270,7 @@ struct TcScratch {
     float* xb = nullptr;                   // kSuper x kOuter     its product with T_i
 };
 TcScratch carve_tc(Arena&, int m, int ld);
-// C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kOuter, on the tensor cores: three bf16 products of
+// C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kSuper, on the tensor cores: three bf16 products of
 // (high, low) operand pairs, or (tf32) one tf32 product straight from the fp32 operands
 int tc_update_f32(gelo_ctx*, const TcScratch&, bool tf32, int M, int N, int K, const float* A, int lda, const float* B,
                   int ldb, float* C, int ldc, cudaStream_t);

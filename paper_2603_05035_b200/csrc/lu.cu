@@ -510,38 +510,60 @@ LuScratch carve_lu(Arena& a, int m, int ld)
 // Level-3 variant: outer blocks of kOuter columns.  Inside a block the 32-column panels and rank-32
 // updates above run on the block only; everything outside the block is updated once per block by a
 // split-precision tensor-core product (K = kOuter), which cuts the passes over the big matrices by four.
+// Blocked LU with partial pivoting and the inverse, level-3 work on the tensor cores.  Panels of 32 columns and
+// blocks of 128 are factorised as in run_lu_inverse; blocks are grouped into superblocks of kSuper = 512 columns.
+// Inside a superblock a finished block updates the superblock's remaining columns only; everything right of (below)
+// the superblock is updated ONCE with all 512 columns of L (rows of U), after the 512-row strip of U (of the
+// right-hand sides) has been solved block by block.  The big matrices thus stream through the GPU once per 512
+// columns instead of once per 128, which is what the 128-column updates were bound by.
 int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const LuScratch& s, const TcScratch& tc,
                       bool tf32, cudaStream_t st)
 {
     float* M = s.M;
     GELO_CUDA_OK(cudaMemcpyAsync(M, A, (size_t)m * ld * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    for (int b0 = 0; b0 < m; b0 += kOuter) {
-        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
-        const int bend = b0 + ob;
-        for (int j0 = b0; j0 < bend; j0 += NB) {
-            const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
-            GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
-            if (ob > jb) {       // interchanges on the other columns of this block
-                GELO_TRY(launch_swaps(ctx, M, ld, j0, jb, s.ipiv, s.swap_table, true, b0, bend, j0, j0 + jb, st));
+    auto at = [&](float* base, int r, int c) { return base + (size_t)r * ld + c; };
+    for (int s0 = 0; s0 < m; s0 += kSuper) {
+        const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+        const int send = s0 + sw;
+        for (int b0 = s0; b0 < send; b0 += kOuter) {
+            const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+            const int bend = b0 + ob;
+            for (int j0 = b0; j0 < bend; j0 += NB) {
+                const int jb = (bend - j0 < NB) ? (bend - j0) : NB;
+                GELO_TRY(launch_lu_panel(ctx, M, ld, m, j0, jb, s.ipiv, st));
+                if (ob > jb) {       // interchanges on the other columns of this block
+                    GELO_TRY(launch_swaps(ctx, M, ld, j0, jb, s.ipiv, s.swap_table, true, b0, bend, j0, j0 + jb, st));
+                }
+                const int ncb = bend - (j0 + jb);
+                if (ncb > 0) {
+                    tri_solve_block_kernel<false><<<ceil_div(ncb, 256), 256, 0, st>>>(M, ld, M, ld, j0, jb, j0 + jb, bend);
+                    GELO_TRY(after_launch(ctx));
+                    GELO_TRY(launch_rank_update(ctx, M + (size_t)(j0 + jb) * ld + j0, ld, M + (size_t)j0 * ld + j0 + jb, ld,
+                                                M + (size_t)(j0 + jb) * ld + j0 + jb, ld, m - j0 - jb, ncb, jb, st));
+                }
             }
-            const int ncb = bend - (j0 + jb);
-            if (ncb > 0) {
-                tri_solve_block_kernel<false><<<ceil_div(ncb, 256), 256, 0, st>>>(M, ld, M, ld, j0, jb, j0 + jb, bend);
-                GELO_TRY(after_launch(ctx));
-                GELO_TRY(launch_rank_update(ctx, M + (size_t)(j0 + jb) * ld + j0, ld, M + (size_t)j0 * ld + j0 + jb, ld,
-                                            M + (size_t)(j0 + jb) * ld + j0 + jb, ld, m - j0 - jb, ncb, jb, st));
+            if (m > ob) {            // the block's interchanges on everything left and right of it
+                GELO_TRY(launch_swaps(ctx, M, ld, b0, ob, s.ipiv, s.swap_table, true, 0, m, b0, bend, st));
+            }
+            if (send > bend) {       // the rest of the superblock: U12 = L11^-1 A12, A22 -= L21 U12
+                GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, M, ld, b0, ob, bend, send, st));
+                GELO_TRY(tc_update_f32(ctx, tc, tf32, m - bend, send - bend, ob, at(M, bend, b0), ld, at(M, b0, bend), ld,
+                                       at(M, bend, bend), ld, st));
             }
         }
-        if (m > ob) {            // the block's interchanges on everything left and right of it
-            GELO_TRY(launch_swaps(ctx, M, ld, b0, ob, s.ipiv, s.swap_table, true, 0, m, b0, bend, st));
-        }
-        const int nc = m - bend;
+        const int nc = m - send;
         if (nc <= 0) continue;
-        // U12 = L11^-1 A12 on the block's row strip
-        GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, M, ld, b0, ob, bend, m, st));
-        // A22 -= L21 U12
-        GELO_TRY(tc_update_f32(ctx, tc, tf32, nc, nc, ob, M + (size_t)bend * ld + b0, ld, M + (size_t)b0 * ld + bend, ld,
-                               M + (size_t)bend * ld + bend, ld, st));
+        // the superblock's row strip of U, block row by block row
+        for (int b0 = s0; b0 < send; b0 += kOuter) {
+            const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+            const int bend = b0 + ob;
+            GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, M, ld, b0, ob, send, m, st));
+            if (send > bend)
+                GELO_TRY(tc_update_f32(ctx, tc, tf32, send - bend, nc, ob, at(M, bend, b0), ld, at(M, b0, send), ld,
+                                       at(M, bend, send), ld, st));
+        }
+        // A22 -= L21 U12 with all sw columns at once
+        GELO_TRY(tc_update_f32(ctx, tc, tf32, nc, nc, sw, at(M, send, s0), ld, at(M, s0, send), ld, at(M, send, send), ld, st));
     }
     // ---- X = P, then L Y = P, then U X = Y ----
     const size_t perm_smem = (size_t)m * sizeof(int);
@@ -551,22 +573,34 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
     GELO_TRY(after_launch(ctx));
     permuted_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(X, ld, m, s.perm);
     GELO_TRY(after_launch(ctx));
-    for (int b0 = 0; b0 < m; b0 += kOuter) {
-        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
-        const int bend = b0 + ob;
-        GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
-        if (m - bend > 0)
-            GELO_TRY(tc_update_f32(ctx, tc, tf32, m - bend, m, ob, M + (size_t)bend * ld + b0, ld, X + (size_t)b0 * ld, ld,
-                                   X + (size_t)bend * ld, ld, st));
+    for (int s0 = 0; s0 < m; s0 += kSuper) {
+        const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+        const int send = s0 + sw;
+        for (int b0 = s0; b0 < send; b0 += kOuter) {
+            const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+            const int bend = b0 + ob;
+            GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
+            if (send > bend)
+                GELO_TRY(tc_update_f32(ctx, tc, tf32, send - bend, m, ob, at(M, bend, b0), ld, at(X, b0, 0), ld, at(X, bend, 0),
+                                       ld, st));
+        }
+        if (m > send)
+            GELO_TRY(tc_update_f32(ctx, tc, tf32, m - send, m, sw, at(M, send, s0), ld, at(X, s0, 0), ld, at(X, send, 0), ld, st));
     }
-    const int nblocks = ceil_div(m, kOuter);
-    for (int blk = nblocks - 1; blk >= 0; --blk) {
-        const int b0 = blk * kOuter;
-        const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
-        const int bend = b0 + ob;
-        GELO_TRY(launch_tri_solve128<true>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
-        if (b0 > 0)
-            GELO_TRY(tc_update_f32(ctx, tc, tf32, b0, m, ob, M + b0, ld, X + (size_t)b0 * ld, ld, X, ld, st));
+    const int nsuper = ceil_div(m, kSuper);
+    for (int sb = nsuper - 1; sb >= 0; --sb) {
+        const int s0 = sb * kSuper;
+        const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+        const int send = s0 + sw;
+        const int nblk = ceil_div(sw, kOuter);
+        for (int bi = nblk - 1; bi >= 0; --bi) {
+            const int b0 = s0 + bi * kOuter;
+            const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+            GELO_TRY(launch_tri_solve128<true>(ctx, M, ld, X, ld, b0, ob, 0, m, st));
+            if (b0 > s0)
+                GELO_TRY(tc_update_f32(ctx, tc, tf32, b0 - s0, m, ob, at(M, s0, b0), ld, at(X, b0, 0), ld, at(X, s0, 0), ld, st));
+        }
+        if (s0 > 0) GELO_TRY(tc_update_f32(ctx, tc, tf32, s0, m, sw, at(M, 0, s0), ld, at(X, s0, 0), ld, X, ld, st));
     }
     return GELO_OK;
 }

@@ -262,9 +262,9 @@ TcScratch carve_tc(Arena& a, int m, int ld)
 {
     TcScratch t;
     for (int h = 0; h < 2; ++h) {
-        t.panA[h] = a.take((size_t)m * kOuter * 2);
+        t.panA[h] = a.take((size_t)m * kSuper * 2);
         t.panAt[h] = a.take((size_t)kOuter * ld * 2);
-        t.rowB[h] = a.take((size_t)kOuter * ld * 2);
+        t.rowB[h] = a.take((size_t)kSuper * ld * 2);
         t.rowB2[h] = a.take((size_t)kOuter * ld * 2);
         t.tt[h] = a.take((size_t)kOuter * kOuter * 2);
         t.big[h] = a.take((size_t)m * ld * 2);
@@ -283,12 +283,13 @@ int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, bool tf32, int M, int N, in
                   const float* B, int ldb, float* C, int ldc, cudaStream_t st)
 {
     if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
-    if (K > kOuter) return GELO_ERR_INVALID;
+    if (K > kSuper) return GELO_ERR_INVALID;
     if (tf32) return launch_gemm_tf32(ctx, M, N, K, A, lda, false, B, ldb, true, C, ldc, false, 1.0f, 1, 0, nullptr, st);
     const int ldn = (N + 7) & ~7;
-    GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], kOuter, false, st));
+    const int ldk = (K + 63) & ~63;
+    GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], ldk, false, st));
     GELO_TRY(launch_split(ctx, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, false, st));
-    return launch_gemm_tc_split(ctx, M, N, K, t.panA[0], t.panA[1], kOuter, t.rowB[0], t.rowB[1], ldn, C, ldc,
+    return launch_gemm_tc_split(ctx, M, N, K, t.panA[0], t.panA[1], ldk, t.rowB[0], t.rowB[1], ldn, C, ldc,
                                 nullptr, nullptr, 0, false, st);
 }
 
