@@ -46,8 +46,10 @@ struct Layout {
     void* S = nullptr;        // k x d
     void* U = nullptr;        // m x d
     void* Yp = nullptr;       // m x p
-    void* Hd = nullptr;       // n x d   staging of the host variant
+    void* Hd = nullptr;       // n x d   staging of the host variants
     void* Yd = nullptr;       // n x p
+    void* Hd2 = nullptr;      // second pair: the batched host variant alternates between the two
+    void* Yd2 = nullptr;
 };
 
 Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
@@ -75,6 +77,8 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     if (host_staging) {
         L.Hd = a.take((size_t)n * d * es);
         L.Yd = a.take((size_t)n * p * es);
+        L.Hd2 = a.take((size_t)n * d * es);
+        L.Yd2 = a.take((size_t)n * p * es);
     }
     return L;
 }
@@ -315,32 +319,54 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     };
 
     for (int i = 0; i < D; ++i) GELO_TRY(enqueue_sample(i));
+    // Host variant: activations come in on the context's copy-in stream and results leave on its copy-out stream,
+    // through two staging pairs used alternately, so that the copies of call i overlap the products of calls i-1 and
+    // i+1 (the two directions use different copy engines):
+    //   copy-in :  [wait h_free_b]  H_i -> Hd_b                      -> record h_ready_b
+    //   stream  :  [wait h_ready_b] shields  [wait lane_ready, y_free_b]  mix, project, unmix -> Yd_b
+    //                                                                  -> record h_free_b, y_ready_b, lane_free
+    //   copy-out:  [wait y_ready_b] Yd_b -> Q_i, K_i, V_i              -> record y_free_b
+    // and at the end the caller's stream waits for the last copies out.
     for (int i = 0; i < calls; ++i) {
         const int l = i % D;
+        const int b = i & 1;
         const void* Hi = H[i];
-        char* y = static_cast<char*>(L[0].Yd);
+        char* y = static_cast<char*>(b ? L[0].Yd2 : L[0].Yd);
         void *Qi = Q[i], *Ki = split ? K[i] : nullptr, *Vi = split ? V[i] : nullptr;
         if (host) {
-            GELO_CUDA_OK(cudaMemcpyAsync(L[0].Hd, H[i], (size_t)n * d * es, cudaMemcpyHostToDevice, st));
-            Hi = L[0].Hd;
+            void* hd = b ? L[0].Hd2 : L[0].Hd;
+            GELO_CUDA_OK(cudaStreamWaitEvent(ctx->copy_in, ctx->h_free[b], 0));
+            GELO_CUDA_OK(cudaMemcpyAsync(hd, H[i], (size_t)n * d * es, cudaMemcpyHostToDevice, ctx->copy_in));
+            GELO_CUDA_OK(cudaEventRecord(ctx->h_ready[b], ctx->copy_in));
+            GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->h_ready[b], 0));
+            Hi = hd;
             Qi = y; Ki = split ? y + third : nullptr; Vi = split ? y + 2 * third : nullptr;
         }
         GELO_TRY(run_shield_rows(ctx, Hi, n, d, k, shield_scale, seeds[i], dtype, L[0].S, L[0].sh, st));
         GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
+        if (host) GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[b], 0));
         GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st));
         GELO_TRY(project_impl(ctx, L[0].U, W[i], m, d, p, dtype, L[0].Yp, st));
         GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, L[0].Yp, n, k, p, dtype, Qi, Ki, Vi, st));
         GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
         if (host) {
+            GELO_CUDA_OK(cudaEventRecord(ctx->h_free[b], st));
+            GELO_CUDA_OK(cudaEventRecord(ctx->y_ready[b], st));
+            GELO_CUDA_OK(cudaStreamWaitEvent(ctx->copy_out, ctx->y_ready[b], 0));
             if (split) {
-                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, third, cudaMemcpyDeviceToHost, st));
-                GELO_CUDA_OK(cudaMemcpyAsync(K[i], y + third, third, cudaMemcpyDeviceToHost, st));
-                GELO_CUDA_OK(cudaMemcpyAsync(V[i], y + 2 * third, third, cudaMemcpyDeviceToHost, st));
+                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, third, cudaMemcpyDeviceToHost, ctx->copy_out));
+                GELO_CUDA_OK(cudaMemcpyAsync(K[i], y + third, third, cudaMemcpyDeviceToHost, ctx->copy_out));
+                GELO_CUDA_OK(cudaMemcpyAsync(V[i], y + 2 * third, third, cudaMemcpyDeviceToHost, ctx->copy_out));
             } else {
-                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, (size_t)n * p * es, cudaMemcpyDeviceToHost, st));
+                GELO_CUDA_OK(cudaMemcpyAsync(Q[i], y, (size_t)n * p * es, cudaMemcpyDeviceToHost, ctx->copy_out));
             }
+            GELO_CUDA_OK(cudaEventRecord(ctx->y_free[b], ctx->copy_out));
         }
         if (i + D < calls) GELO_TRY(enqueue_sample(i + D));
+    }
+    if (host) {
+        GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[0], 0));
+        GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[1], 0));
     }
     ctx->tc_update_ctas = 0;
     ctx->chain_valid = calls >= D && !ctx->prof_on;
@@ -413,6 +439,13 @@ int gelo_create(gelo_ctx** out, int device)
                    cudaEventCreateWithFlags(&ctx->lane_ready[l], cudaEventDisableTiming) == cudaSuccess &&
                    cudaEventCreateWithFlags(&ctx->lane_free[l], cudaEventDisableTiming) == cudaSuccess;
     lanes_ok = lanes_ok && cudaMalloc(&ctx->lane_seed_dev, kMaxLanes * 8 * sizeof(uint64_t)) == cudaSuccess;
+    lanes_ok = lanes_ok && cudaStreamCreateWithFlags(&ctx->copy_in, cudaStreamNonBlocking) == cudaSuccess &&
+               cudaStreamCreateWithFlags(&ctx->copy_out, cudaStreamNonBlocking) == cudaSuccess;
+    for (int b = 0; b < 2 && lanes_ok; ++b)
+        lanes_ok = cudaEventCreateWithFlags(&ctx->h_ready[b], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->h_free[b], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->y_ready[b], cudaEventDisableTiming) == cudaSuccess &&
+                   cudaEventCreateWithFlags(&ctx->y_free[b], cudaEventDisableTiming) == cudaSuccess;
     if (!lanes_ok) { gelo_destroy(ctx); return GELO_ERR_CUDA; }
     cudaDriverEntryPointQueryResult qres;
     void* fn = nullptr;
@@ -433,6 +466,14 @@ int gelo_destroy(gelo_ctx* ctx)
         if (ctx->lane_free[l]) cudaEventDestroy(ctx->lane_free[l]);
     }
     drop_graphs(ctx);
+    if (ctx->copy_in) { cudaStreamSynchronize(ctx->copy_in); cudaStreamDestroy(ctx->copy_in); }
+    if (ctx->copy_out) { cudaStreamSynchronize(ctx->copy_out); cudaStreamDestroy(ctx->copy_out); }
+    for (int b = 0; b < 2; ++b) {
+        if (ctx->h_ready[b]) cudaEventDestroy(ctx->h_ready[b]);
+        if (ctx->h_free[b]) cudaEventDestroy(ctx->h_free[b]);
+        if (ctx->y_ready[b]) cudaEventDestroy(ctx->y_ready[b]);
+        if (ctx->y_free[b]) cudaEventDestroy(ctx->y_free[b]);
+    }
     if (ctx->lane_seed_dev) cudaFree(ctx->lane_seed_dev);
     if (ctx->batch_start) cudaEventDestroy(ctx->batch_start);
     cudaFree(ctx->status_dev);

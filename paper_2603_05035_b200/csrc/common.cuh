@@ -74,6 +74,9 @@ struct gelo_ctx {
     struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3, tc_ctas; cudaGraphExec_t exec; long long launches; };
     std::vector<SampleGraph> graphs;
     uint64_t* lane_seed_dev = nullptr;              // one seed slot per lane
+    // the batched host variant moves activations in and results out on streams of their own, through two staging pairs
+    cudaStream_t copy_in = nullptr, copy_out = nullptr;
+    cudaEvent_t h_ready[2] = {}, h_free[2] = {}, y_ready[2] = {}, y_free[2] = {};
     // optional per-launch timing (gelo_profile_start / gelo_profile_stop)
     bool prof_on = false;
     std::vector<gelo::ProfEntry> prof;
