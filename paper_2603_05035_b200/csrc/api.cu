@@ -142,8 +142,8 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, ldi, L.G, ldi, GELO_F32, L.A32, nullptr, ldi, st));
     const float s = ctx->gamma / sqrtf((float)m);
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G1, attempt, s, L.A32, L.A32, st, seed_dev));
-    GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st));
-    if (dtype != GELO_F32) GELO_TRY(launch_widen(ctx, m, A_out, lda, dtype, L.A32, ldi, st));
+    // the inverse is that of the stored A: round, and carry on from the rounded values
+    GELO_TRY(launch_narrow(ctx, m, L.A32, ldi, dtype, A_out, lda, st, dtype != GELO_F32 ? L.A32 : nullptr, ldi));
     // tensor-core updates serve the bf16 path; the fp32 path stays exact
     const int l3lu = level3_kind(ctx, m, dtype, false);
     if (l3lu) GELO_TRY(run_lu_inverse_tc(ctx, m, L.A32, ldi, L.X32, L.lu, L.tc, l3lu == 3, st));

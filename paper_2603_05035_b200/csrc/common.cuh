@@ -237,10 +237,9 @@ int run_cond_estimate(gelo_ctx*, int m, const void* A, const void* Ainv, int ld,
 // sign_diag (optional, fp32 matrix with stride lds): column j is multiplied by sign(sign_diag[j*lds + j]).
 int launch_finish_mixing(gelo_ctx*, int m, const float* src, int lds_src, const float* sign_diag,
                          int lds_diag, int dtype, void* dst, void* dstT, int ldd, cudaStream_t);
-// dst (fp32, stride ldd) = widen(src (dtype, stride lds)) for an m x m matrix
-int launch_widen(gelo_ctx*, int m, const void* src, int lds, int dtype, float* dst, int ldd, cudaStream_t);
-// dst (dtype) = round(src fp32), m x m
-int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t);
+// dst (dtype) = round(src fp32), m x m; back (optional, fp32, stride ldb, may alias src) = the stored values widened again
+int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t,
+                  float* back = nullptr, int ldb = 0);
 
 // (hi, lo) bf16 pair of an fp32 block, optionally transposed (output is cols x rows then)
 int launch_split(gelo_ctx*, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
@@ -269,7 +268,7 @@ struct TcScratch {
     float* wf32 = nullptr;                 // kMaxKSplit planes of kOuter x ld fp32 (split-K partial products)
     float* w32[2] = {nullptr, nullptr};    // kSuper x ld fp32    block rows W and T W of the tf32 updates
     float* tsuper = nullptr;               // ceil(m / kSuper) merged triangular factors, kSuper x kSuper each
-    float* sx = nullptr;                   // kOuter x kSuper     V_i^T V_(<i) of the block being merged
+    float* sx = nullptr;                   // kOuter x (kSuper + kOuter)   V_i^T [V_(<i) | V_i] of the block being merged
     float* xb = nullptr;                   // kSuper x kOuter     its product with T_i
 };
 TcScratch carve_tc(Arena&, int m, int ld);

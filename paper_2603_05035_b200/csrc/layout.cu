@@ -42,12 +42,49 @@ __global__ void __launch_bounds__(256) finish_mixing_kernel(int m, const float* 
     }
 }
 
-template <typename TS, typename TD>
-__global__ void __launch_bounds__(256) convert_kernel(int m, const TS* __restrict__ src, int lds, TD* __restrict__ dst, int ldd)
+// dst = convert(src) for an m x m matrix, four consecutive columns per thread (rows start 16-byte aligned for the
+// wider of the two types, which every row stride of this library guarantees); `back`, if given, receives the stored
+// values widened again (what a later fp32 computation on the stored matrix must start from).
+__device__ __forceinline__ void load4(const float* p, float (&x)[4])
 {
-    const int c = blockIdx.x * blockDim.x + threadIdx.x;
+    const float4 t = *reinterpret_cast<const float4*>(p);
+    x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+}
+__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&x)[4])
+{
+    const uint2 t = *reinterpret_cast<const uint2*>(p);
+    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xffff0000u);
+    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xffff0000u);
+}
+__device__ __forceinline__ void store4(float* p, const float (&x)[4]) { *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]); }
+__device__ __forceinline__ void store4(__nv_bfloat16* p, float (&x)[4])
+{
+    __nv_bfloat162 a = __floats2bfloat162_rn(x[0], x[1]), b = __floats2bfloat162_rn(x[2], x[3]);
+    uint2 t;
+    t.x = *reinterpret_cast<uint32_t*>(&a); t.y = *reinterpret_cast<uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = t;
+    const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+    x[0] = fa.x; x[1] = fa.y; x[2] = fb.x; x[3] = fb.y;       // the stored values
+}
+
+template <typename TS, typename TD>
+__global__ void __launch_bounds__(256) convert_kernel(int m, const TS* __restrict__ src, int lds, TD* __restrict__ dst, int ldd,
+                                                      float* __restrict__ back, int ldb)
+{
+    const int c4 = (blockIdx.x * blockDim.x + threadIdx.x) * 4;
     const int r = blockIdx.y;
-    if (c < m) put(dst + (size_t)r * ldd + c, get(src + (size_t)r * lds + c));
+    if (c4 >= m) return;
+    if (c4 + 3 < m) {
+        float x[4];
+        load4(src + (size_t)r * lds + c4, x);
+        store4(dst + (size_t)r * ldd + c4, x);
+        if (back) *reinterpret_cast<float4*>(back + (size_t)r * ldb + c4) = make_float4(x[0], x[1], x[2], x[3]);
+    } else {
+        for (int c = c4; c < m; ++c) {
+            put(dst + (size_t)r * ldd + c, get(src + (size_t)r * lds + c));
+            if (back) back[(size_t)r * ldb + c] = get(dst + (size_t)r * ldd + c);
+        }
+    }
 }
 
 // hi = bf16(x), lo = bf16(x - hi) for a rows x cols block (fp32, stride lds) -> bf16 pair (stride ldo);
@@ -211,23 +248,17 @@ int launch_finish_mixing(gelo_ctx* ctx, int m, const float* src, int lds, const 
     return after_launch(ctx);
 }
 
-int launch_widen(gelo_ctx* ctx, int m, const void* src, int lds, int dtype, float* dst, int ldd, cudaStream_t st)
+int launch_narrow(gelo_ctx* ctx, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t st, float* back,
+                  int ldb)
 {
-    dim3 grid(ceil_div(m, 256), m);
+    if ((lds % 4) || (ldd % 4) || (back && (ldb % 4)) || (reinterpret_cast<uintptr_t>(src) & 15u) ||
+        (reinterpret_cast<uintptr_t>(dst) & 15u) || (reinterpret_cast<uintptr_t>(back) & 15u))
+        return GELO_ERR_INVALID;
+    dim3 grid(ceil_div(m, 1024), m);
     if (dtype == GELO_BF16)
-        convert_kernel<__nv_bfloat16, float><<<grid, 256, 0, st>>>(m, static_cast<const __nv_bfloat16*>(src), lds, dst, ldd);
+        convert_kernel<float, __nv_bfloat16><<<grid, 256, 0, st>>>(m, src, lds, static_cast<__nv_bfloat16*>(dst), ldd, back, ldb);
     else
-        convert_kernel<float, float><<<grid, 256, 0, st>>>(m, static_cast<const float*>(src), lds, dst, ldd);
-    return after_launch(ctx);
-}
-
-int launch_narrow(gelo_ctx* ctx, int m, const float* src, int lds, int dtype, void* dst, int ldd, cudaStream_t st)
-{
-    dim3 grid(ceil_div(m, 256), m);
-    if (dtype == GELO_BF16)
-        convert_kernel<float, __nv_bfloat16><<<grid, 256, 0, st>>>(m, src, lds, static_cast<__nv_bfloat16*>(dst), ldd);
-    else
-        convert_kernel<float, float><<<grid, 256, 0, st>>>(m, src, lds, static_cast<float*>(dst), ldd);
+        convert_kernel<float, float><<<grid, 256, 0, st>>>(m, src, lds, static_cast<float*>(dst), ldd, back, ldb);
     return after_launch(ctx);
 }
 

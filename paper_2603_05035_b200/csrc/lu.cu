@@ -485,14 +485,18 @@ __global__ void build_perm_kernel(const int* __restrict__ ipiv, int* __restrict_
     for (int i = threadIdx.x; i < m; i += blockDim.x) perm[i] = sp[i];
 }
 
-__global__ void permuted_identity_kernel(float* __restrict__ X, int ld, int m, const int* __restrict__ perm)
+__global__ void permuted_ones_kernel(float* __restrict__ X, int ld, int m, const int* __restrict__ perm)
 {
-    const size_t total = (size_t)m * ld;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (size_t)gridDim.x * blockDim.x) {
-        const int r = (int)(idx / ld), c = (int)(idx % ld);
-        X[idx] = (c == perm[r]) ? 1.0f : 0.0f;
-    }
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < m) X[(size_t)r * ld + perm[r]] = 1.0f;
+}
+
+// X = P (X[i, perm[i]] = 1): a memset at copy speed, then the ones.
+int set_permutation(gelo_ctx* ctx, float* X, int ld, int m, const int* perm, cudaStream_t st)
+{
+    GELO_CUDA_OK(cudaMemsetAsync(X, 0, (size_t)m * ld * sizeof(float), st));
+    permuted_ones_kernel<<<ceil_div(m, 256), 256, 0, st>>>(X, ld, m, perm);
+    return after_launch(ctx);
 }
 
 }  // namespace
@@ -571,8 +575,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         GELO_CUDA_OK(cudaFuncSetAttribute(build_perm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)perm_smem));
     build_perm_kernel<<<1, 256, perm_smem, st>>>(s.ipiv, s.perm, m);
     GELO_TRY(after_launch(ctx));
-    permuted_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(X, ld, m, s.perm);
-    GELO_TRY(after_launch(ctx));
+    GELO_TRY(set_permutation(ctx, X, ld, m, s.perm, st));
     for (int s0 = 0; s0 < m; s0 += kSuper) {
         const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
         const int send = s0 + sw;
@@ -631,8 +634,7 @@ int run_lu_inverse(gelo_ctx* ctx, int m, const float* A, int ld, float* X, const
         GELO_CUDA_OK(cudaFuncSetAttribute(build_perm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)perm_smem));
     build_perm_kernel<<<1, 256, perm_smem, st>>>(s.ipiv, s.perm, m);
     GELO_TRY(after_launch(ctx));
-    permuted_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(X, ld, m, s.perm);
-    GELO_TRY(after_launch(ctx));
+    GELO_TRY(set_permutation(ctx, X, ld, m, s.perm, st));
     for (int pnl = 0; pnl < npanels; ++pnl) {
         const int i0 = pnl * NB, ib = (m - i0 < NB) ? (m - i0) : NB;
         tri_solve_block_kernel<false><<<ceil_div(m, 256), 256, 0, st>>>(M, ld, X, ld, i0, ib, 0, m);

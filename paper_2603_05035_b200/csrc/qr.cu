@@ -349,14 +349,18 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
     return after_launch(ctx);
 }
 
-__global__ void set_identity_kernel(float* __restrict__ Q, int ld, int m)
+__global__ void set_diagonal_kernel(float* __restrict__ Q, int ld, int m)
 {
-    const size_t total = (size_t)m * ld;
-    for (size_t idx = (size_t)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
-         idx += (size_t)gridDim.x * blockDim.x) {
-        const int r = (int)(idx / ld), c = (int)(idx % ld);
-        Q[idx] = (r == c) ? 1.0f : 0.0f;
-    }
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < m) Q[(size_t)r * ld + r] = 1.0f;
+}
+
+// Q = I: a memset at copy speed, then the ones.
+int set_identity(gelo_ctx* ctx, float* Q, int ld, int m, cudaStream_t st)
+{
+    GELO_CUDA_OK(cudaMemsetAsync(Q, 0, (size_t)m * ld * sizeof(float), st));
+    set_diagonal_kernel<<<ceil_div(m, 256), 256, 0, st>>>(Q, ld, m);
+    return after_launch(ctx);
 }
 
 
@@ -425,12 +429,12 @@ gram128_kernel(const float* __restrict__ V, int ld, int nr, int ob, float* __res
 
 // Triangular factor of an outer block from the factors of its 32-column panels:
 //   (I - V1 T1 V1^T)(I - V2 T2 V2^T) = I - [V1 V2] [[T1, -T1 (V1^T V2) T2], [0, T2]] [V1 V2]^T,
-// applied panel after panel.  part: `slabs` partial Gram matrices (summed here in slab order); T32: the panels'
-// factors.  One CTA, everything in shared memory.
+// applied panel after panel.  part: `slabs` partial Gram matrices of 128 rows with row stride ldp (summed here in
+// slab order); T32: the panels' factors.  One CTA, everything in shared memory.
 constexpr int kMergeSmemBytes = (2 * 128 * 129 + 96 * 33 + 32 * 33) * 4;
 
 __global__ void __launch_bounds__(1024)
-t_merge_kernel(const float* __restrict__ part, int slabs, const float* __restrict__ T32, int ob, float* __restrict__ T128)
+t_merge_kernel(const float* __restrict__ part, int slabs, int ldp, const float* __restrict__ T32, int ob, float* __restrict__ T128)
 {
     extern __shared__ float msm[];
     float (*S)[129] = reinterpret_cast<float (*)[129]>(msm);
@@ -440,7 +444,7 @@ t_merge_kernel(const float* __restrict__ part, int slabs, const float* __restric
     const int tid = threadIdx.x;
     for (int idx = tid; idx < 128 * 128; idx += 1024) {
         float acc = 0.0f;
-        for (int q = 0; q < slabs; ++q) acc += part[(size_t)q * 128 * 128 + idx];
+        for (int q = 0; q < slabs; ++q) acc += part[((size_t)q * 128 + (idx >> 7)) * ldp + (idx & 127)];
         S[idx >> 7][idx & 127] = acc;
         Tm[idx >> 7][idx & 127] = 0.0f;
     }
@@ -512,8 +516,7 @@ int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const Q
         GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, nc, jb, st));
     }
     // ---- accumulate Q backwards from the identity ----
-    set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
-    GELO_TRY(after_launch(ctx));
+    GELO_TRY(set_identity(ctx, Q, ld, m, st));
     for (int pnl = npanels - 1; pnl >= 0; --pnl) {
         const int j0 = pnl * NB, jb = (m - j0 < NB) ? (m - j0) : NB;
         const int nr = m - j0;
@@ -600,14 +603,13 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
         gram128_kernel<<<slabs, 256, 0, st>>>(Vb, ld, m - b0, ob, tc.gram);
         GELO_TRY(after_launch(ctx));
         float* Tb = s.T128 + (size_t)blk * 128 * 128;
-        t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.gram, slabs, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
+        t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.gram, slabs, 128, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
         GELO_TRY(after_launch(ctx));
         const int nc = m - bend;
         if (nc > 0) GELO_TRY(block_apply(b0, ob, R + (size_t)b0 * ld + bend, nc, true));
     }
     // ---- accumulate Q backwards from the identity ----
-    set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
-    GELO_TRY(after_launch(ctx));
+    GELO_TRY(set_identity(ctx, Q, ld, m, st));
     for (int blk = nblocks - 1; blk >= 0; --blk) {
         const int b0 = blk * kOuter;
         const int ob = (m - b0 < kOuter) ? (m - b0) : kOuter;
@@ -632,6 +634,8 @@ int run_householder_qr_tf32(gelo_ctx* ctx, int m, float* R, int ld, float* Q, co
     GELO_CUDA_OK(cudaFuncSetAttribute(t_merge_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, kMergeSmemBytes));
     const float back2 = (1.0f + kTf32TruncLoss) * (1.0f + kTf32TruncLoss);
     const int width = ctx->tc_update_ctas > 0 ? ctx->tc_update_ctas : ctx->sm_count;   // CTAs one launch may use
+    // the Gram slots are read in full by the merge kernel; entries that no product writes must at least be finite
+    GELO_CUDA_OK(cudaMemsetAsync(tc.sx, 0, (size_t)kOuter * (kSuper + kOuter) * sizeof(float), st));
 
     // C (nr x nc, rows from row r0 of the matrix) <- (I - V op(T) V^T) C with V = reflector columns c0 .. c0+kv-1
     // (rows from r0 = c0), T: kv x kv with row stride ldt; planes hold `maxsplit` slices of kv x ld.
@@ -680,31 +684,36 @@ int run_householder_qr_tf32(gelo_ctx* ctx, int m, float* R, int ld, float* Q, co
                     GELO_TRY(launch_rank_update(ctx, Vp, ld, s.W2, ld, C, ld, nr, ncb, jb, st));
                 }
             }
-            // block factor T_i from the Gram matrix of the block's reflectors and the panel factors
+            // S = V_i^T [V_(<i) | V_i]  (ob x (r + ob)): the block's own Gram matrix and its products with the reflectors
+            // already merged, in one tf32 product over the rows from b0 down (both operands reach the tensor core
+            // truncated, hence the scale)
             const float* Vb = s.V + (size_t)b0 * ld + b0;
-            const int slabs = ceil_div(m - b0, kGramRows);
-            gram128_kernel<<<slabs, 256, 0, st>>>(Vb, ld, m - b0, ob, tc.gram);
-            GELO_TRY(after_launch(ctx));
             float* Tb = s.T128 + (size_t)(b0 / kOuter) * 128 * 128;
-            t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.gram, slabs, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
-            GELO_TRY(after_launch(ctx));
-            // ... into the superblock's factor
             const int r = b0 - s0;                           // reflector columns already merged
-            GELO_CUDA_OK(cudaMemcpy2DAsync(Ts + (size_t)r * kSuper + r, (size_t)kSuper * sizeof(float), Tb, 128 * sizeof(float),
-                                           (size_t)ob * sizeof(float), ob, cudaMemcpyDeviceToDevice, st));
-            if (r > 0) {
+            const int ob8 = (ob + 7) & ~7;
+            const int lds = kSuper + kOuter;
+            {
+                // all 128 columns of the block's slot where the row has them (columns past the block are still zero):
+                // the merge kernel reads the whole 128 x 128 Gram slot
                 const int nr = m - b0;
-                const int ob8 = (ob + 7) & ~7;
-                // S = V_i^T V_(<i)  (ob x r); both operands reach the tensor core truncated
-                int want = ceil_div(2 * width, ceil_div(r, 256));
+                const int ns = (r + kOuter <= ld - s0) ? r + kOuter : ld - s0;
+                int want = ceil_div(2 * width, ceil_div(ns, 256));
                 if (want > kMaxKSplit) want = kMaxKSplit;
                 int used = 0;
                 const size_t plane = (size_t)kOuter * ld;
-                GELO_TRY(launch_gemm_tf32(ctx, ob, r, nr, Vb, ld, true, s.V + (size_t)b0 * ld + s0, ld, false, tc.wf32, ld, false,
+                GELO_TRY(launch_gemm_tf32(ctx, ob, ns, nr, Vb, ld, true, s.V + (size_t)b0 * ld + s0, ld, false, tc.wf32, ld, false,
                                           1.0f, want, plane, &used, st));
-                GELO_TRY(launch_sum_planes(ctx, tc.wf32, plane, used, ld, ob, r, back2, tc.sx, kSuper, st));
+                GELO_TRY(launch_sum_planes(ctx, tc.wf32, plane, used, ld, ob, ns, back2, tc.sx, lds, st));
+            }
+            // block factor T_i from its Gram matrix and the panel factors ...
+            t_merge_kernel<<<1, 1024, kMergeSmemBytes, st>>>(tc.sx + r, 1, lds, s.T + (size_t)(b0 / NB) * NB * NB, ob, Tb);
+            GELO_TRY(after_launch(ctx));
+            // ... into the superblock's factor
+            GELO_CUDA_OK(cudaMemcpy2DAsync(Ts + (size_t)r * kSuper + r, (size_t)kSuper * sizeof(float), Tb, 128 * sizeof(float),
+                                           (size_t)ob * sizeof(float), ob, cudaMemcpyDeviceToDevice, st));
+            if (r > 0) {
                 // X = S^T T_i  (r x ob),  then  T[0:r, r:r+ob] = -T[0:r, 0:r] X  (that part of T is still zero)
-                GELO_TRY(launch_gemm_tf32(ctx, r, ob8, ob, tc.sx, kSuper, true, Tb, 128, false, tc.xb, kOuter, true, 1.0f, 1, 0,
+                GELO_TRY(launch_gemm_tf32(ctx, r, ob8, ob, tc.sx, lds, true, Tb, 128, false, tc.xb, kOuter, true, 1.0f, 1, 0,
                                           nullptr, st));
                 GELO_TRY(launch_gemm_tf32(ctx, r, ob, r, Ts, kSuper, false, tc.xb, kOuter, true, Ts + r, kSuper, false, 1.0f, 1, 0,
                                           nullptr, st));
@@ -716,8 +725,7 @@ int run_householder_qr_tf32(gelo_ctx* ctx, int m, float* R, int ld, float* Q, co
         if (m > send) GELO_TRY(apply(s0, sw, Ts, kSuper, R + (size_t)s0 * ld + send, m - send, true, kSuperKSplit));
     }
     // ---- accumulate Q backwards from the identity, one superblock at a time ----
-    set_identity_kernel<<<4 * ctx->sm_count, 256, 0, st>>>(Q, ld, m);
-    GELO_TRY(after_launch(ctx));
+    GELO_TRY(set_identity(ctx, Q, ld, m, st));
     for (int sb = nsuper - 1; sb >= 0; --sb) {
         const int s0 = sb * kSuper;
         const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;

@@ -274,7 +274,7 @@ TcScratch carve_tc(Arena& a, int m, int ld)
     t.wf32 = static_cast<float*>(a.take((size_t)kMaxKSplit * kOuter * ld * 4));
     for (int h = 0; h < 2; ++h) t.w32[h] = static_cast<float*>(a.take((size_t)kSuper * ld * 4));
     t.tsuper = static_cast<float*>(a.take((size_t)ceil_div(m, kSuper) * kSuper * kSuper * 4));
-    t.sx = static_cast<float*>(a.take((size_t)kOuter * kSuper * 4));
+    t.sx = static_cast<float*>(a.take((size_t)kOuter * (kSuper + kOuter) * 4));
     t.xb = static_cast<float*>(a.take((size_t)kSuper * kOuter * 4));
     return t;
 }
