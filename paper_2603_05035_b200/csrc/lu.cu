@@ -99,7 +99,7 @@ lu_panel_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, int* __res
 // (largest magnitude, smallest row on a tie), swap in registers and eliminate without further
 // traffic.  Only a warp's first row can lie above row j, so the other rows run branch-free.
 constexpr int kClusterMax = 8;
-constexpr int kMaxRowsPerThread = 17;
+constexpr int kMaxRowsPerThread = 20;   // rows a thread can hold in registers (64 each at 1024 threads) without heavy spills
 constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kMaxRowsPerThread;
 
 template <int RPT>
@@ -129,7 +129,7 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
     const bool col_ok = lane < jb;
     const unsigned full = 0xffffffffu;
 
-    float x[RPT], xc[RPT];
+    float x[RPT];
 #pragma unroll
     for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
@@ -141,14 +141,17 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
         const int j = j0 + c;
         const int par = c & 1;
         // ---- this warp's candidate (same in every lane); rows ascend with i, strict > keeps the first ----
+        // (column c of a row is fetched from lane c again for the elimination below rather than kept: registers
+        // decide how many rows a thread can hold, and with them how few SMs a panel occupies)
         float bv = -1.0f;
         int bi = -1;
-        xc[0] = __shfl_sync(full, x[0], c);
-        if (gw >= c && j0 + gw < m) { bv = fabsf(xc[0]); bi = 0; }
+        {
+            const float a0 = fabsf(__shfl_sync(full, x[0], c));
+            if (gw >= c && j0 + gw < m) { bv = a0; bi = 0; }
+        }
 #pragma unroll
         for (int i = 1; i < RPT; ++i) {
-            xc[i] = __shfl_sync(full, x[i], c);
-            const float a = fabsf(xc[i]);
+            const float a = fabsf(__shfl_sync(full, x[i], c));
             if (a > bv && j0 + i * stride + gw < m) { bv = a; bi = i; }
         }
         const int br = (bi >= 0) ? j0 + bi * stride + gw : 0x7fffffff;
@@ -215,16 +218,18 @@ lu_panel_cluster_kernel(float* __restrict__ M, int ld, int m, int j0, int jb, in
             if (poff % stride == gw) {                       // this warp holds row pr: it receives old row j
                 const int pi = poff / stride;
                 const float oldj = rowj_buf[par][lane];
-                const float oc = __shfl_sync(full, oldj, c);
 #pragma unroll
-                for (int i = 0; i < RPT; ++i) if (i == pi) { x[i] = oldj; xc[i] = oc; }
+                for (int i = 0; i < RPT; ++i) if (i == pi) x[i] = oldj;
             }
             if (gw == c) x[0] = prow_s[lane];                // rank 0, warp c: row j receives the pivot row
         }
         // ---- eliminate below row j ----
 #pragma unroll
-        for (int i = 1; i < RPT; ++i) x[i] = fmaf(coef, xc[i], (lane == c) ? 0.0f : x[i]);
-        if (gw > c) x[0] = fmaf(coef, xc[0], (lane == c) ? 0.0f : x[0]);
+        for (int i = 1; i < RPT; ++i) x[i] = fmaf(coef, __shfl_sync(full, x[i], c), (lane == c) ? 0.0f : x[i]);
+        {
+            const float xc0 = __shfl_sync(full, x[0], c);
+            if (gw > c) x[0] = fmaf(coef, xc0, (lane == c) ? 0.0f : x[0]);
+        }
     }
 #pragma unroll
     for (int i = 0; i < RPT; ++i) {
@@ -257,8 +262,11 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
         lu_panel_kernel<<<1, kPanelThreads, 0, st>>>(M, ld, m, j0, jb, ipiv, ctx->status_dev);
         return after_launch(ctx);
     }
+    // alone on the GPU: as many SMs as give every thread at least two rows; in a batch with many sampling lanes: as
+    // few SMs as hold the panel (every SM it occupies is one that the other lanes' kernels cannot use)
+    const int rows_per_thread = ctx->tc_update_ctas > 0 ? kMaxRowsPerThread : 2;
     int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
+    while (cs < kClusterMax && cs * kPanelWarps * rows_per_thread < rows) cs *= 2;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
     int* sd = ctx->status_dev;
     ProfScope ps(ctx, PROF_LU_PANEL, 1.0 * rows * (double)jb * jb, st);   // flops of the eliminations
@@ -271,7 +279,8 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     else if (rpt <= 11) e = launch_cluster_lu_panel<11>(cs, st, M, ld, m, j0, jb, ipiv, sd);
     else if (rpt <= 13) e = launch_cluster_lu_panel<13>(cs, st, M, ld, m, j0, jb, ipiv, sd);
     else if (rpt <= 15) e = launch_cluster_lu_panel<15>(cs, st, M, ld, m, j0, jb, ipiv, sd);
-    else e = launch_cluster_lu_panel<17>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else if (rpt <= 17) e = launch_cluster_lu_panel<17>(cs, st, M, ld, m, j0, jb, ipiv, sd);
+    else e = launch_cluster_lu_panel<20>(cs, st, M, ld, m, j0, jb, ipiv, sd);
     if (e != cudaSuccess) return GELO_ERR_CUDA;
     return after_launch(ctx);
 }

@@ -166,8 +166,8 @@ qr_panel_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
 // during the previous column's update, so no separate Gram pass is needed.  All sums run in a
 // fixed order: results are bit-reproducible.
 constexpr int kClusterMax = 8;
-constexpr int kMaxRowsPerThread = 17;                      // 8 CTAs * 32 warps * 17 rows = 4352
-constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kMaxRowsPerThread;
+constexpr int kMaxRowsPerThread = 28;                      // rows a thread can hold in registers (64 each at 1024 threads)
+constexpr int kClusterPanelMaxRows = kClusterMax * kPanelWarps * kMaxRowsPerThread;   // 7168
 
 template <int RPT>
 __global__ void __launch_bounds__(kPanelThreads, 1)
@@ -196,7 +196,7 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
     const bool col_ok = lane < jb;
     const unsigned full = 0xffffffffu;
 
-    float x[RPT], xc[RPT];
+    float x[RPT];
 #pragma unroll
     for (int i = 0; i < RPT; ++i) {
         const int row = j0 + i * stride + gw;
@@ -210,14 +210,12 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
         const int par = c & 1;
         const int csrc = c & 31;
         // ---- lanes >= c: x_c^T x_lane over the rows below the pivot row j = j0 + c ----
+        // (column c of a row is fetched from lane c again in the update below rather than kept: registers decide how
+        // many rows a thread can hold, and with them how few SMs a panel occupies)
         float acc = 0.0f;
 #pragma unroll
-        for (int i = 1; i < RPT; ++i) {
-            xc[i] = __shfl_sync(full, x[i], csrc);
-            acc = fmaf(xc[i], x[i], acc);
-        }
-        xc[0] = __shfl_sync(full, x[0], csrc);
-        if (gw > c) acc = fmaf(xc[0], x[0], acc);          // a warp's first row is below row j only past warp c
+        for (int i = 1; i < RPT; ++i) acc = fmaf(__shfl_sync(full, x[i], csrc), x[i], acc);
+        if (gw > c) acc = fmaf(__shfl_sync(full, x[0], csrc), x[0], acc);   // a warp's first row is below row j only past warp c
         red[warp][lane] = (lane >= c) ? acc : ((lane < c - 1) ? g : 0.0f);
         __syncthreads();
         {
@@ -263,13 +261,15 @@ qr_panel_cluster_kernel(float* __restrict__ R, int ld, int m, int j0, int jb,
         float graw = 0.0f;
 #pragma unroll
         for (int i = 1; i < RPT; ++i) {
-            graw = fmaf(xc[i], x[i], graw);
-            x[i] = fmaf(coef, xc[i], (lane == c) ? 0.0f : x[i]);
+            const float xci = __shfl_sync(full, x[i], csrc);
+            graw = fmaf(xci, x[i], graw);
+            x[i] = fmaf(coef, xci, (lane == c) ? 0.0f : x[i]);
         }
         g = 0.0f;
+        const float xc0 = __shfl_sync(full, x[0], csrc);
         if (gw > c) {
-            graw = fmaf(xc[0], x[0], graw);
-            x[0] = fmaf(coef, xc[0], (lane == c) ? 0.0f : x[0]);
+            graw = fmaf(xc0, x[0], graw);
+            x[0] = fmaf(coef, xc0, (lane == c) ? 0.0f : x[0]);
         } else if (gw == c) {                               // row j itself: v_c(j) = 1
             g = x[0];
             if (lane > c) x[0] -= tw_s[lane];
@@ -331,8 +331,12 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
         qr_panel_kernel<<<1, kPanelThreads, 0, st>>>(R, ld, m, j0, jb, V, T);
         return after_launch(ctx);
     }
+    // Alone on the GPU a panel spreads over as many SMs as give every thread at least two rows (shortest column
+    // step); in a batch with many sampling lanes it packs up to 28 rows per thread and occupies as few SMs as
+    // possible, since every SM it holds is one that the other lanes' kernels cannot use.
+    const int rows_per_thread = ctx->tc_update_ctas > 0 ? kMaxRowsPerThread : 2;
     int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * 2 < rows) cs *= 2;
+    while (cs < kClusterMax && cs * kPanelWarps * rows_per_thread < rows) cs *= 2;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
     ProfScope ps(ctx, PROF_QR_PANEL, 2.0 * rows * (double)jb * jb, st);   // flops of the column dots and updates
     cudaError_t e;
@@ -344,7 +348,10 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
     else if (rpt <= 11) e = launch_cluster_panel<11>(cs, st, R, ld, m, j0, jb, V, T);
     else if (rpt <= 13) e = launch_cluster_panel<13>(cs, st, R, ld, m, j0, jb, V, T);
     else if (rpt <= 15) e = launch_cluster_panel<15>(cs, st, R, ld, m, j0, jb, V, T);
-    else e = launch_cluster_panel<17>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 17) e = launch_cluster_panel<17>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 20) e = launch_cluster_panel<20>(cs, st, R, ld, m, j0, jb, V, T);
+    else if (rpt <= 24) e = launch_cluster_panel<24>(cs, st, R, ld, m, j0, jb, V, T);
+    else e = launch_cluster_panel<28>(cs, st, R, ld, m, j0, jb, V, T);
     if (e != cudaSuccess) return GELO_ERR_CUDA;
     return after_launch(ctx);
 }
