@@ -109,15 +109,27 @@ __global__ void __launch_bounds__(256) cond_step_kernel(CondViews v)
     const T* op = static_cast<const T*>(v.op[z]);
     const float* x = v.xhat + (size_t)z * v.mpad;
     const int groups = (v.m + 7) >> 3;
+    // loads are issued four at a time before anything is consumed: with one CTA's few warps per SM the kernel lives
+    // on memory-level parallelism
     for (int r = r0 + warp; r < r1; r += 8) {
         const T* a = op + (size_t)r * v.ld;
         float s = 0.0f;
-        for (int g = lane; g < groups; g += 32) {
-            float e[8];
-            load8(a + 8 * g, e);
+        for (int g0 = lane; g0 < groups; g0 += 128) {
+            float e[4][8];
 #pragma unroll
-            for (int t = 0; t < 8; ++t)
-                if (8 * g + t < v.m) s = fmaf(e[t], x[8 * g + t], s);
+            for (int u = 0; u < 4; ++u) {
+                const int g = g0 + 32 * u;
+                if (g < groups) load8(a + 8 * g, e[u]);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const int g = g0 + 32 * u;
+                if (g < groups) {
+#pragma unroll
+                    for (int t = 0; t < 8; ++t)
+                        if (8 * g + t < v.m) s = fmaf(e[u][t], x[8 * g + t], s);
+                }
+            }
         }
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
@@ -127,12 +139,19 @@ __global__ void __launch_bounds__(256) cond_step_kernel(CondViews v)
     float* out = v.partial + ((size_t)z * v.slabs + slab) * v.mpad;
     for (int g = threadIdx.x; g < groups; g += 256) {
         float acc[8] = {0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f, 0.f};
-        for (int r = r0; r < r1; ++r) {
-            float e[8];
-            load8(op + (size_t)r * v.ld + 8 * g, e);
-            const float y = ys[r - r0];
+        for (int rb = r0; rb < r1; rb += 4) {
+            float e[4][8];
 #pragma unroll
-            for (int t = 0; t < 8; ++t) acc[t] = fmaf(e[t], y, acc[t]);
+            for (int u = 0; u < 4; ++u)
+                if (rb + u < r1) load8(op + (size_t)(rb + u) * v.ld + 8 * g, e[u]);
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                if (rb + u < r1) {                           // rows ascend: the sum keeps its fixed order
+                    const float y = ys[rb + u - r0];
+#pragma unroll
+                    for (int t = 0; t < 8; ++t) acc[t] = fmaf(e[u][t], y, acc[t]);
+                }
+            }
         }
 #pragma unroll
         for (int t = 0; t < 8; ++t)
