@@ -84,10 +84,14 @@ int gelo_set_workspace(gelo_ctx* ctx, void* dev_ws, size_t bytes);
  * each with the next attempt number in the Philox counter). */
 int gelo_set_nonorthogonal(gelo_ctx* ctx, float gamma, float cond_bound, int max_attempts);
 
-/* How the trailing updates of the blocked QR / LU are computed.  0 (default): split-precision tensor-core
- * products for bf16 calls with m >= 256, fp32 FMA otherwise; 1: always fp32 FMA; 2: always tensor cores.
- * The tensor-core products are good to about 1e-5 relative, which the fp32 path's 1e-4 budget does not leave
- * room for, hence the default. */
+/* How the level-3 updates of the blocked QR / LU are computed.
+ *   0 (default): fp32 FMA kernels for fp32 calls and for m < 256; for bf16 calls with m >= 256 the QR runs single
+ *      tf32 tensor-core products straight from the fp32 matrices (followed, for an orthogonal A, by one
+ *      Newton-Schulz step that squares the orthogonality defect tf32 leaves) and the LU runs three bf16 products of
+ *      operands held as (high, low) pairs;
+ *   1: always fp32 FMA;  2: always the split-precision products;  3: always tf32.
+ * The split-precision products are good to about 1e-5 relative and tf32 to about 1e-3, neither of which the fp32
+ * path's 1e-4 budget leaves room for, hence the default. */
 int gelo_set_level3(gelo_ctx* ctx, int mode);
 
 /* Preferred row stride (elements) of an m x m mixing matrix: m rounded up to 64. */
@@ -138,7 +142,9 @@ int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ai
  * the level-3 update of the blocked QR / LU, on the tensor cores with every operand held as a bf16
  * (high, low) pair and the product accumulated as hi*hi + hi*lo + lo*hi in fp32 (relative error of the
  * product about 1e-5).  ldc must be a multiple of 4 and >= N rounded up to 8; columns N .. that bound are
- * scratch.  Needs workspace for (max(M, N), 0). */
+ * scratch.  Needs workspace for (max(M, N), 0).  With gelo_set_level3(ctx, 3) the same update runs as one tf32
+ * product read straight from A_dev and B_dev (lda and ldb multiples of 4, both 16-byte aligned, no scratch columns);
+ * the tensor core truncates the operands to tf32, so the product comes out 7e-4 short on average. */
 int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int lda, const float* B_dev, int ldb,
                     float* C_dev, int ldc, void* stream);
 
