@@ -272,6 +272,24 @@ int gelo_set_lanes(gelo_ctx* ctx, int lanes);
 int gelo_set_lane_share(gelo_ctx* ctx, int share);
 size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lanes);
 
+/* ---- structured variant: block-diagonal orthogonal mixing -------------------------------------- */
+
+/* The same offload with a block-diagonal orthogonal A (the paper lists "structured orthogonal transforms" as
+ * future work for cheaper A-generation; this is one such structure, NOT the dense mixing of its Section 3.2).
+ * The m = n + k rows are dealt into nb = ceil(m / block) groups (block a multiple of 64, nb <= lanes, n >= nb);
+ * group j holds data rows [n j / nb, n (j+1) / nb) and shield rows [k j / nb, k (j+1) / nb), i.e. every group
+ * mixes its share of the shield rows with its data rows, and gets an independent Haar-orthogonal A_j from a
+ * Householder QR (seed of the call combined with j).  Rows mix only inside their group: an observer of U learns
+ * which group a row belongs to, so this trades part of the hiding for cost: A-generation nb (8/3) block^3 instead
+ * of (8/3) m^3 flops, mixing and unmixing 2 m block (d + p) instead of 2 m^2 (d + p).  The result is H W as
+ * before.  Arguments as gelo_qkv_offload_batch (orthogonal kind only); workspace
+ * gelo_blockdiag_workspace_bytes(..., block, lanes), 0 if the sizes are not supported. */
+size_t gelo_blockdiag_workspace_bytes(int n, int k, int d, int p, int dtype, int block, int lanes);
+int gelo_qkv_offload_blockdiag_batch(gelo_ctx* ctx, int calls, const void* const* H_dev, const void* const* W_dev,
+                                     int n, int k, int d, int p, int block, const uint64_t* seeds,
+                                     float shield_scale, int dtype, void* const* Q_dev, void* const* K_dev,
+                                     void* const* V_dev, void* stream);
+
 /* ---- per-launch timing (measurement aid; no counterpart in the paper) ----------------------- */
 
 /* Between gelo_profile_start and gelo_profile_stop every launch of the main kernel classes is

@@ -57,6 +57,8 @@ EXPORTS = {
     "gelo_qkv_offload": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_blockdiag_workspace_bytes": (ctypes.c_size_t, [_i, _i, _i, _i, _i, _i, _i]),
+    "gelo_qkv_offload_blockdiag_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _i, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch_host_async": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_lanes": (_i, [_vp, _i]),
     "gelo_set_lane_share": (_i, [_vp, _i]),
@@ -296,6 +298,27 @@ class Context:
         """Lists with one entry per call; sampling of different calls runs on concurrent lanes."""
         self._batch(self._lib.gelo_qkv_offload_batch, "gelo_qkv_offload_batch", H, W, n, k, d, p, kinds, seeds,
                     shield_scale, dtype, Q, K, V, stream)
+
+    def ensure_blockdiag_workspace(self, n, k, d, p, dtype, block, lanes=None):
+        """Workspace for the block-diagonal variant."""
+        lanes = int(lanes if lanes is not None else getattr(self, "lanes", 4))
+        need = int(self._lib.gelo_blockdiag_workspace_bytes(n, k, d, p, dtype_code(dtype), block, lanes))
+        if need == 0:
+            raise ValueError("unsupported sizes for the block-diagonal variant")
+        if self._ws is None or self._ws.numel() < need:
+            self.set_workspace(torch.empty(need, dtype=torch.uint8, device=f"cuda:{self.device}"))
+        return need
+
+    def qkv_offload_blockdiag_batch(self, H, W, n, k, d, p, block, seeds, shield_scale, dtype, Q, K=None, V=None, stream=None):
+        """Block-diagonal orthogonal mixing (structured variant); lists with one entry per call."""
+        calls = len(H)
+        if not (len(W) == len(seeds) == len(Q) == calls):
+            raise ValueError("per-call lists must have one entry per call")
+        seeds_a = (ctypes.c_uint64 * calls)(*[int(x) for x in seeds])
+        self._check(self._lib.gelo_qkv_offload_blockdiag_batch(
+            self._h, calls, self._ptr_array(H, calls), self._ptr_array(W, calls), n, k, d, p, block, seeds_a, shield_scale,
+            dtype_code(dtype), self._ptr_array(Q, calls), self._ptr_array(K, calls), self._ptr_array(V, calls),
+            _stream(stream)), "gelo_qkv_offload_blockdiag_batch")
 
     def qkv_offload_batch_host(self, H_host, W, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host=None,
                                V_host=None, stream=None):

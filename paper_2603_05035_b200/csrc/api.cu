@@ -377,6 +377,121 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     return GELO_OK;
 }
 
+// ---- block-diagonal orthogonal mixing (a structured variant; the paper names structured orthogonal transforms as
+//      future work) -------------------------------------------------------------------------------------------------
+//
+// The m = n + k mixed rows are dealt into nb = ceil(m / block) groups; group j takes the data rows
+// [n j / nb, n (j+1) / nb) and the shield rows [k j / nb, k (j+1) / nb), so every group mixes its share of shield rows
+// with its data rows.  Each group gets its own Haar-orthogonal A_j (Householder QR of a Gaussian, sampled on a lane of
+// its own): U_j = A_j [H_j; S_j], one projection for all of U, Y_j = (A_j^T Y'_j)[data rows].  A-generation costs
+// nb (8/3) b^3 instead of (8/3) m^3 and the two mixing products 2 m b (d + p) instead of 2 m^2 (d + p).
+struct BlockPlan {
+    int nb = 0, bmax = 0;
+    int nd[kMaxLanes], ns[kMaxLanes], d0[kMaxLanes], s0[kMaxLanes];
+};
+
+bool plan_blocks(int n, int k, int block, BlockPlan* P)
+{
+    const int m = n + k;
+    if (block <= 0 || (block % 64) != 0) return false;
+    const int nb = (m + block - 1) / block;
+    if (nb < 1 || nb > kMaxLanes || n < nb) return false;
+    P->nb = nb; P->bmax = 0;
+    for (int j = 0; j < nb; ++j) {
+        P->d0[j] = (int)((long long)n * j / nb);
+        P->s0[j] = (int)((long long)k * j / nb);
+        P->nd[j] = (int)((long long)n * (j + 1) / nb) - P->d0[j];
+        P->ns[j] = (int)((long long)k * (j + 1) / nb) - P->s0[j];
+        if (P->nd[j] + P->ns[j] > P->bmax) P->bmax = P->nd[j] + P->ns[j];
+    }
+    return true;
+}
+
+size_t blockdiag_workspace(int n, int k, int d, int p, int dtype, int block, int lanes)
+{
+    BlockPlan P;
+    if (!plan_blocks(n, k, block, &P)) return 0;
+    Arena a;
+    a.cap = ~size_t(0) >> 1;
+    carve(a, P.bmax, 0, 0, 0, dtype, false);                  // lane 0 ...
+    {   // ... which also carries the buffers of the whole call: S, U, Y'
+        const size_t es = elem_size(dtype);
+        a.take((size_t)(k > 0 ? k : 1) * d * es); a.take((size_t)(n + k) * d * es); a.take((size_t)(n + k) * p * es);
+        carve_shield(a, n);
+    }
+    for (int i = 1; i < lanes; ++i) carve(a, P.bmax, 0, 0, 0, dtype, false);
+    return a.off + 256;
+}
+
+int offload_blockdiag_impl(gelo_ctx* ctx, int calls, const void* const* H, const void* const* W, int n, int k, int d, int p,
+                           int block, const uint64_t* seeds, float shield_scale, int dtype, void* const* Q, void* const* K,
+                           void* const* V, cudaStream_t st)
+{
+    BlockPlan P;
+    if (!plan_blocks(n, k, block, &P)) return GELO_ERR_UNSUPPORTED;
+    const int D = ctx->lanes;
+    if (P.nb > D) return GELO_ERR_UNSUPPORTED;                // all groups of a call are alive at once: one lane each
+    if (!ctx->ws) return GELO_ERR_WORKSPACE;
+    const int m = n + k;
+    const size_t es = elem_size(dtype);
+    Arena a;
+    a.base = static_cast<char*>(ctx->ws);
+    a.cap = ctx->ws_bytes;
+    Layout L[kMaxLanes];
+    L[0] = carve(a, P.bmax, 0, 0, 0, dtype, false);
+    char* S = static_cast<char*>(a.take((size_t)(k > 0 ? k : 1) * d * es));
+    char* U = static_cast<char*>(a.take((size_t)m * d * es));
+    char* Yp = static_cast<char*>(a.take((size_t)m * p * es));
+    ShieldScratch sh = carve_shield(a, n);
+    for (int i = 1; i < D; ++i) L[i] = carve(a, P.bmax, 0, 0, 0, dtype, false);
+    if (!a.ok) return GELO_ERR_WORKSPACE;
+    const bool split = K[0] != nullptr;
+    const int qcols = split ? p / 3 : p;
+    ctx->chain_valid = false;                                 // this layout is not the one a later plain batch chains onto
+    ctx->tc_update_ctas = (D >= ctx->lane_tc_share && ctx->lane_tc_share > 1) ? ctx->sm_count / ctx->lane_tc_share : 0;
+    GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
+    for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaStreamWaitEvent(ctx->lane_stream[l], ctx->batch_start, 0));
+
+    const long long total = (long long)calls * P.nb;
+    auto enqueue_sample = [&](long long v) -> int {
+        const int l = (int)(v % D), c = (int)(v / P.nb), j = (int)(v % P.nb);
+        cudaStream_t ls = ctx->lane_stream[l];
+        if (v >= D) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->lane_free[l], 0));
+        const uint64_t seed = seeds[c] ^ (0x9E3779B97F4A7C15ull * (uint64_t)(j + 1));     // a fresh A_j per group and call
+        GELO_TRY(sample_on_lane(ctx, L[l], l, P.nd[j] + P.ns[j], GELO_ORTHOGONAL, seed, dtype, ls));
+        GELO_CUDA_OK(cudaEventRecord(ctx->lane_ready[l], ls));
+        return GELO_OK;
+    };
+    for (long long v = 0; v < total && v < D; ++v) GELO_TRY(enqueue_sample(v));
+    for (int c = 0; c < calls; ++c) {
+        const char* Hc = static_cast<const char*>(H[c]);
+        GELO_TRY(run_shield_rows(ctx, Hc, n, d, k, shield_scale, seeds[c], dtype, S, sh, st));
+        for (int j = 0; j < P.nb; ++j) {
+            const int l = (int)(((long long)c * P.nb + j) % D);
+            const int u0 = P.d0[j] + P.s0[j];
+            GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
+            GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hc + (size_t)P.d0[j] * d * es, P.ns[j] ? S + (size_t)P.s0[j] * d * es : nullptr,
+                              P.nd[j], P.ns[j], d, dtype, U + (size_t)u0 * d * es, st));
+        }
+        GELO_TRY(project_impl(ctx, U, W[c], m, d, p, dtype, Yp, st));
+        for (int j = 0; j < P.nb; ++j) {
+            const int l = (int)(((long long)c * P.nb + j) % D);
+            const int u0 = P.d0[j] + P.s0[j];
+            const size_t qoff = (size_t)P.d0[j] * qcols * es;
+            GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, Yp + (size_t)u0 * p * es, P.nd[j], P.ns[j], p, dtype,
+                                static_cast<char*>(Q[c]) + qoff, split ? static_cast<char*>(K[c]) + qoff : nullptr,
+                                split ? static_cast<char*>(V[c]) + qoff : nullptr, st));
+            GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
+        }
+        for (int j = 0; j < P.nb; ++j) {
+            const long long v = (long long)c * P.nb + j + D;
+            if (v < total) GELO_TRY(enqueue_sample(v));
+        }
+    }
+    ctx->tc_update_ctas = 0;
+    return GELO_OK;
+}
+
 int check_batch_args(gelo_ctx* ctx, int calls, const void* const* H, const void* const* W, int n, int k, int d, int p,
                      const int* kinds, const uint64_t* seeds, int dtype, void* const* Q, void* const* K,
                      void* const* V, bool host)
@@ -783,6 +898,32 @@ int gelo_qkv_offload_batch_host_async(gelo_ctx* ctx, int calls, const void* cons
     DeviceGuard guard(ctx->device);
     return offload_batch_impl(ctx, calls, H_host, W_dev, n, k, d, p, kinds, seeds, shield_scale, dtype, Q_host, K_host,
                               V_host, as_stream(stream), true, false);
+}
+
+size_t gelo_blockdiag_workspace_bytes(int n, int k, int d, int p, int dtype, int block, int lanes)
+{
+    if (n <= 0 || k < 0 || d <= 0 || p <= 0 || bad_dtype(dtype) || lanes < 1 || lanes > kMaxLanes) return 0;
+    return blockdiag_workspace(n, k, d, p, dtype, block, lanes);
+}
+
+int gelo_qkv_offload_blockdiag_batch(gelo_ctx* ctx, int calls, const void* const* H_dev, const void* const* W_dev, int n,
+                                     int k, int d, int p, int block, const uint64_t* seeds, float shield_scale, int dtype,
+                                     void* const* Q_dev, void* const* K_dev, void* const* V_dev, void* stream)
+{
+    if (!ctx || calls < 0 || n <= 0 || k < 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype))
+        return GELO_ERR_INVALID;
+    if (calls == 0) return GELO_OK;
+    if (!H_dev || !W_dev || !seeds || !Q_dev || !K_dev || !V_dev) return GELO_ERR_INVALID;
+    const bool split = K_dev[0] != nullptr;
+    for (int i = 0; i < calls; ++i) {
+        if (!H_dev[i] || !W_dev[i] || misaligned(H_dev[i]) || misaligned(W_dev[i]) || misaligned(Q_dev[i]) ||
+            misaligned(K_dev[i]) || misaligned(V_dev[i]) || (K_dev[i] != nullptr) != split)
+            return GELO_ERR_INVALID;
+        GELO_TRY(check_split(p, Q_dev[i], K_dev[i], V_dev[i]));
+    }
+    DeviceGuard guard(ctx->device);
+    return offload_blockdiag_impl(ctx, calls, H_dev, W_dev, n, k, d, p, block, seeds, shield_scale, dtype, Q_dev, K_dev,
+                                  V_dev, as_stream(stream));
 }
 
 int gelo_profile_start(gelo_ctx* ctx)

@@ -574,6 +574,53 @@ def test_output_projection_unsplit(ctx, oracle, dt, kind):
     assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL[dt]
 
 
+# ------------------------------------------------------------------------- block-diagonal variant
+
+@pytest.mark.parametrize("dt,n,k,d,block,split", [("bf16", 1024, 52, 512, 256, True), ("f32", 300, 20, 256, 128, True),
+                                                   ("bf16", 700, 0, 512, 192, False), ("bf16", 4096, 204, 4096, 512, True)])
+def test_block_diagonal_variant(oracle, dt, n, k, d, block, split):
+    """Block-diagonal orthogonal A: every group mixes its share of shield rows with its data rows, and the result
+    is H W whatever the grouping (Eq. 4 holds for any invertible A)."""
+    p = 3 * d if split else d
+    calls = 3
+    c = binding.Context(0)
+    c.set_lanes(16)
+    c.ensure_blockdiag_workspace(n, k, d, p, dt, block, 16)
+    Hs = [inputs.make_hidden(n, d, dt, 60 + i, True, "cuda") for i in range(calls)]
+    Ws = [inputs.make_weight(d, p, dt, 60 + i, "cuda") for i in range(calls)]
+    mk = lambda cols: [torch.full((n, cols), float("nan"), device="cuda", dtype=TDT[dt]) for _ in range(calls)]
+    if split:
+        Q, K, V = mk(p // 3), mk(p // 3), mk(p // 3)
+        c.qkv_offload_blockdiag_batch(Hs, Ws, n, k, d, p, block, [500 + i for i in range(calls)], 10.0, dt, Q, K, V)
+    else:
+        Q = mk(p)
+        c.qkv_offload_blockdiag_batch(Hs, Ws, n, k, d, p, block, [500 + i for i in range(calls)], 10.0, dt, Q)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    for i in range(calls):
+        y = np.hstack([f64(Q[i]), f64(K[i]), f64(V[i])]) if split else f64(Q[i])
+        if n * d * p < 2e9:
+            assert oracle.rel_fro(y, oracle.direct(f64(Hs[i]), f64(Ws[i]))) <= TOL[dt]
+        else:
+            rows = sample_rows(n, 48, seed=i, extra=[n * j // 9 + e for j in range(1, 9) for e in (-1, 0)])
+            assert oracle.rel_fro(y[rows], oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)) <= TOL[dt]
+    # a different seed draws different A_j and still lands on the same product
+    Q2, K2, V2 = mk(p // 3 if split else p), mk(p // 3), mk(p // 3)
+    if split:
+        c.qkv_offload_blockdiag_batch(Hs[:1], Ws[:1], n, k, d, p, block, [99], 10.0, dt, Q2[:1], K2[:1], V2[:1])
+    else:
+        c.qkv_offload_blockdiag_batch(Hs[:1], Ws[:1], n, k, d, p, block, [99], 10.0, dt, Q2[:1])
+    torch.cuda.synchronize()
+    assert oracle.rel_fro(f64(Q2[0]), f64(Q[0])) <= 2 * TOL[dt]
+    if dt == "bf16":
+        assert not torch.equal(Q2[0], Q[0])                   # rounding differs with A: the mixing really changed
+    # unsupported groupings are refused before any launch
+    L = binding.load_library()
+    assert L.gelo_blockdiag_workspace_bytes(n, k, d, p, binding.dtype_code(dt), 100, 16) == 0       # not a multiple of 64
+    assert L.gelo_blockdiag_workspace_bytes(4096, 0, d, p, binding.dtype_code(dt), 64, 16) == 0     # 64 groups > 32 lanes
+    c.close()
+
+
 def test_batch_of_zero_calls_and_bad_batches():
     c = binding.Context(0)
     c.ensure_batch_workspace(64, 0, 64, 192, "f32", 2)
