@@ -337,6 +337,30 @@ def run_ours(args):
                          "unit": "TFLOP/s" if st_["unit"] == "flops" else "GB/s"}
     dominant = max(kernels, key=lambda k_: kernels[k_]["ms"])
 
+    # ---- structured variant (reported beside the method, never as the method): block-diagonal orthogonal A ----
+    variants = {}
+    if not args.no_variants:
+        for block in (512, 1024):
+            ctx.ensure_blockdiag_workspace(n, k, d, p, w.dtype, block, args.lanes)
+            def vsweep(step):
+                ctx.qkv_offload_blockdiag_batch(Hs, Ws, n, k, d, p, block, [s_ + 300000 + 1000 * step for s_ in seeds],
+                                                w.shield_scale, w.dtype, [Q] * calls, [K] * calls, [V] * calls)
+            for i in range(3):
+                vsweep(-1 - i)
+            torch.cuda.synchronize()
+            a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
+            a.record()
+            for s_i in range(args.steps):
+                vsweep(s_i)
+            b.record()
+            torch.cuda.synchronize()
+            vms = a.elapsed_time(b) / args.steps
+            variants[f"block_{block}"] = {"ms_per_step": vms, "value": float(n) * calls / (vms * 1e-3), "unit": UNIT,
+                                          "groups": -(-m // block),
+                                          "note": "rows mix inside groups of about `block` rows only (weaker hiding than the dense A of the method)"}
+        if ctx.last_status() != gelo.OK:
+            raise SystemExit("device-side error in the variant runs")
+
     if rank == 0:
         es = 2 if w.dtype == "bf16" else 4
         dk = kernels[dominant]
@@ -394,6 +418,8 @@ def run_ours(args):
                       "frac_of_peak": chain_flops / (chain_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
             "checksum": float(checksum),
         }
+        if variants:
+            line["variants_block_diagonal_A"] = variants
         if world == 1 and not args.no_cpu_baseline:
             import oracle
             oracle.build()
@@ -514,6 +540,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-variants", action="store_true", help="skip the block-diagonal variant runs")
     ap.add_argument("--lanes", type=int, default=32, help="concurrent sampling lanes of the batched call (1..32)")
     ap.add_argument("--lane-share", type=int, default=4, help="each level-3 update uses 1/share of the SMs in batches")
     ap.add_argument("--level3", type=int, default=0, choices=[0, 1, 2, 3],
