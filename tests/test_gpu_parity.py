@@ -621,6 +621,21 @@ def test_block_diagonal_variant(oracle, dt, n, k, d, block, split):
     c.close()
 
 
+@pytest.mark.parametrize("d,p", [(512, 1376), (1376, 512)])
+def test_mlp_shaped_projections(ctx, oracle, d, p):
+    """The same procedure on MLP-shaped weights (up: d -> 2.6875 d, down: back), one unsplit result, widths that are
+    not multiples of the 256-column tiles."""
+    n, k = 320, 16
+    ctx.ensure_workspace(n, k, d, p, "bf16")
+    H = inputs.make_hidden(n, d, "bf16", 43, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 43, "cuda")
+    for kind in (ORTHOGONAL, NONORTHOGONAL):
+        Y = torch.full((n, p), float("nan"), device="cuda", dtype=torch.bfloat16)
+        ctx.qkv_offload(H, W, n, k, d, p, kind, 4343, 10.0, "bf16", Y)
+        torch.cuda.synchronize()
+        assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL["bf16"]
+
+
 def test_batch_of_zero_calls_and_bad_batches():
     c = binding.Context(0)
     c.ensure_batch_workspace(64, 0, 64, 192, "f32", 2)
