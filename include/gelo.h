@@ -24,7 +24,8 @@
  *     asynchronous).  The library never frees or keeps caller memory.
  *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Work is
  *     enqueued on it; calls return without waiting unless stated otherwise.
- *   - Element type: GELO_F32 stores float, GELO_BF16 stores bfloat16; products always
+ *   - Element type: GELO_F32 stores float, GELO_BF16 stores bfloat16, GELO_F16 stores IEEE half (the 16-bit
+ *     types share every code path; half keeps 11 significant bits instead of 8); products always
  *     accumulate in fp32.
  *   - A and A^-1 are m x m with a row stride `lda` (in elements) that is a multiple of
  *     8 and >= m; gelo_mixing_ld(m) returns the stride the library prefers.  Columns
@@ -55,7 +56,7 @@ typedef enum {
 } gelo_status;
 
 typedef enum { GELO_ORTHOGONAL = 0, GELO_NONORTHOGONAL = 1 } gelo_kind;
-typedef enum { GELO_F32 = 0, GELO_BF16 = 1 } gelo_dtype;
+typedef enum { GELO_F32 = 0, GELO_BF16 = 1, GELO_F16 = 2 } gelo_dtype;
 
 /* Philox stream ids used by the library (third counter word). */
 enum { GELO_STREAM_G0 = 0, GELO_STREAM_G1 = 1, GELO_STREAM_SHIELD = 2, GELO_STREAM_POWER = 3 };

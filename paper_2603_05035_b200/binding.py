@@ -18,12 +18,12 @@ _lib = None
 
 OK, ERR_INVALID, ERR_WORKSPACE, ERR_COND, ERR_TIMEOUT, ERR_CUDA, ERR_UNSUPPORTED = range(7)
 ORTHOGONAL, NONORTHOGONAL = 0, 1
-F32, BF16 = 0, 1
+F32, BF16, F16 = 0, 1, 2
 STREAM_G0, STREAM_G1, STREAM_SHIELD, STREAM_POWER = 0, 1, 2, 3
 
 __all__ = [
     "OK", "ERR_INVALID", "ERR_WORKSPACE", "ERR_COND", "ERR_TIMEOUT", "ERR_CUDA", "ERR_UNSUPPORTED",
-    "ORTHOGONAL", "NONORTHOGONAL", "F32", "BF16", "GeloError", "Context", "load_library", "library_path",
+    "ORTHOGONAL", "NONORTHOGONAL", "F32", "BF16", "F16", "GeloError", "Context", "load_library", "library_path",
     "dtype_code", "EXPORTS",
 ]
 
@@ -104,6 +104,8 @@ def dtype_code(dtype) -> int:
         return F32
     if dtype in (BF16, "bf16", torch.bfloat16):
         return BF16
+    if dtype in ("f16", torch.float16) or (dtype == F16 and not isinstance(dtype, (str, torch.dtype))):
+        return F16
     raise ValueError(f"unsupported dtype {dtype!r}")
 
 

@@ -23,7 +23,7 @@ inline int level3_kind(const gelo_ctx* ctx, int m, int dtype, bool qr)
 {
     if (ctx->level3 == 1) return 0;
     if (ctx->level3 == 2 || ctx->level3 == 3) return m > gelo::kPanel ? ctx->level3 : 0;
-    if (dtype != GELO_BF16 || m < kTcMinRows) return 0;
+    if (dtype == GELO_F32 || m < kTcMinRows) return 0;
     return qr ? 3 : 2;
 }
 
@@ -94,7 +94,7 @@ bool carve_ctx(gelo_ctx* ctx, int n, int k, int d, int p, int dtype, bool host_s
     return a.ok;
 }
 
-bool bad_dtype(int t) { return t != GELO_F32 && t != GELO_BF16; }
+bool bad_dtype(int t) { return t != GELO_F32 && t != GELO_BF16 && t != GELO_F16; }
 bool bad_ld(int lda, int m) { return lda < m || (lda % 8) != 0; }
 bool misaligned(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) != 0; }
 
@@ -112,7 +112,7 @@ __global__ void set_scalar_kernel(float* p, float v) { *p = v; }
 
 int gemm_dispatch(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
 {
-    if (g.dtype == GELO_BF16 && gemm_tc_supports(g)) return launch_gemm_tc(ctx, g, st);
+    if (g.dtype != GELO_F32 && gemm_tc_supports(g)) return launch_gemm_tc(ctx, g, st);
     return launch_gemm_simt(ctx, g, st);
 }
 

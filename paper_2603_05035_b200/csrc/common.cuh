@@ -3,6 +3,7 @@
 #pragma once
 
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 #include <cuda_runtime.h>
 #include <stddef.h>
 #include <stdint.h>
@@ -117,7 +118,7 @@ struct ProfScope {
 };
 
 static inline int ceil_div(int a, int b) { return (a + b - 1) / b; }
-static inline size_t elem_size(int dtype) { return dtype == GELO_BF16 ? 2 : 4; }
+static inline size_t elem_size(int dtype) { return dtype == GELO_F32 ? 4 : 2; }
 
 // ---- sampling ---------------------------------------------------------------------
 

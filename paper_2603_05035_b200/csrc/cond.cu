@@ -95,6 +95,17 @@ __device__ __forceinline__ void load8(const __nv_bfloat16* p, float (&a)[8])
     }
 }
 
+__device__ __forceinline__ void load8(const __half* p, float (&a)[8])
+{
+    const uint4 raw = *reinterpret_cast<const uint4*>(p);
+    const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+    for (int t = 0; t < 4; ++t) {
+        const float2 f = __half22float2(h[t]);
+        a[2 * t] = f.x; a[2 * t + 1] = f.y;
+    }
+}
+
 // One power-iteration step Op^T (Op xhat) in a single pass over the operator: CTA (slab, z) first forms y_r =
 // Op[r, :] . xhat for its rows (one warp per row), then accumulates sum_r y_r Op[r, :] for every column; the
 // second read of the slab comes from L2.  partial[z][slab][:] receives the slab's contribution.
@@ -191,6 +202,7 @@ int run_cond_estimate(gelo_ctx* ctx, int m, const void* A, const void* Ainv, int
     for (int it = 0; it < kPowerIters; ++it) {
         dim3 g(v.slabs, 2);
         if (dtype == GELO_BF16) cond_step_kernel<__nv_bfloat16><<<g, 256, ys_bytes, st>>>(v);
+        else if (dtype == GELO_F16) cond_step_kernel<__half><<<g, 256, ys_bytes, st>>>(v);
         else cond_step_kernel<float><<<g, 256, ys_bytes, st>>>(v);
         GELO_TRY(after_launch(ctx));
         cond_normalise_kernel<<<2, 1024, 0, st>>>(v);

@@ -23,6 +23,9 @@ struct GemmParams {
 
 __device__ __forceinline__ float ldf(const float* p) { return __ldg(p); }
 __device__ __forceinline__ float ldf(const __nv_bfloat16* p) { return __bfloat162float(*p); }
+__device__ __forceinline__ float ldf(const __half* p) { return __half2float(*p); }
+__device__ __forceinline__ float ldc(const __half* p) { return __half2float(*p); }
+__device__ __forceinline__ void stf(__half* p, float v) { *p = __float2half_rn(v); }
 __device__ __forceinline__ float ldc(const float* p) { return *p; }
 __device__ __forceinline__ float ldc(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 __device__ __forceinline__ void stf(float* p, float v) { *p = v; }
@@ -173,6 +176,9 @@ int launch_gemm_simt(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
     if (g.dtype == GELO_BF16) {
         if (g.transA || g.transB) return GELO_ERR_UNSUPPORTED;
         launch_tiles<__nv_bfloat16, false, false>(p, small, st);
+    } else if (g.dtype == GELO_F16) {
+        if (g.transA || g.transB) return GELO_ERR_UNSUPPORTED;
+        launch_tiles<__half, false, false>(p, small, st);
     } else {
         if (!g.transA && !g.transB) launch_tiles<float, false, false>(p, small, st);
         else if (g.transA && !g.transB) launch_tiles<float, true, false>(p, small, st);

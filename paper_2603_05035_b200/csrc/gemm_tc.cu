@@ -58,6 +58,8 @@ struct TcParams {
     float out_scale;                // TC_STORE_F32 with round_tf32: factor applied before the rounding
     float diag_sub;                 // TC_STORE_F32 with round_tf32: subtracted from the scaled diagonal entries
     float post_scale;               //   ... and the factor applied after that: out = post_scale * (out_scale * acc - diag_sub [row == col])
+    int out_f16;                    // TC_STORE_BF16: operands and output are IEEE half instead of bfloat16
+    uint32_t idesc;                 // instruction descriptor (filled in by the launcher)
     int* status;
 };
 
@@ -206,6 +208,11 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t a, uint32_t b)
     __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
     return *reinterpret_cast<uint32_t*>(&h);
 }
+__device__ __forceinline__ uint32_t pack_f16(uint32_t a, uint32_t b)
+{
+    __half2 h = __floats2half2_rn(__uint_as_float(a), __uint_as_float(b));
+    return *reinterpret_cast<uint32_t*>(&h);
+}
 __device__ __forceinline__ uint32_t pack_bf16f(float a, float b)
 {
     __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
@@ -233,8 +240,13 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
         void* base = chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2);
         const size_t off = (size_t)gm * prm.ldc + (gn - chunk * prm.csplit);
         uint4 pk;
-        pk.x = pack_bf16(v[0], v[1]); pk.y = pack_bf16(v[2], v[3]);
-        pk.z = pack_bf16(v[4], v[5]); pk.w = pack_bf16(v[6], v[7]);
+        if (prm.out_f16) {
+            pk.x = pack_f16(v[0], v[1]); pk.y = pack_f16(v[2], v[3]);
+            pk.z = pack_f16(v[4], v[5]); pk.w = pack_f16(v[6], v[7]);
+        } else {
+            pk.x = pack_bf16(v[0], v[1]); pk.y = pack_bf16(v[2], v[3]);
+            pk.z = pack_bf16(v[4], v[5]); pk.w = pack_bf16(v[6], v[7]);
+        }
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
     } else if (prm.mode == TC_STORE_F32) {
         float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)slice * prm.plane + (size_t)gm * prm.ldc + gn);
@@ -378,8 +390,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                                                  : smem_desc(sa + ks * 32, 16, 1024);
                         // B: N-major, 128-byte-wide boxes kBoxBytes apart, k-row atoms kMnSbo bytes apart
                         const uint64_t db = smem_desc(sb + ks * Cfg::kMnStep, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout);
-                        if (kTf32) tc_mma_tf32(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
-                        else tc_mma_bf16(tmem_d, da, db, Cfg::kInstrDesc, (kb | ks) != 0 ? 1u : 0u);
+                        if (kTf32) tc_mma_tf32(tmem_d, da, db, prm.idesc, (kb | ks) != 0 ? 1u : 0u);
+                        else tc_mma_bf16(tmem_d, da, db, prm.idesc, (kb | ks) != 0 ? 1u : 0u);
                     }
                     tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
                 }
@@ -485,6 +497,7 @@ bool make_map(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols, u
     const cuuint64_t strides[1] = { ld * 2 };
     const cuuint32_t box[2] = { box_cols, box_rows };
     const cuuint32_t estr[2] = { 1, 1 };
+    // (the copy engine only needs the element size and a zero fill: the same map serves IEEE half data)
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(ptr), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
@@ -507,9 +520,12 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
     const int tiles = ceil_div(p.M, BM) * ceil_div(p.N, BN) * p.ksplit;
     int grid = tiles < ctx->sm_count ? tiles : ctx->sm_count;
     if (p.mode != TC_STORE_BF16 && ctx->tc_update_ctas > 0 && grid > ctx->tc_update_ctas) grid = ctx->tc_update_ctas;
+    TcParams q = p;
+    // both operands of a kind::f16 instruction have the same 16-bit format: 1 = bfloat16, 0 = IEEE half
+    q.idesc = (!kTf32 && p.out_f16) ? (Cfg::kInstrDesc & ~((7u << 7) | (7u << 10))) : Cfg::kInstrDesc;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
-        gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, p);
+        gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, q);
     }
     return after_launch(ctx);
 }
@@ -535,7 +551,7 @@ bool make_map_f32_box(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t
 
 bool gemm_tc_supports(const GemmArgs& g)
 {
-    if (g.dtype != GELO_BF16 || g.transA || g.transB || g.alpha != 1.0f || g.beta != 0.0f) return false;
+    if (g.dtype == GELO_F32 || g.transA || g.transB || g.alpha != 1.0f || g.beta != 0.0f) return false;
     if (g.M <= 0 || g.N <= 0 || g.K <= 0) return false;
     if ((g.lda % 8) || (g.ldb % 8) || (g.ldc % 8) || (g.N % 8)) return false;
     if (g.nsplit < 1 || g.nsplit > 3 || g.N % g.nsplit || ((g.N / g.nsplit) % 8)) return false;
@@ -573,6 +589,7 @@ int launch_gemm_tc(gelo_ctx* ctx, const GemmArgs& g, cudaStream_t st)
     }
     p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
     p.mode = TC_STORE_BF16;
+    p.out_f16 = g.dtype == GELO_F16 ? 1 : 0;
     p.C0 = g.C[0]; p.C1 = g.C[g.nsplit > 1 ? 1 : 0]; p.C2 = g.C[g.nsplit > 2 ? 2 : 0];
     p.ldc = g.ldc; p.csplit = g.N / g.nsplit; p.lde = 0;
     p.status = ctx->status_dev;

@@ -9,6 +9,8 @@ namespace {
 
 __device__ __forceinline__ void put(float* p, float v) { *p = v; }
 __device__ __forceinline__ void put(__nv_bfloat16* p, float v) { *p = __float2bfloat16_rn(v); }
+__device__ __forceinline__ void put(__half* p, float v) { *p = __float2half_rn(v); }
+__device__ __forceinline__ float get(const __half* p) { return __half2float(*p); }
 __device__ __forceinline__ float get(const float* p) { return *p; }
 __device__ __forceinline__ float get(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
@@ -64,6 +66,16 @@ __device__ __forceinline__ void store4(__nv_bfloat16* p, float (&x)[4])
     t.x = *reinterpret_cast<uint32_t*>(&a); t.y = *reinterpret_cast<uint32_t*>(&b);
     *reinterpret_cast<uint2*>(p) = t;
     const float2 fa = __bfloat1622float2(a), fb = __bfloat1622float2(b);
+    x[0] = fa.x; x[1] = fa.y; x[2] = fb.x; x[3] = fb.y;       // the stored values
+}
+
+__device__ __forceinline__ void store4(__half* p, float (&x)[4])
+{
+    __half2 a = __floats2half2_rn(x[0], x[1]), b = __floats2half2_rn(x[2], x[3]);
+    uint2 t;
+    t.x = *reinterpret_cast<uint32_t*>(&a); t.y = *reinterpret_cast<uint32_t*>(&b);
+    *reinterpret_cast<uint2*>(p) = t;
+    const float2 fa = __half22float2(a), fb = __half22float2(b);
     x[0] = fa.x; x[1] = fa.y; x[2] = fb.x; x[3] = fb.y;       // the stored values
 }
 
@@ -242,6 +254,9 @@ int launch_finish_mixing(gelo_ctx* ctx, int m, const float* src, int lds, const 
     if (dtype == GELO_BF16)
         finish_mixing_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(m, src, lds, sign_diag, ldg,
             static_cast<__nv_bfloat16*>(dst), static_cast<__nv_bfloat16*>(dstT), ldd);
+    else if (dtype == GELO_F16)
+        finish_mixing_kernel<__half><<<grid, 256, 0, st>>>(m, src, lds, sign_diag, ldg,
+            static_cast<__half*>(dst), static_cast<__half*>(dstT), ldd);
     else
         finish_mixing_kernel<float><<<grid, 256, 0, st>>>(m, src, lds, sign_diag, ldg,
             static_cast<float*>(dst), static_cast<float*>(dstT), ldd);
@@ -257,6 +272,8 @@ int launch_narrow(gelo_ctx* ctx, int m, const float* src, int lds, int dtype, vo
     dim3 grid(ceil_div(m, 1024), m);
     if (dtype == GELO_BF16)
         convert_kernel<float, __nv_bfloat16><<<grid, 256, 0, st>>>(m, src, lds, static_cast<__nv_bfloat16*>(dst), ldd, back, ldb);
+    else if (dtype == GELO_F16)
+        convert_kernel<float, __half><<<grid, 256, 0, st>>>(m, src, lds, static_cast<__half*>(dst), ldd, back, ldb);
     else
         convert_kernel<float, float><<<grid, 256, 0, st>>>(m, src, lds, static_cast<float*>(dst), ldd, back, ldb);
     return after_launch(ctx);

@@ -23,6 +23,22 @@ __device__ __forceinline__ float sumsq8(const uint4& q)
     return s;
 }
 
+__device__ __forceinline__ float sumsq8h(const uint4& q)
+{
+    const __half2* h = reinterpret_cast<const __half2*>(&q);
+    float s = 0.0f;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h[i]);
+        s = fmaf(f.x, f.x, s);
+        s = fmaf(f.y, f.y, s);
+    }
+    return s;
+}
+
+template <typename T> struct is_half_t { static constexpr bool value = false; };
+template <> struct is_half_t<__half> { static constexpr bool value = true; };
+
 template <typename T>
 __global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, int n, int d, float* __restrict__ norms)
 {
@@ -39,7 +55,7 @@ __global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, 
         }
     } else {
         const uint4* h8 = reinterpret_cast<const uint4*>(h);
-        for (int j = lane; j < d / 8; j += 32) s += sumsq8(__ldg(h8 + j));
+        for (int j = lane; j < d / 8; j += 32) s += is_half_t<T>::value ? sumsq8h(__ldg(h8 + j)) : sumsq8(__ldg(h8 + j));
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
@@ -83,6 +99,13 @@ __global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int
     gaussian_block(seed, q, GELO_STREAM_SHIELD, 0u, z);
     if (sizeof(T) == 4) {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(S) + e0) = make_float4(f * z[0], f * z[1], f * z[2], f * z[3]);
+    } else if (is_half_t<T>::value) {
+        __half2 lo = __floats2half2_rn(f * z[0], f * z[1]);
+        __half2 hi = __floats2half2_rn(f * z[2], f * z[3]);
+        uint2 pk;
+        pk.x = *reinterpret_cast<uint32_t*>(&lo);
+        pk.y = *reinterpret_cast<uint32_t*>(&hi);
+        *reinterpret_cast<uint2*>(reinterpret_cast<__half*>(S) + e0) = pk;
     } else {
         __nv_bfloat162 lo = __floats2bfloat162_rn(f * z[0], f * z[1]);
         __nv_bfloat162 hi = __floats2bfloat162_rn(f * z[2], f * z[3]);
@@ -109,6 +132,8 @@ int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float sca
     if (k <= 0) return GELO_OK;
     if (dtype == GELO_BF16)
         row_norm_kernel<__nv_bfloat16><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(H), n, d, s.norms);
+    else if (dtype == GELO_F16)
+        row_norm_kernel<__half><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const __half*>(H), n, d, s.norms);
     else
         row_norm_kernel<float><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const float*>(H), n, d, s.norms);
     GELO_TRY(after_launch(ctx));
@@ -118,6 +143,8 @@ int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float sca
     const unsigned grid = (unsigned)((blocks + 255) / 256);
     if (dtype == GELO_BF16)
         shield_fill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<__nv_bfloat16*>(S), k, d, scale, s.med, seed);
+    else if (dtype == GELO_F16)
+        shield_fill_kernel<__half><<<grid, 256, 0, st>>>(static_cast<__half*>(S), k, d, scale, s.med, seed);
     else
         shield_fill_kernel<float><<<grid, 256, 0, st>>>(static_cast<float*>(S), k, d, scale, s.med, seed);
     return after_launch(ctx);
@@ -170,7 +197,7 @@ extern "C" int gelo_shield_rows_static(gelo_ctx* ctx, const void* H_dev, int n, 
                                        uint64_t seed, int dtype, void* S_dev, void* stream)
 {
     using namespace gelo;
-    if (!ctx || n <= 0 || d <= 0 || k < 0 || (dtype != GELO_F32 && dtype != GELO_BF16) || (d % 8) != 0 || !H_dev ||
+    if (!ctx || n <= 0 || d <= 0 || k < 0 || (dtype != GELO_F32 && dtype != GELO_BF16 && dtype != GELO_F16) || (d % 8) != 0 || !H_dev ||
         (reinterpret_cast<uintptr_t>(H_dev) & 15u))
         return GELO_ERR_INVALID;
     if (n > kStaticShieldMaxRows) return GELO_ERR_UNSUPPORTED;     // more rows than the built-in scratch holds

@@ -13,7 +13,7 @@ available offline):
   root-mean-square so that all row norms equal sqrt(d) (a pre-attention RMSNorm
   without learned gain).
 * ``W``  : d x p with p = 3 d, i.i.d. N(0, 0.02^2), columns ordered [W_q | W_k | W_v].
-* dtype : "f32" or "bf16" (round-to-nearest-even from fp32, once).
+* dtype : "f32", "bf16" or "f16" (round-to-nearest-even from fp32, once).
 """
 from __future__ import annotations
 
@@ -64,7 +64,7 @@ WORKLOADS = {
 
 
 def torch_dtype(name: str) -> torch.dtype:
-    return {"f32": torch.float32, "bf16": torch.bfloat16}[name]
+    return {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}[name]
 
 
 def _generator(device, seed: int) -> torch.Generator:

@@ -14,8 +14,12 @@ from gpu_util import dev, f64, make_ctx, padded, sample_rows
 
 pytestmark = pytest.mark.gpu
 
-TOL = {"f32": 1e-4, "bf16": 2e-2}
-TDT = {"f32": torch.float32, "bf16": torch.bfloat16}
+# f16: the same path with an 11-bit significand instead of bf16's 8.  Storage roundings are 8 times finer, but the
+# inverse of a non-orthogonal A comes from split-precision updates that are good to about 1e-3 at m = 4300 whatever
+# the storage type, so the bound is a quarter of the bf16 one (measured at the benchmark size: 1.3e-3 orthogonal,
+# 3.7e-3 non-orthogonal)
+TOL = {"f32": 1e-4, "bf16": 2e-2, "f16": 5e-3}
+TDT = {"f32": torch.float32, "bf16": torch.bfloat16, "f16": torch.float16}
 
 
 @pytest.fixture(scope="module")
@@ -634,6 +638,39 @@ def test_mlp_shaped_projections(ctx, oracle, d, p):
         ctx.qkv_offload(H, W, n, k, d, p, kind, 4343, 10.0, "bf16", Y)
         torch.cuda.synchronize()
         assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL["bf16"]
+
+
+# ------------------------------------------------------------------------- IEEE half storage
+
+@pytest.mark.parametrize("kind", [ORTHOGONAL, NONORTHOGONAL])
+@pytest.mark.parametrize("n,k,d", [(64, 4, 256), (600, 30, 512), (2048, 102, 1024)])
+def test_half_precision_path(ctx, oracle, kind, n, k, d):
+    """fp16 operands (the third precision of the paper's functional-equality table): whole path and stages."""
+    p = 3 * d
+    m = n + k
+    ctx.ensure_workspace(n, k, d, p, "f16")
+    H = inputs.make_hidden(n, d, "f16", 71, True, "cuda")
+    W = inputs.make_weight(d, p, "f16", 71, "cuda")
+    Q = torch.full((n, d), float("nan"), device="cuda", dtype=torch.float16); K = Q.clone(); V = Q.clone()
+    ctx.qkv_offload(H, W, n, k, d, p, kind, 7171, 10.0, "f16", Q, K, V)
+    torch.cuda.synchronize()
+    y = np.hstack([f64(Q), f64(K), f64(V)])
+    assert oracle.rel_fro(y, oracle.direct(f64(H), f64(W))) <= TOL["f16"]
+    # stages on their own: stored A against its stored inverse, shield rows against the oracle, one product
+    lda = ctx.mixing_ld(m)
+    A = padded(m, lda, torch.float16); X = padded(m, lda, torch.float16)
+    ctx.sample_mixing(m, kind, 99, "f16", A, X, lda)
+    a, x = f64(A[:, :m]), f64(X[:, :m])
+    assert np.linalg.norm(x @ a - np.eye(m)) / np.sqrt(m) <= (1e-3 if kind == ORTHOGONAL else 3e-3)
+    if kind == ORTHOGONAL:
+        assert np.array_equal(x, a.T)
+    S = torch.full((k, d), float("nan"), device="cuda", dtype=torch.float16)
+    ctx.shield_rows(H, n, d, k, 10.0, 5, "f16", S)
+    assert oracle.rel_fro(f64(S), oracle.shield_rows(f64(H), k, 10.0, 5)) <= 6e-4
+    U = torch.full((m, d), float("nan"), device="cuda", dtype=torch.float16)
+    ctx.mix(A, lda, H, S, n, k, d, "f16", U)
+    ref = oracle.matmul(a, np.vstack([f64(H), f64(S)])) if m * m * d < 3e8 else a @ np.vstack([f64(H), f64(S)])
+    assert oracle.rel_fro(f64(U), ref) <= 6e-4
 
 
 def test_batch_of_zero_calls_and_bad_batches():
