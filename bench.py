@@ -393,8 +393,8 @@ def run_ours(args):
         proj_tflops = 2.0 * m * d * p / (stage_ms["project"] * 1e-3) / 1e12
         projection = {"kernel": "gemm_tc_kernel, Y' = U W", "bound": "tensor", "achieved": proj_tflops,
                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": proj_tflops / peaks["bf16_tflops"],
-                      # ncu: dram read 157.1 MB + write 85.9 MB per launch (algorithmic 241.6 MB)
-                      "traffic": 243.0e6}
+                      # ncu: dram read 152.5 MB + write 85.0 MB per launch (algorithmic 241.6 MB)
+                      "traffic": 237.5e6}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,

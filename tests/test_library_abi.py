@@ -49,3 +49,17 @@ def test_host_only_entry_points(lib):
     assert L.gelo_set_workspace(None, None, 0) == binding.ERR_INVALID
     assert L.gelo_destroy(None) == binding.ERR_INVALID
     assert L.gelo_launch_count(None, 0) == -1
+
+
+def test_block_diagonal_grouping_is_checked_on_the_host(lib):
+    from paper_2603_05035_b200 import binding
+    L = binding.load_library()
+    ws = L.gelo_blockdiag_workspace_bytes
+    base = ws(4096, 204, 4096, 12288, 1, 512, 32)
+    assert base > 0
+    assert ws(4096, 204, 4096, 12288, 1, 1024, 32) > base               # larger groups, larger per-lane scratch
+    assert ws(4096, 204, 4096, 12288, 1, 500, 32) == 0                  # group size not a multiple of 64
+    assert ws(4096, 204, 4096, 12288, 1, 64, 32) == 0                   # 68 groups: more than the 32 lanes
+    assert ws(4, 0, 64, 192, 0, 64, 8) > 0 and ws(0, 0, 64, 192, 0, 64, 8) == 0
+    assert ws(4096, 204, 4096, 12288, 7, 512, 32) == 0                  # unknown element type
+    assert ws(4096, 204, 4096, 12288, 2, 512, 32) == base               # half and bfloat16 have the same footprint
