@@ -139,7 +139,7 @@ int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ain
 int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
                        float* cond_dev, void* stream);
 
-/* C_dev (M x N fp32, stride ldc) -= A_dev (M x K fp32, stride lda) * B_dev (K x N fp32, stride ldb), K <= 128:
+/* C_dev (M x N fp32, stride ldc) -= A_dev (M x K fp32, stride lda) * B_dev (K x N fp32, stride ldb), K <= 512:
  * the level-3 update of the blocked QR / LU, on the tensor cores with every operand held as a bf16
  * (high, low) pair and the product accumulated as hi*hi + hi*lo + lo*hi in fp32 (relative error of the
  * product about 1e-5).  ldc must be a multiple of 4 and >= N rounded up to 8; columns N .. that bound are

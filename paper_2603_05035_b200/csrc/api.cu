@@ -960,7 +960,7 @@ int gelo_profile_stop(gelo_ctx* ctx, void* stream, double* out)
 int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int lda, const float* B_dev, int ldb,
                     float* C_dev, int ldc, void* stream)
 {
-    if (!ctx || M <= 0 || N <= 0 || K <= 0 || K > kOuter || !A_dev || !B_dev || !C_dev || lda < K || ldb < N ||
+    if (!ctx || M <= 0 || N <= 0 || K <= 0 || K > kSuper || !A_dev || !B_dev || !C_dev || lda < K || ldb < N ||
         ldc < ((N + 7) & ~7) || (ldc % 4) != 0 || misaligned(C_dev))
         return GELO_ERR_INVALID;
     DeviceGuard guard(ctx->device);

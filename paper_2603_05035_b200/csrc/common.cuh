@@ -59,6 +59,7 @@ struct gelo_ctx {
                                   // 2: always tensor cores, three bf16 products of split operands; 3: always tensor cores, tf32
     long long launches = 0;
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
+    bool tma_3d = true;           // N-major operand tiles as one three-dimensional TMA box where the layout allows
     // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
     int lanes = 4;
     cudaStream_t lane_stream[gelo::kMaxLanes] = {};
