@@ -290,6 +290,15 @@ def run_ours(args):
     timed("project", lambda r: ctx.project(U, Ws[r % calls], m, d, p, w.dtype, Yp), 8)
     timed("unmix", lambda r: ctx.unmix(X, lda, Yp, n, k, p, w.dtype, Q, K, V), 8)
     timed("plain_project", lambda r: ctx.project(Hs[r % calls], Ws[r % calls], n, d, p, w.dtype, Yp), 8)
+    # the level-3 update that leads the SM time of the factorisations: C -= V W with the 512 reflectors of a superblock,
+    # one tf32 product straight from the fp32 matrices (first superblock of the QR: 4300 x 3788, K = 512)
+    um, un, uk = m, m - 512, 512
+    uV = torch.randn((um, uk), device=dev); uW = torch.randn((uk, lda), device=dev)
+    uC = [torch.randn((um, lda), device=dev) for _ in range(4)]             # 4 x 75 MB: C never waits in L2
+    ctx.set_level3(3)
+    timed("tf32_update", lambda r: ctx.update_f32(um, un, uk, uV, uk, uW, lda, uC[r % 4], lda), 16)
+    ctx.set_level3(args.level3)
+    del uV, uW, uC
     chain_ms = stage_ms["mix"] + stage_ms["project"] + stage_ms["unmix"]
     chain_flops = 2.0 * m * m * d + 2.0 * m * d * p + 2.0 * n * m * p
     plain_flops = 2.0 * n * d * p
@@ -395,6 +404,16 @@ def run_ours(args):
                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": proj_tflops / peaks["bf16_tflops"],
                       # ncu: dram read 152.5 MB + write 85.0 MB per launch (algorithmic 241.6 MB)
                       "traffic": 237.5e6}
+        upd_tflops = 2.0 * um * un * uk / (stage_ms["tf32_update"] * 1e-3) / 1e12
+        tf32_peak = 0.5 * peaks["bf16_tflops"]          # nominal dense tf32 : bf16 = 1.125 : 2.25
+        update_roof = {"kernel": "gemm_tc_kernel (tf32, reduce-add epilogue), C -= V W, M=4300 N=3788 K=512",
+                       "bound": "tensor", "achieved": upd_tflops, "peak": tf32_peak, "unit": "TFLOP/s",
+                       "frac": upd_tflops / tf32_peak,
+                       "peak_source": peaks["source"] + " bf16 GEMM x nominal tf32/bf16 ratio 0.5",
+                       # ncu: dram read 82.1 MB + write 8.9 MB per launch (algorithmic 147 MB, half of C stays in L2)
+                       "traffic": 91.0e6,
+                       "note": "largest share of SM time among the sampling kernels (profiles/launch_list_*); "
+                               "its epilogue (read-modify-write of C at the L2) outlasts the main loop"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
@@ -410,6 +429,7 @@ def run_ours(args):
             "gpu_launches": launches,
             "roofline": roofline,
             "roofline_projection_gemm": projection,
+            "roofline_level3_update": update_roof,
             "kernels": kernels,
             "stage_ms": {k_: round(v, 4) for k_, v in stage_ms.items()},
             "chain": {"ms": chain_ms, "tflops": chain_flops / (chain_ms * 1e-3) / 1e12,
