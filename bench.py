@@ -413,7 +413,8 @@ def run_ours(args):
                        # ncu: dram read 82.1 MB + write 8.9 MB per launch (algorithmic 147 MB, half of C stays in L2)
                        "traffic": 91.0e6,
                        "note": "largest share of SM time among the sampling kernels (profiles/launch_list_*); "
-                               "its epilogue (read-modify-write of C at the L2) outlasts the main loop"}
+                               "510 tiles of 16 k-blocks on 148 CTAs: bound by the tf32 main-loop rate (571 TFLOP/s sustained at large K) "
+                               "and the 3.45-wave quantisation"}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
