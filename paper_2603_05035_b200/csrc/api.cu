@@ -125,7 +125,7 @@ int sample_attempt(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t see
     GELO_TRY(launch_gaussian(ctx, m, m, ldi, seed, GELO_STREAM_G0, attempt, 1.0f, nullptr, L.G, st, seed_dev));
     const int l3 = level3_kind(ctx, m, dtype, true);
     if (l3 == 3) GELO_TRY(run_householder_qr_tf32(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, st));
-    else if (l3) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, false, st));
+    else if (l3) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, ldi, L.Qraw, L.qr, L.tc, st));
     else GELO_TRY(run_householder_qr(ctx, m, L.G, ldi, L.Qraw, L.qr, st));
     if (kind == GELO_ORTHOGONAL) {
         // tf32 updates: polish Q (A32 and X32 are free for this kind).  The non-orthogonal kind skips it: there Q0 only
@@ -692,7 +692,7 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
     const int tcp = level3_kind(ctx, m, GELO_F32, true);
     if (ld == L.ldi) {
         if (tcp == 3) GELO_TRY(run_householder_qr_tf32(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, st));
-        else if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, false, st));
+        else if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, G_dev, ld, L.Qraw, L.qr, L.tc, st));
         else GELO_TRY(run_householder_qr(ctx, m, G_dev, ld, L.Qraw, L.qr, st));
         if (tcp == 3) GELO_TRY(polish_orthogonal_tf32(ctx, m, L.Qraw, ld, L.X32, L.A32, st));
         return launch_finish_mixing(ctx, m, L.Qraw, ld, G_dev, ld, GELO_F32, Q_dev, Qt_dev, ld, st);
@@ -700,7 +700,7 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
     GELO_CUDA_OK(cudaMemcpy2DAsync(L.G, (size_t)L.ldi * 4, G_dev, (size_t)ld * 4, (size_t)m * 4, m,
                                    cudaMemcpyDeviceToDevice, st));
     if (tcp == 3) GELO_TRY(run_householder_qr_tf32(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, st));
-    else if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, false, st));
+    else if (tcp) GELO_TRY(run_householder_qr_tc(ctx, m, L.G, L.ldi, L.Qraw, L.qr, L.tc, st));
     else GELO_TRY(run_householder_qr(ctx, m, L.G, L.ldi, L.Qraw, L.qr, st));
     if (tcp == 3) GELO_TRY(polish_orthogonal_tf32(ctx, m, L.Qraw, L.ldi, L.X32, L.A32, st));
     GELO_TRY(launch_finish_mixing(ctx, m, L.Qraw, L.ldi, L.G, L.ldi, GELO_F32, Q_dev, Qt_dev, ld, st));

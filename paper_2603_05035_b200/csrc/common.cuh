@@ -201,8 +201,7 @@ QrScratch carve_qr(Arena&, int m, int ld);
 int run_householder_qr(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, cudaStream_t);
 struct TcScratch;
 // Same factorisation with 128-column outer blocks whose updates run on the tensor cores in split precision.
-int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, bool tf32,
-                          cudaStream_t);
+int run_householder_qr_tc(gelo_ctx*, int m, float* R, int ld, float* Q, const QrScratch&, const TcScratch&, cudaStream_t);
 // The tf32 route: 128-column blocks grouped four by four; only the group's merged reflector (512 columns) is
 // applied to the columns right of the group and, later, to Q, so the big matrices stream through the GPU once per
 // 512 columns instead of once per 128.

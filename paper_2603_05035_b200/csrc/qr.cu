@@ -538,7 +538,7 @@ int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const Q
 }
 
 int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const QrScratch& s, const TcScratch& tc,
-                          bool tf32, cudaStream_t st)
+                          cudaStream_t st)
 {
     // reflector entries above a panel's first row are read (as zeros) by the block-level products
     GELO_CUDA_OK(cudaMemsetAsync(s.V, 0, (size_t)m * ld * sizeof(float), st));
@@ -551,20 +551,6 @@ int run_householder_qr_tc(gelo_ctx* ctx, int m, float* R, int ld, float* Q, cons
         const int nc8 = (nc + 7) & ~7;
         const float* Vb = s.V + (size_t)b0 * ld + b0;
         const float* Tb = s.T128 + (size_t)(b0 / kOuter) * 128 * 128;
-        if (tf32) {
-            // the same three products, each a single tf32 product that reads the fp32 matrices directly:
-            // V^T C takes V as an MN-major operand, T^T W takes T as one; W and T W are rounded to tf32 when stored
-            const int n_tiles = ceil_div(nc8, 256);
-            int want = ceil_div(2 * (ctx->tc_update_ctas > 0 ? ctx->tc_update_ctas : ctx->sm_count), n_tiles);   // slices fill the CTAs this launch may use
-            if (want > kMaxKSplit) want = kMaxKSplit;
-            int used = 0;
-            const size_t plane = (size_t)kOuter * ld;
-            GELO_TRY(launch_gemm_tf32(ctx, ob, nc8, nr, Vb, ld, true, C, ld, false, tc.wf32, ld, false, 1.0f, want, plane, &used, st));
-            GELO_TRY(launch_sum_planes(ctx, tc.wf32, plane, used, ld, ob, nc8, 1.0f, tc.w32[0], ld, st));
-            GELO_TRY(launch_gemm_tf32(ctx, ob, nc8, ob, Tb, 128, transpose_t, tc.w32[0], ld, false, tc.w32[1], ld, true, 1.0f, 1, 0,
-                                      nullptr, st));
-            return launch_gemm_tf32(ctx, nr, nc, ob, Vb, ld, false, tc.w32[1], ld, true, C, ld, false, 1.0f, 1, 0, nullptr, st);
-        }
         GELO_TRY(launch_split(ctx, C, ld, nr, nc, tc.big[0], tc.big[1], ld, false, st));
         GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panA[0], tc.panA[1], kOuter, false, st));
         GELO_TRY(launch_split(ctx, Vb, ld, nr, ob, tc.panAt[0], tc.panAt[1], ld, true, st));
