@@ -37,7 +37,6 @@ constexpr int kAccStages = 2;
 constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kABytes = BM * BK * 2;            // 16 KiB
-constexpr uint32_t kBBoxBytes = 64 * BK * 2;         // 8 KiB per 64-column box
 constexpr uint32_t kTmemCols = 512;
 constexpr unsigned long long kWaitLimit = 40ull * 1000 * 1000;   // try_wait rounds before giving up
 
@@ -219,11 +218,6 @@ __device__ __forceinline__ uint32_t pack_bf16(uint32_t a, uint32_t b)
 __device__ __forceinline__ uint32_t pack_f16(uint32_t a, uint32_t b)
 {
     __half2 h = __floats2half2_rn(__uint_as_float(a), __uint_as_float(b));
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-__device__ __forceinline__ uint32_t pack_bf16f(float a, float b)
-{
-    __nv_bfloat162 h = __floats2bfloat162_rn(a, b);
     return *reinterpret_cast<uint32_t*>(&h);
 }
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi)

@@ -52,12 +52,6 @@ __device__ __forceinline__ void load4(const float* p, float (&x)[4])
     const float4 t = *reinterpret_cast<const float4*>(p);
     x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
 }
-__device__ __forceinline__ void load4(const __nv_bfloat16* p, float (&x)[4])
-{
-    const uint2 t = *reinterpret_cast<const uint2*>(p);
-    x[0] = __uint_as_float(t.x << 16); x[1] = __uint_as_float(t.x & 0xffff0000u);
-    x[2] = __uint_as_float(t.y << 16); x[3] = __uint_as_float(t.y & 0xffff0000u);
-}
 __device__ __forceinline__ void store4(float* p, const float (&x)[4]) { *reinterpret_cast<float4*>(p) = make_float4(x[0], x[1], x[2], x[3]); }
 __device__ __forceinline__ void store4(__nv_bfloat16* p, float (&x)[4])
 {

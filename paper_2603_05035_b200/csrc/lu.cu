@@ -398,6 +398,13 @@ tri_solve_block_kernel(const float* M, int ldm, float* X, int ldx,
 // shared memory, every thread owns one column of X (its 128 entries in a shared-memory tile) and works through
 // the four 32-row sub-blocks with the sub-block in registers: first the contributions of the rows already solved
 // (32 independent FMAs per shared-memory value), then the 32 x 32 substitution.
+// one 4-byte asynchronous copy global -> shared
+__device__ __forceinline__ void cp_async_f32(float* smem_dst, const float* gsrc)
+{
+    const uint32_t d = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(d), "l"(gsrc) : "memory");
+}
+
 constexpr int kTri128LtStride = 132;
 constexpr int kTri128SmemBytes = (128 * kTri128LtStride + 128 * 129) * 4;
 
@@ -411,11 +418,17 @@ tri_solve128_kernel(const float* M, int ldm, float* X, int ldx, int b0, int ob, 
     const int tid = threadIdx.x;
     const int col = c_lo + blockIdx.x * 128 + tid;
     const bool ok = col < c_hi;
-    // many independent loads in flight: these two fills and the write-back are pure latency otherwise
-#pragma unroll 16
-    for (int i = 0; i < 128; ++i) Lt[tid][i] = (i < ob && tid < ob) ? M[(size_t)(b0 + i) * ldm + b0 + tid] : 0.0f;
-#pragma unroll 16
-    for (int t = 0; t < 128; ++t) tile[t][tid] = (ok && t < ob) ? X[(size_t)(b0 + t) * ldx + col] : 0.0f;
+    // The two fills are pure latency (the arithmetic of the solve is about 6 us): every element goes straight from
+    // global to shared memory as an asynchronous 4-byte copy, so that all 256 loads of a thread are in flight at once.
+#pragma unroll 8
+    for (int i = 0; i < 128; ++i) {
+        if (i < ob && tid < ob) cp_async_f32(&Lt[tid][i], M + (size_t)(b0 + i) * ldm + b0 + tid);
+        else Lt[tid][i] = 0.0f;
+        if (ok && i < ob) cp_async_f32(&tile[i][tid], X + (size_t)(b0 + i) * ldx + col);
+        else tile[i][tid] = 0.0f;
+    }
+    asm volatile("cp.async.commit_group;" ::: "memory");
+    asm volatile("cp.async.wait_group 0;" ::: "memory");
     __syncthreads();
     const int nsub = (ob + NB - 1) / NB;
     for (int q = 0; q < nsub; ++q) {
