@@ -50,6 +50,7 @@ struct Layout {
     void* Yd = nullptr;       // n x p
     void* Hd2 = nullptr;      // second pair: the batched host variant alternates between the two
     void* Yd2 = nullptr;
+    Tf32x3Scratch t3;         // fp32 path: tf32 (hi, lo) copies of the operands of the three products
 };
 
 Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
@@ -74,6 +75,17 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     L.S = a.take((size_t)(k > 0 ? k : 1) * d * es);
     L.U = a.take((size_t)L.m * d * es);
     L.Yp = a.take((size_t)L.m * p * es);
+    if (dtype == GELO_F32 && d > 0 && p > 0) {
+        const size_t wide = (size_t)(L.m > d ? L.m : d);
+        L.t3.a_elems = (size_t)L.m * round_up((int)wide, 4);
+        L.t3.b_elems = wide * round_up(p > d ? p : d, 32);
+        for (int h = 0; h < 2; ++h) {
+            L.t3.a[h] = static_cast<float*>(a.take(L.t3.a_elems * 4));
+            L.t3.b[h] = static_cast<float*>(a.take(L.t3.b_elems * 4));
+        }
+        L.t3.c_elems = (size_t)L.m * (p > d ? p : d);
+        L.t3.planes = static_cast<float*>(a.take(L.t3.c_elems * kTf32x3Slices * 4));
+    }
     if (host_staging) {
         L.Hd = a.take((size_t)n * d * es);
         L.Yd = a.take((size_t)n * p * es);
@@ -169,8 +181,28 @@ int sample_mixing_impl(gelo_ctx* ctx, const Layout& L, int m, int kind, uint64_t
     return GELO_ERR_COND;
 }
 
+// A product of the offload.  Large fp32 products run on the tensor cores as three tf32 products of (hi, lo) operand
+// pairs when the call has scratch for the pairs (error about 1e-6, inside the fp32 path's 1e-4); everything else goes
+// to the bf16 / half tensor-core kernel or the FFMA kernel.
+int product(gelo_ctx* ctx, const GemmArgs& g, const Tf32x3Scratch* t3, cudaStream_t st)
+{
+    const int lda3 = round_up(g.K, 4), ldb3 = round_up(g.N, 32);
+    if (g.dtype == GELO_F32 && t3 && t3->a[0] && !g.B2 && !g.transA && !g.transB && g.M >= 128 &&
+        2.0 * g.M * (double)g.N * g.K >= 1e9 && (g.lda % 4) == 0 && (g.ldb % 4) == 0 && (g.ldc % 4) == 0 && (g.K % 4) == 0 &&
+        (g.N % 4) == 0 && (g.N % g.nsplit) == 0 && ((g.N / g.nsplit) % 8) == 0 && !misaligned(g.A) && !misaligned(g.B) &&
+        (size_t)g.M * lda3 <= t3->a_elems && (size_t)g.K * ldb3 <= t3->b_elems) {
+        GELO_TRY(launch_split_tf32(ctx, static_cast<const float*>(g.A), g.lda, g.M, g.K, t3->a[0], t3->a[1], lda3, st));
+        GELO_TRY(launch_split_tf32(ctx, static_cast<const float*>(g.B), g.ldb, g.K, g.N, t3->b[0], t3->b[1], ldb3, st));
+        float* const C[3] = { static_cast<float*>(g.C[0]), static_cast<float*>(g.C[1]), static_cast<float*>(g.C[2]) };
+        float* planes = (size_t)g.M * g.N <= t3->c_elems ? t3->planes : nullptr;
+        return launch_gemm_tf32x3(ctx, g.M, g.N, g.K, t3->a[0], t3->a[1], lda3, t3->b[0], t3->b[1], ldb3, C, g.ldc, g.nsplit,
+                                  planes, st);
+    }
+    return gemm_dispatch(ctx, g, st);
+}
+
 int mix_impl(gelo_ctx* ctx, const void* A, int lda, const void* H, const void* S, int n, int k, int d,
-             int dtype, void* U, cudaStream_t st)
+             int dtype, void* U, cudaStream_t st, const Tf32x3Scratch* t3 = nullptr)
 {
     GemmArgs g;
     g.M = n + k; g.N = d; g.K = n + k;
@@ -178,21 +210,21 @@ int mix_impl(gelo_ctx* ctx, const void* A, int lda, const void* H, const void* S
     g.B = H; g.ldb = d;
     if (k > 0) { g.B2 = S; g.b_split = n; }
     g.C[0] = U; g.ldc = d; g.dtype = dtype;
-    return gemm_dispatch(ctx, g, st);
+    return product(ctx, g, t3, st);
 }
 
 int project_impl(gelo_ctx* ctx, const void* U, const void* W, int m, int d, int p, int dtype, void* Yp,
-                 cudaStream_t st)
+                 cudaStream_t st, const Tf32x3Scratch* t3 = nullptr)
 {
     GemmArgs g;
     g.M = m; g.N = p; g.K = d;
     g.A = U; g.lda = d; g.B = W; g.ldb = p;
     g.C[0] = Yp; g.ldc = p; g.dtype = dtype;
-    return gemm_dispatch(ctx, g, st);
+    return product(ctx, g, t3, st);
 }
 
 int unmix_impl(gelo_ctx* ctx, const void* Ainv, int lda, const void* Yp, int n, int k, int p, int dtype,
-               void* Q, void* K, void* V, cudaStream_t st)
+               void* Q, void* K, void* V, cudaStream_t st, const Tf32x3Scratch* t3 = nullptr)
 {
     GemmArgs g;
     g.M = n; g.N = p; g.K = n + k;
@@ -200,7 +232,7 @@ int unmix_impl(gelo_ctx* ctx, const void* Ainv, int lda, const void* Yp, int n, 
     g.dtype = dtype;
     if (K || V) { g.nsplit = 3; g.C[0] = Q; g.C[1] = K; g.C[2] = V; g.ldc = p / 3; }
     else { g.nsplit = 1; g.C[0] = Q; g.ldc = p; }
-    return gemm_dispatch(ctx, g, st);
+    return product(ctx, g, t3, st);
 }
 
 int check_split(int p, const void* Q, const void* K, const void* V)
@@ -218,9 +250,9 @@ int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, i
     const int m = n + k;
     GELO_TRY(sample_mixing_impl(ctx, L, m, kind, seed, dtype, L.A, L.Ainv, L.ldi, nullptr, st));
     GELO_TRY(run_shield_rows(ctx, H, n, d, k, shield_scale, seed, dtype, L.S, L.sh, st));
-    GELO_TRY(mix_impl(ctx, L.A, L.ldi, H, k > 0 ? L.S : nullptr, n, k, d, dtype, L.U, st));
-    GELO_TRY(project_impl(ctx, L.U, W, m, d, p, dtype, L.Yp, st));
-    return unmix_impl(ctx, L.Ainv, L.ldi, L.Yp, n, k, p, dtype, Q, K, V, st);
+    GELO_TRY(mix_impl(ctx, L.A, L.ldi, H, k > 0 ? L.S : nullptr, n, k, d, dtype, L.U, st, &L.t3));
+    GELO_TRY(project_impl(ctx, L.U, W, m, d, p, dtype, L.Yp, st, &L.t3));
+    return unmix_impl(ctx, L.Ainv, L.ldi, L.Yp, n, k, p, dtype, Q, K, V, st, &L.t3);
 }
 
 
@@ -345,9 +377,9 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         GELO_TRY(run_shield_rows(ctx, Hi, n, d, k, shield_scale, seeds[i], dtype, L[0].S, L[0].sh, st));
         GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
         if (host) GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[b], 0));
-        GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st));
-        GELO_TRY(project_impl(ctx, L[0].U, W[i], m, d, p, dtype, L[0].Yp, st));
-        GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, L[0].Yp, n, k, p, dtype, Qi, Ki, Vi, st));
+        GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st, &L[0].t3));
+        GELO_TRY(project_impl(ctx, L[0].U, W[i], m, d, p, dtype, L[0].Yp, st, &L[0].t3));
+        GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, L[0].Yp, n, k, p, dtype, Qi, Ki, Vi, st, &L[0].t3));
         GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
         if (host) {
             GELO_CUDA_OK(cudaEventRecord(ctx->h_free[b], st));

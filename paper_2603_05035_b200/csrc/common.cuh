@@ -173,6 +173,30 @@ int launch_gemm_tf32(gelo_ctx*, int M, int N, int K, const float* A, int lda, bo
 // when it stored them pass through the tensor core unchanged and need no correction.
 constexpr float kTf32TruncLoss = 3.5224e-4f;
 
+// fp32 products on the tensor cores with fp32-grade accuracy: every operand is held as a pair of tf32 values
+// (hi = x rounded to tf32, lo = the remainder rounded to tf32) and the product is accumulated as
+// hi*hi + hi*lo + lo*hi in fp32 (the dropped lo*lo term is 2^-22 of the product).  C_q (q = 0 .. nsplit-1) receives
+// the q-th column block of the M x N result; strides in elements, all multiples of 4, N / nsplit a multiple of 8.
+// The tensor core adds into its fp32 accumulator with truncation, which costs about 2^-25 of the running sum per
+// instruction, coherently: 5e-5 after the 1536 instructions of a K = 4096 product.  With `planes` (room for
+// kTf32x3Slices * M * N floats) the K range is cut into that many slices with an accumulator each, summed afterwards in
+// round-to-nearest fp32 in a fixed order, which brings the product back to a few 1e-6.
+constexpr int kTf32x3Slices = 8;
+int launch_gemm_tf32x3(gelo_ctx*, int M, int N, int K, const float* Ahi, const float* Alo, int lda, const float* Bhi,
+                       const float* Blo, int ldb, float* const C[3], int ldc, int nsplit, float* planes, cudaStream_t);
+// C_q[r, c] = sum over `parts` planes (M x N, dense) of the entry (r, q * csplit + c), planes added in order
+int launch_sum_planes_routed(gelo_ctx*, const float* planes, size_t plane, int parts, int rows, int cols, float* const C[3],
+                             int ldc, int csplit, cudaStream_t);
+// hi / lo tf32 pair of a rows x cols fp32 block (cols a multiple of 4, 16-byte aligned rows)
+int launch_split_tf32(gelo_ctx*, const float* src, int lds, int rows, int cols, float* hi, float* lo, int ldo, cudaStream_t);
+// scratch of the tf32-pair products of the fp32 path: operand copies of at most a_elems / b_elems floats each
+struct Tf32x3Scratch {
+    float* a[2] = {nullptr, nullptr};
+    float* b[2] = {nullptr, nullptr};
+    float* planes = nullptr;              // kTf32x3Slices partial products of at most c_elems floats each
+    size_t a_elems = 0, b_elems = 0, c_elems = 0;
+};
+
 // ---- factorizations -------------------------------------------------------------------
 
 // ---- rank-32 updates of the factorisations (HBM streamers) ---------------------------------

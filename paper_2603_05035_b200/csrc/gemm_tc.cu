@@ -251,7 +251,9 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
         }
         *reinterpret_cast<uint4*>(static_cast<__nv_bfloat16*>(base) + off) = pk;
     } else if (prm.mode == TC_STORE_F32) {
-        float4* dst = reinterpret_cast<float4*>(static_cast<float*>(prm.C0) + (size_t)slice * prm.plane + (size_t)gm * prm.ldc + gn);
+        const int chunk = gn / prm.csplit;                    // column block -> C0 / C1 / C2 (0 unless the output is split)
+        float* base = static_cast<float*>(chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2));
+        float4* dst = reinterpret_cast<float4*>(base + (size_t)slice * prm.plane + (size_t)gm * prm.ldc + (gn - chunk * prm.csplit));
         float f[8];
 #pragma unroll
         for (int j = 0; j < 8; ++j) {
@@ -788,6 +790,48 @@ int launch_gemm_tf32(gelo_ctx* ctx, int M, int N, int K, const float* A, int lda
     if (used) *used = p.ksplit;
     return a_mn ? launch_tiles<256, 4, false, true, true>(ctx, ma, ma, mb, mb, mc, p, flops, st)
                 : launch_tiles<256, 4, false, true, false>(ctx, ma, ma, mb, mb, mc, p, flops, st);
+}
+
+int launch_gemm_tf32x3(gelo_ctx* ctx, int M, int N, int K, const float* Ahi, const float* Alo, int lda, const float* Bhi,
+                       const float* Blo, int ldb, float* const C[3], int ldc, int nsplit, float* planes, cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if (nsplit < 1 || nsplit > 3 || (N % nsplit) || ((N / nsplit) % 8) || (lda % 4) || (ldb % 4) || (ldc % 4) ||
+        !aligned16(Ahi) || !aligned16(Alo) || !aligned16(Bhi) || !aligned16(Blo))
+        return GELO_ERR_INVALID;
+    for (int q = 0; q < nsplit; ++q)
+        if (!C[q] || !aligned16(C[q])) return GELO_ERR_INVALID;
+    CUtensorMap a0, a1, b0, b1;
+    bool b3d = false, b3d1 = false;
+    if (!make_map_f32_box(ctx, &a0, Ahi, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM) ||
+        !make_map_f32_box(ctx, &a1, Alo, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BM) ||
+        !make_map_nmajor(ctx, &b0, Bhi, 4, true, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, 256, &b3d) ||
+        !make_map_nmajor(ctx, &b1, Blo, 4, true, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 32, 256, &b3d1) || b3d != b3d1)
+        return GELO_ERR_CUDA;
+    TcParams p = {};
+    p.M = M; p.N = N;
+    const int kb = ceil_div(K, 32);
+    p.nseg = 3;
+    p.seg[0] = TcSegment{0, 0, 0, 0, kb};
+    p.seg[1] = TcSegment{0, 1, 0, 0, kb};
+    p.seg[2] = TcSegment{1, 0, 0, 0, kb};
+    p.status = ctx->status_dev;
+    p.b3d = b3d ? 1 : 0;
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
+    p.mode = TC_STORE_F32;
+    p.out_scale = 1.0f; p.post_scale = 1.0f;
+    float* const Cq[3] = { C[0], C[nsplit > 1 ? 1 : 0], C[nsplit > 2 ? 2 : 0] };
+    if (planes && kb >= 2 * kTf32x3Slices && aligned16(planes) && (N % 4) == 0) {
+        const int per = ceil_div(kb, kTf32x3Slices);
+        p.ksplit = ceil_div(kb, per); p.kb_per_split = per; p.plane = (long long)M * N;
+        p.C0 = planes; p.C1 = planes; p.C2 = planes; p.ldc = N; p.csplit = N;
+        GELO_TRY((launch_tiles<256, 4, false, true, false>(ctx, a0, a1, b0, b1, a0, p, 6.0 * M * (double)N * K, st)));
+        return launch_sum_planes_routed(ctx, planes, (size_t)M * N, p.ksplit, M, N, Cq, ldc, N / nsplit, st);
+    }
+    p.C0 = Cq[0]; p.C1 = Cq[1]; p.C2 = Cq[2];
+    p.ldc = ldc; p.csplit = N / nsplit;
+    return launch_tiles<256, 4, false, true, false>(ctx, a0, a1, b0, b1, a0, p, 6.0 * M * (double)N * K, st);
 }
 
 }  // namespace gelo

@@ -232,6 +232,64 @@ int launch_sum_split(gelo_ctx* ctx, const float* planes, size_t plane, int parts
     return after_launch(ctx);
 }
 
+// hi = x rounded to tf32, lo = (x - hi) rounded to tf32: both pass through the tensor core unchanged
+__global__ void __launch_bounds__(256) split_tf32_kernel(const float* __restrict__ src, int lds, int rows, int cols,
+                                                         float* __restrict__ hi, float* __restrict__ lo, int ldo)
+{
+    const int c4 = (blockIdx.x * 256 + threadIdx.x) * 4;
+    if (c4 >= cols) return;
+    for (int r = blockIdx.y; r < rows; r += gridDim.y) {
+        const float4 t = *reinterpret_cast<const float4*>(src + (size_t)r * lds + c4);
+        const float x[4] = {t.x, t.y, t.z, t.w};
+        uint32_t h[4], l[4];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(h[j]) : "f"(x[j]));
+            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(l[j]) : "f"(x[j] - __uint_as_float(h[j])));
+        }
+        *reinterpret_cast<uint4*>(hi + (size_t)r * ldo + c4) = make_uint4(h[0], h[1], h[2], h[3]);
+        *reinterpret_cast<uint4*>(lo + (size_t)r * ldo + c4) = make_uint4(l[0], l[1], l[2], l[3]);
+    }
+}
+
+__global__ void __launch_bounds__(256) sum_planes_routed_kernel(const float* __restrict__ planes, size_t plane, int parts,
+                                                                int cols, float* __restrict__ C0, float* __restrict__ C1,
+                                                                float* __restrict__ C2, int ldc, int csplit)
+{
+    const int c4 = (blockIdx.x * 256 + threadIdx.x) * 4;
+    const int r = blockIdx.y;
+    if (c4 >= cols) return;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int q = 0; q < parts; ++q) {
+        const float4 t = *reinterpret_cast<const float4*>(planes + q * plane + (size_t)r * cols + c4);
+        acc.x += t.x; acc.y += t.y; acc.z += t.z; acc.w += t.w;
+    }
+    const int chunk = c4 / csplit;                            // csplit is a multiple of 8: a group of four never straddles
+    float* base = chunk == 0 ? C0 : (chunk == 1 ? C1 : C2);
+    *reinterpret_cast<float4*>(base + (size_t)r * ldc + (c4 - chunk * csplit)) = acc;
+}
+
+int launch_sum_planes_routed(gelo_ctx* ctx, const float* planes, size_t plane, int parts, int rows, int cols,
+                             float* const C[3], int ldc, int csplit, cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return GELO_OK;
+    dim3 grid(ceil_div(cols, 1024), rows);
+    sum_planes_routed_kernel<<<grid, 256, 0, st>>>(planes, plane, parts, cols, C[0], C[1], C[2], ldc, csplit);
+    return after_launch(ctx);
+}
+
+int launch_split_tf32(gelo_ctx* ctx, const float* src, int lds, int rows, int cols, float* hi, float* lo, int ldo,
+                      cudaStream_t st)
+{
+    if (rows <= 0 || cols <= 0) return GELO_OK;
+    if ((cols % 4) || (lds % 4) || (ldo % 4) || (reinterpret_cast<uintptr_t>(src) & 15u) ||
+        (reinterpret_cast<uintptr_t>(hi) & 15u) || (reinterpret_cast<uintptr_t>(lo) & 15u))
+        return GELO_ERR_INVALID;
+    dim3 grid(ceil_div(cols, 1024), rows < 4096 ? rows : 4096);
+    split_tf32_kernel<<<grid, 256, 0, st>>>(src, lds, rows, cols, hi, lo, ldo);
+    return after_launch(ctx);
+}
+
 int launch_sum_planes(gelo_ctx* ctx, const float* planes, size_t plane, int parts, int ld, int rows, int cols, float scale,
                       float* out, int ldo, cudaStream_t st)
 {
