@@ -270,6 +270,10 @@ int launch_narrow(gelo_ctx*, int m, const float* src, int lds, int dtype, void* 
 int launch_split(gelo_ctx*, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
                  bool transpose, cudaStream_t);
 
+// the same for two blocks in one launch (neither transposed)
+int launch_split_pair(gelo_ctx*, const float* A, int lda, int rows_a, int cols_a, void* Ahi, void* Alo, int ldoa,
+                      const float* B, int ldb, int rows_b, int cols_b, void* Bhi, void* Blo, int ldob, cudaStream_t);
+
 int launch_sum_split(gelo_ctx*, const float* planes, size_t plane, int parts, int ld, int rows, int cols, void* hi,
                      void* lo, int ldo, cudaStream_t);
 // out = scale * (sum of `parts` fp32 planes in plane order), rounded to tf32 (cols a multiple of 4)

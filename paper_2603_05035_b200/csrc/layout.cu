@@ -199,7 +199,79 @@ __global__ void __launch_bounds__(256) split_transpose_kernel(const float* __res
     }
 }
 
+// Two split jobs in one launch (blockIdx.z selects the job): the A and B operands of one split-precision update.  A
+// row takes min(256, cols / 4) threads (four columns each), the rest of the CTA's threads take further rows, so a thin
+// block column keeps all 256 threads busy.
+struct SplitJob { const float* src; int lds, rows, cols; __nv_bfloat16* hi; __nv_bfloat16* lo; int ldo, tpr; };
+
+__global__ void __launch_bounds__(256) split_pair_kernel(const SplitJob ja, const SplitJob jb)
+{
+    const SplitJob& j = blockIdx.z ? jb : ja;
+    const int tpr = j.tpr;                                   // threads per row (a power of two <= 256)
+    const int c4 = (blockIdx.x * tpr + (threadIdx.x & (tpr - 1))) * 4;
+    const int rpc = 256 / tpr;                               // rows per CTA and pass
+    if (c4 >= j.cols) return;
+    for (int r = blockIdx.y * rpc + threadIdx.x / tpr; r < j.rows; r += gridDim.y * rpc) {
+        const float* p = j.src + (size_t)r * j.lds + c4;
+        float x[4];
+        if (c4 + 3 < j.cols) {
+            const float4 t = *reinterpret_cast<const float4*>(p);
+            x[0] = t.x; x[1] = t.y; x[2] = t.z; x[3] = t.w;
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) x[q] = (c4 + q < j.cols) ? p[q] : 0.0f;
+        }
+        __nv_bfloat16 h[4], l[4];
+#pragma unroll
+        for (int q = 0; q < 4; ++q) {
+            h[q] = __float2bfloat16_rn(x[q]);
+            l[q] = __float2bfloat16_rn(x[q] - __bfloat162float(h[q]));
+        }
+        __nv_bfloat16* ph = j.hi + (size_t)r * j.ldo + c4;
+        __nv_bfloat16* pl = j.lo + (size_t)r * j.ldo + c4;
+        if (c4 + 3 < j.cols) {
+            *reinterpret_cast<uint2*>(ph) = *reinterpret_cast<const uint2*>(h);
+            *reinterpret_cast<uint2*>(pl) = *reinterpret_cast<const uint2*>(l);
+        } else {
+#pragma unroll
+            for (int q = 0; q < 4; ++q)
+                if (c4 + q < j.cols) { ph[q] = h[q]; pl[q] = l[q]; }
+        }
+    }
+}
+
 }  // namespace
+
+int launch_split_pair(gelo_ctx* ctx, const float* A, int lda, int rows_a, int cols_a, void* Ahi, void* Alo, int ldoa,
+                      const float* B, int ldb, int rows_b, int cols_b, void* Bhi, void* Blo, int ldob, cudaStream_t st)
+{
+    auto vec_ok = [](const float* s, int lds, const void* hi, const void* lo, int ldo) {
+        return (lds & 3) == 0 && (ldo & 3) == 0 && (reinterpret_cast<uintptr_t>(s) & 15u) == 0 &&
+               (reinterpret_cast<uintptr_t>(hi) & 7u) == 0 && (reinterpret_cast<uintptr_t>(lo) & 7u) == 0;
+    };
+    if (rows_a <= 0 || cols_a <= 0 || rows_b <= 0 || cols_b <= 0 || !vec_ok(A, lda, Ahi, Alo, ldoa) || !vec_ok(B, ldb, Bhi, Blo, ldob)) {
+        GELO_TRY(launch_split(ctx, A, lda, rows_a, cols_a, Ahi, Alo, ldoa, false, st));
+        return launch_split(ctx, B, ldb, rows_b, cols_b, Bhi, Blo, ldob, false, st);
+    }
+    auto job = [](const float* s, int lds, int rows, int cols, void* hi, void* lo, int ldo) {
+        SplitJob j;
+        j.src = s; j.lds = lds; j.rows = rows; j.cols = cols;
+        j.hi = static_cast<__nv_bfloat16*>(hi); j.lo = static_cast<__nv_bfloat16*>(lo); j.ldo = ldo;
+        int tpr = 1;
+        while (tpr < 256 && tpr * 4 < cols) tpr *= 2;
+        j.tpr = tpr;
+        return j;
+    };
+    const SplitJob ja = job(A, lda, rows_a, cols_a, Ahi, Alo, ldoa), jb = job(B, ldb, rows_b, cols_b, Bhi, Blo, ldob);
+    auto gx = [](const SplitJob& j) { return ceil_div(j.cols, 4 * j.tpr); };
+    auto gy = [](const SplitJob& j) { return ceil_div(j.rows, 256 / j.tpr); };
+    const int grid_x = gx(ja) > gx(jb) ? gx(ja) : gx(jb);
+    int grid_y = gy(ja) > gy(jb) ? gy(ja) : gy(jb);
+    const int cap = ceil_div(4 * ctx->sm_count, grid_x);      // a few CTAs per SM and job; rows beyond that are strided
+    if (grid_y > cap) grid_y = cap;
+    split_pair_kernel<<<dim3(grid_x, grid_y, 2), 256, 0, st>>>(ja, jb);
+    return after_launch(ctx);
+}
 
 int launch_split(gelo_ctx* ctx, const float* src, int lds, int rows, int cols, void* hi, void* lo, int ldo,
                  bool transpose, cudaStream_t st)

@@ -287,8 +287,7 @@ int tc_update_f32(gelo_ctx* ctx, const TcScratch& t, bool tf32, int M, int N, in
     if (tf32) return launch_gemm_tf32(ctx, M, N, K, A, lda, false, B, ldb, true, C, ldc, false, 1.0f, 1, 0, nullptr, st);
     const int ldn = (N + 7) & ~7;
     const int ldk = (K + 63) & ~63;
-    GELO_TRY(launch_split(ctx, A, lda, M, K, t.panA[0], t.panA[1], ldk, false, st));
-    GELO_TRY(launch_split(ctx, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, false, st));
+    GELO_TRY(launch_split_pair(ctx, A, lda, M, K, t.panA[0], t.panA[1], ldk, B, ldb, K, N, t.rowB[0], t.rowB[1], ldn, st));
     return launch_gemm_tc_split(ctx, M, N, K, t.panA[0], t.panA[1], ldk, t.rowB[0], t.rowB[1], ldn, C, ldc,
                                 nullptr, nullptr, 0, false, st);
 }
