@@ -33,8 +33,8 @@ if ROOT not in sys.path:
 METRIC = "obfuscated-QKV tokens/s at Llama-2-7B shapes"
 UNIT = "tokens/s"
 WORKLOAD = "prefill_bf16"
-# DRAM bytes over algorithmic bytes of the panel kernels, from one ncu capture (profiles/qr_panel_cluster_kernel_*):
-# the capture ran a panel of 3300 rows; traffic scales with the rows, so other panel heights use the same ratio.
+# DRAM bytes over algorithmic bytes of the panel kernels, from one ncu capture of a panel of 3300 rows; traffic
+# scales with the rows, so other panel heights use the same ratio.
 PANEL_TRAFFIC_RATIO = 0.49
 
 
@@ -370,6 +370,16 @@ def run_ours(args):
         if ctx.last_status() != gelo.OK:
             raise SystemExit("device-side error in the variant runs")
 
+    workloads = {}
+    if world == 1 and not args.no_workloads:
+        # the other configurations, a few sweeps each; their numbers ride along in the main line
+        ctx.set_workspace(None)
+        torch.cuda.empty_cache()
+        for name_ in ("tiny_f32", "layer_f32", "shield_bf16", "decode_bf16"):
+            lat = args.latency_steps if name_ == "decode_bf16" else 0
+            workloads[name_] = compact(measure_workload(name_, min(args.lanes, 16) if name_ != "shield_bf16" else args.lanes,
+                                                        5, 3, 0, lat))
+
     if rank == 0:
         es = 2 if w.dtype == "bf16" else 4
         dk = kernels[dominant]
@@ -412,9 +422,23 @@ def run_ours(args):
                        "peak_source": peaks["source"] + " bf16 GEMM x nominal tf32/bf16 ratio 0.5",
                        # ncu: dram read 82.1 MB + write 8.9 MB per launch (algorithmic 147 MB, half of C stays in L2)
                        "traffic": 91.0e6,
-                       "note": "largest share of SM time among the sampling kernels (profiles/launch_list_*); "
+                       "note": "largest share of SM time among the sampling kernels; "
                                "510 tiles of 16 k-blocks on 148 CTAs: bound by the tf32 main-loop rate (571 TFLOP/s sustained at large K) "
                                "and the 3.45-wave quantisation"}
+        per_call_ms = ms_max / args.steps / calls
+        chain_tflops = chain_flops / (chain_ms * 1e-3) / 1e12
+        # all arithmetic of a sweep against the time the sweep takes with every lane busy: the Householder QR of every
+        # call ((8/3) m^3 with the explicit Q), one Newton-Schulz step (4 m^3) per orthogonal call on the tf32 route, LU
+        # and inverse (2 m^3) per non-orthogonal call, and the three products; tf32 and split-bf16 flops are counted
+        # once each, so this is a lower-is-slack figure against the bf16 peak
+        n_orth = sum(1 for c_ in range(calls) if kinds[c_] == gelo.ORTHOGONAL)
+        sweep_flops = calls * ((8.0 / 3.0) * m ** 3 + chain_flops) + n_orth * 4.0 * m ** 3 + (calls - n_orth) * 2.0 * m ** 3
+        sweep_tflops = sweep_flops / (ms_max / args.steps * 1e-3) / 1e12
+        sweep_roof = {"kernel": "all kernels of one sweep, lanes saturated (SM-time-weighted)", "bound": "tensor",
+                      "achieved": sweep_tflops, "unit": "TFLOP/s", "peak": peaks["bf16_tflops_sustained"],
+                      "frac": sweep_tflops / peaks["bf16_tflops_sustained"],
+                      "peak_source": peaks["source"] + " (sustained bf16 GEMM)", "traffic": None,
+                      "algorithmic_flops_per_sweep": sweep_flops}
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_max / args.steps, "higher_is_better": True,
@@ -433,12 +457,23 @@ def run_ours(args):
             "roofline_level3_update": update_roof,
             "kernels": kernels,
             "stage_ms": {k_: round(v, 4) for k_, v in stage_ms.items()},
-            "chain": {"ms": chain_ms, "tflops": chain_flops / (chain_ms * 1e-3) / 1e12,
-                      "overhead_vs_plain_gemm": chain_ms / stage_ms["plain_project"],
+            # the metric's second half: the WHOLE obfuscated call (sampling A, shields, three products) against the plain,
+            # unprotected H W on the same kernel; the products alone and their arithmetic floor beside it
+            "overhead_vs_plain_gemm": per_call_ms / stage_ms["plain_project"],
+            "products_vs_plain_gemm": chain_ms / stage_ms["plain_project"],
+            "flop_floor_vs_plain": chain_flops / plain_flops,
+            "per_call_ms": per_call_ms,
+            "chain": {"ms": chain_ms, "tflops": chain_tflops,
+                      "products_vs_plain_gemm": chain_ms / stage_ms["plain_project"],
                       "flop_floor_vs_plain": chain_flops / plain_flops,
-                      "frac_of_peak": chain_flops / (chain_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]},
+                      "frac_of_peak": {"measured_burst": chain_tflops / peaks["bf16_tflops"],
+                                       "measured_sustained": chain_tflops / peaks["bf16_tflops_sustained"],
+                                       "nominal_2250": chain_tflops / 2250.0}},
+            "roofline_whole_sweep": sweep_roof,
             "checksum": float(checksum),
         }
+        if workloads:
+            line["workloads"] = workloads
         if variants:
             line["variants_block_diagonal_A"] = variants
         if world == 1 and not args.no_cpu_baseline:
@@ -456,23 +491,24 @@ def run_ours(args):
     return 0
 
 
-def run_workload(args):
-    """A secondary line for one of the other workloads (parity-test configurations): whole-path rate through the
-    batched entry point, per-stage device times, overhead against the plain H W GEMM on the same kernel."""
+def measure_workload(name, lanes, steps, warmup, calls=0, latency_steps=0):
+    """Whole-path rate of one of the other workloads (the parity-test configurations) through the batched entry
+    point, per-stage device times, overhead against the plain H W GEMM on the same kernel.  With `latency_steps`
+    (the decode-shaped workload) also the distribution of the per-call latency over that many sweeps."""
+    import numpy as np
     import torch
     import paper_2603_05035_b200 as gelo
     from paper_2603_05035_b200 import inputs
 
-    w = inputs.WORKLOADS[args.workload]
+    w = inputs.WORKLOADS[name]
     n, k, d, p, m = w.n, w.k, w.d, w.p, w.m
-    calls = args.calls if args.calls > 0 else 32
+    calls = calls if calls > 0 else 32
     td = inputs.torch_dtype(w.dtype)
-    dev = torch.device("cuda", 0)
-    torch.cuda.set_device(0)
+    dev = torch.device("cuda", torch.cuda.current_device())
     peaks = _peaks()
-    ctx = gelo.Context(0)
-    ctx.set_lanes(args.lanes)
-    ctx.ensure_batch_workspace(n, k, d, p, w.dtype, args.lanes)
+    ctx = gelo.Context(dev.index)
+    ctx.set_lanes(lanes)
+    ctx.ensure_batch_workspace(n, k, d, p, w.dtype, lanes)
     Hs = [inputs.make_hidden(n, d, w.dtype, w.seed + c, w.rms_norm, dev) for c in range(calls)]
     Ws = [inputs.make_weight(d, p, w.dtype, w.seed + c, dev) for c in range(calls)]      # 32 distinct W: larger than L2
     Q = torch.empty((n, p // 3), device=dev, dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
@@ -482,15 +518,15 @@ def run_workload(args):
         ctx.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, [w.seed + 100000 * (step + 7) + c for c in range(calls)],
                               w.shield_scale, w.dtype, [Q] * calls, [K] * calls, [V] * calls)
 
-    for i in range(max(3, args.warmup)):
+    for i in range(max(3, warmup)):
         sweep(-1 - i)
     torch.cuda.synchronize()
-    sampler = ClockSampler(0)
+    sampler = ClockSampler(dev.index)
     sampler.start()
     ctx.launch_count(reset=True)
     e0 = torch.cuda.Event(enable_timing=True); e1 = torch.cuda.Event(enable_timing=True)
     e0.record()
-    for s_ in range(args.steps):
+    for s_ in range(steps):
         sweep(s_)
     e1.record()
     torch.cuda.synchronize()
@@ -498,7 +534,7 @@ def run_workload(args):
     launches = ctx.launch_count()
     clocks = sampler.stop()
     if ctx.last_status() != gelo.OK:
-        raise SystemExit("device-side error in the timed region")
+        raise SystemExit(f"device-side error in the timed region of {name}")
 
     stage_ms = {}
     lda = ctx.mixing_ld(m)
@@ -506,7 +542,7 @@ def run_workload(args):
     S = torch.empty((max(k, 1), d), device=dev, dtype=td)
     U = torch.empty((m, d), device=dev, dtype=td); Yp = torch.empty((m, p), device=dev, dtype=td)
 
-    def timed(name, fn, reps):
+    def timed(key, fn, reps):
         fn(0)
         torch.cuda.synchronize()
         a = torch.cuda.Event(enable_timing=True); b = torch.cuda.Event(enable_timing=True)
@@ -515,7 +551,7 @@ def run_workload(args):
             fn(r + 1)
         b.record()
         torch.cuda.synchronize()
-        stage_ms[name] = a.elapsed_time(b) / reps
+        stage_ms[key] = a.elapsed_time(b) / reps
 
     kind0 = kinds[0]
     timed("sample", lambda r: ctx.sample_mixing(m, kind0, 900 + r, w.dtype, A, X, lda), 4)
@@ -524,33 +560,100 @@ def run_workload(args):
     timed("mix", lambda r: ctx.mix(A, lda, Hs[r % calls], S if k else None, n, k, d, w.dtype, U), 16)
     timed("project", lambda r: ctx.project(U, Ws[r % calls], m, d, p, w.dtype, Yp), 32)
     timed("unmix", lambda r: ctx.unmix(X, lda, Yp, n, k, p, w.dtype, Q, K, V), 16)
+    # the plain, unprotected projection through the same entry point, hence on the same kernel as the chain's products
     timed("plain_project", lambda r: ctx.project(Hs[r % calls], Ws[r % calls], n, d, p, w.dtype, Yp), 32)
-    per_call_ms = ms / (args.steps * calls)
-    es = 2 if w.dtype == "bf16" else 4
+    if w.dtype == "f32":
+        # a context without workspace has no room for operand pairs: the same product on the FP32 FMA pipes
+        bare = gelo.Context(dev.index)
+        timed("plain_project_fma", lambda r: bare.project(Hs[r % calls], Ws[r % calls], n, d, p, w.dtype, Yp), 8)
+        bare.close()
+    per_call_ms = ms / (steps * calls)
+    es = 2 if w.dtype != "f32" else 4
     proj_s = stage_ms["project"] * 1e-3
+    chain_flops = 2.0 * m * m * d + 2.0 * m * d * p + 2.0 * n * m * p
     if w.dtype == "bf16" and m >= 512:
         roof = {"bound": "tensor", "achieved": 2.0 * m * d * p / proj_s / 1e12, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s"}
     elif w.dtype == "bf16":
         roof = {"bound": "hbm", "achieved": es * (m * d + d * p + m * p) / proj_s / 1e9, "peak": peaks["hbm_gbs"], "unit": "GB/s"}
+    elif 2.0 * m * d * p >= 1e9 and m >= 128:
+        # three tf32 products per fp32 product: the tensor cores do 3 x the algorithmic flops at the tf32 rate
+        roof = {"bound": "tensor", "achieved": 2.0 * m * d * p / proj_s / 1e12, "peak": 0.5 * peaks["bf16_tflops"] / 3.0,
+                "unit": "TFLOP/s", "peak_source": peaks["source"] + " bf16 GEMM x nominal tf32/bf16 ratio 0.5 / 3 products"}
     else:
         roof = {"bound": "alu", "achieved": 2.0 * m * d * p / proj_s / 1e12, "peak": 148 * 128 * 2 * 1.965e9 / 1e12,
-                "unit": "TFLOP/s"}
+                "unit": "TFLOP/s", "peak_source": "derived: 148 SMs x 128 FP32 lanes x 2 x 1.965 GHz"}
+    roof.setdefault("peak_source", peaks["source"])
     roof.update({"kernel": "projection GEMM Y' = U W", "frac": roof["achieved"] / roof["peak"], "traffic": None})
     line = {
-        "metric": METRIC, "value": float(n) * calls * args.steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": args.steps,
-        "warmup": max(3, args.warmup), "ms_per_step": ms / args.steps, "higher_is_better": True, "scaling": "weak",
+        "metric": METRIC, "value": float(n) * calls * steps / (ms * 1e-3), "unit": UNIT, "n_gpus": 1, "steps": steps,
+        "warmup": max(3, warmup), "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak",
         "vs_baseline": None, "dtype": w.dtype, "data": "synthetic",
         "config": {"workload": w.name, "n": n, "k": k, "m": m, "d": d, "p": p, "calls_per_step": calls,
                    "mixing": ["orthogonal", "non-orthogonal"][kind0] if len(set(kinds)) == 1 else "alternating",
                    "shield_scale": w.shield_scale, "l2": "inputs_larger_than_l2" if calls * d * p * es > 126e6 else "l2_resident",
-                   "api": "gelo_qkv_offload_batch", "lanes": args.lanes},
+                   "api": "gelo_qkv_offload_batch", "lanes": lanes},
         "clocks": clocks, "gpu_launches": launches, "roofline": roof,
         "per_call_us": 1e3 * per_call_ms, "stage_ms": {k_: round(v, 5) for k_, v in stage_ms.items()},
         "overhead_vs_plain_gemm": per_call_ms / stage_ms["plain_project"],
         "products_vs_plain_gemm": (stage_ms["mix"] + stage_ms["project"] + stage_ms["unmix"]) / stage_ms["plain_project"],
+        "flop_floor_vs_plain": chain_flops / (2.0 * n * d * p),
     }
-    print(json.dumps(line))
+    if "plain_project_fma" in stage_ms:
+        line["overhead_vs_plain_gemm_fma"] = per_call_ms / stage_ms["plain_project_fma"]
+    if latency_steps > 0:
+        # per-call latency over `latency_steps` sweeps of `calls` layers: (a) sweeps through the batched entry point,
+        # one event per sweep, latency = sweep time / calls; (b) single calls through gelo_qkv_offload, one event pair each
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(latency_steps + 1)]
+        ev[0].record()
+        for s_ in range(latency_steps):
+            sweep(1000 + s_)
+            ev[s_ + 1].record()
+        torch.cuda.synchronize()
+        per = np.array([ev[i].elapsed_time(ev[i + 1]) for i in range(latency_steps)]) * 1e3 / calls
+        singles = min(2000, latency_steps * 2)
+        a_ev = [torch.cuda.Event(enable_timing=True) for _ in range(singles)]
+        b_ev = [torch.cuda.Event(enable_timing=True) for _ in range(singles)]
+        for r in range(singles + 8):
+            c_ = r % calls
+            if r >= 8:
+                a_ev[r - 8].record()
+            ctx.qkv_offload(Hs[c_], Ws[c_], n, k, d, p, kinds[c_], 777 + r, w.shield_scale, w.dtype, Q, K, V)
+            if r >= 8:
+                b_ev[r - 8].record()
+        torch.cuda.synchronize()
+        one = np.array([a_ev[i].elapsed_time(b_ev[i]) for i in range(singles)]) * 1e3
+        if ctx.last_status() != gelo.OK:
+            raise SystemExit(f"device-side error in the latency run of {name}")
+        line["latency_us"] = {
+            "calls_timed": int(latency_steps * calls),
+            "batched_per_call": {"p50": float(np.percentile(per, 50)), "p99": float(np.percentile(per, 99)),
+                                 "mean": float(per.mean()), "sweeps": int(latency_steps), "calls_per_sweep": int(calls)},
+            "single_call": {"p50": float(np.percentile(one, 50)), "p99": float(np.percentile(one, 99)),
+                            "mean": float(one.mean()), "calls": int(singles)},
+            "plain_gemm": 1e3 * stage_ms["plain_project"],
+            "batched_p50_vs_plain_gemm": float(np.percentile(per, 50)) / (1e3 * stage_ms["plain_project"]),
+        }
     ctx.close()
+    return line
+
+
+def compact(line):
+    """The part of a secondary workload's line that the main line carries."""
+    keep = ("per_call_us", "overhead_vs_plain_gemm", "overhead_vs_plain_gemm_fma", "products_vs_plain_gemm",
+            "flop_floor_vs_plain", "value", "stage_ms", "latency_us")
+    out = {k_: line[k_] for k_ in keep if k_ in line}
+    out["config"] = {k_: line["config"][k_] for k_ in ("n", "k", "d", "p", "calls_per_step", "mixing", "lanes")}
+    out["dtype"] = line["dtype"]
+    out["projection_roofline"] = {k_: line["roofline"][k_] for k_ in ("bound", "achieved", "peak", "unit", "frac")}
+    return out
+
+
+def run_workload(args):
+    import torch
+    torch.cuda.set_device(0)
+    steps = args.steps
+    latency = args.latency_steps if args.workload == "decode_bf16" else 0
+    print(json.dumps(measure_workload(args.workload, args.lanes, steps, args.warmup, args.calls, latency)))
     return 0
 
 
@@ -567,6 +670,9 @@ def main():
     ap.add_argument("--level3", type=int, default=0, choices=[0, 1, 2, 3],
                     help="factorisation updates: 0 auto (tensor cores for bf16), 1 fp32 FMA, 2 tensor cores")
     ap.add_argument("--calls", type=int, default=0, help="projection calls per step (default: the workload's 32)")
+    ap.add_argument("--latency-steps", type=int, default=1000,
+                    help="decode_bf16: sweeps of 32 calls whose per-call latency distribution is reported")
+    ap.add_argument("--no-workloads", action="store_true", help="skip the secondary workloads in the main line")
     ap.add_argument("--timed-only", action="store_true",
                     help="run only the warm-up and the timed sweeps (for profiler launch lists)")
     ap.add_argument("--workload", default=WORKLOAD, choices=["tiny_f32", "layer_f32", "shield_bf16", "prefill_bf16", "decode_bf16"],

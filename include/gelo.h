@@ -98,6 +98,14 @@ int gelo_set_level3(gelo_ctx* ctx, int mode);
 /* Preferred row stride (elements) of an m x m mixing matrix: m rounded up to 64. */
 int gelo_mixing_ld(int m);
 
+/* Limit, in nanoseconds of the GPU's global timer, of every device-side wait on a pipeline
+ * barrier in the tensor-core kernels (default 2e9 = two seconds).  When a wait runs out the
+ * CTA records GELO_ERR_TIMEOUT in the status word, stops issuing work, frees its tensor
+ * memory and returns, and the outputs of that call are invalid.  A limit of 0 makes every
+ * such kernel give up before it issues its first copy or MMA: a diagnostic setting that lets
+ * a test see the timeout path without making any wait actually run out. */
+int gelo_set_wait_limit_ns(gelo_ctx* ctx, unsigned long long ns);
+
 /* Status word of the context: waits for `stream`, then returns the first device-side
  * error recorded since the last call of this function (GELO_OK if none) and clears it. */
 int gelo_last_status(gelo_ctx* ctx, void* stream);
@@ -107,7 +115,7 @@ long long gelo_launch_count(gelo_ctx* ctx, int reset);
 
 const char* gelo_status_string(int status);
 
-/* ---- sampling (Section 3.2 step 1.2: "sample a fresh, random invertible matrix") ---- */
+/* ---- sampling (Section 3.2 step 1.2: every batch gets a newly drawn random invertible A) ---- */
 
 /* Debug export of the random stream: out_dev[i] = the Philox4x32-10 word of element
  * first+i of (seed, stream_id, attempt).  Element e uses block e/4 -- counter
@@ -118,7 +126,8 @@ int gelo_philox_words(gelo_ctx* ctx, uint64_t seed, uint32_t stream_id, uint32_t
 /* out_dev (rows x cols fp32, row stride ld) = scale * N(0,1).  Element (i,j) is stream
  * element i*cols + j; words (0,1) and (2,3) of a block are Box-Muller pairs, the even
  * word giving r*cos(2 pi u_b), the odd word r*sin(2 pi u_b), r = sqrt(-2 ln u_a),
- * u = ((word >> 8) + 1/2) / 2^24. */
+ * u = ((word >> 9) + 1/2) / 2^23: 23 bits, so that every u is exactly representable in
+ * binary32 and the fp32 device arithmetic starts from the same value as an fp64 check. */
 int gelo_sample_gaussian(gelo_ctx* ctx, int rows, int cols, int ld, uint64_t seed,
                          uint32_t stream_id, uint32_t attempt, float scale, float* out_dev,
                          void* stream);
@@ -153,8 +162,10 @@ int gelo_update_f32(gelo_ctx* ctx, int M, int N, int K, const float* A_dev, int 
  *   GELO_ORTHOGONAL:    A = Q of QR(G0), G0 ~ N(0,1) from stream 0;  A^-1 = A^T.
  *   GELO_NONORTHOGONAL: A = Q0 + gamma * G1 / sqrt(m) (G1 from stream 1), rounded to the
  *                       element type, then A^-1 of that stored A; accepted when the
- *                       kappa_2 estimate * 1.1 <= bound, else resampled with the next
- *                       attempt number.  This kind WAITS for `stream` once per attempt
+ *                       kappa_2 estimate * 1.2 <= bound, else resampled with the next
+ *                       attempt number.  The bound is enforced on an ESTIMATE (power
+ *                       iteration, a lower estimate that tests put at 0.85 .. 1.0 of the
+ *                       true value, hence the factor 1 / 0.85 rounded up).  This kind WAITS for `stream` once per attempt
  *                       to read the verdict; GELO_ERR_COND after the last attempt.
  * A_dev, Ainv_dev: m x m in `dtype`, stride lda.  cond_dev (optional, device float)
  * receives the estimate (1 for orthogonal).  Same (m, kind, seed) => same bytes. */
@@ -225,8 +236,8 @@ int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, 
 /* ---- batches of independent calls ---------------------------------------------------------- */
 
 /* The same path for `calls` independent batches (for instance the Q/K/V projections of the
- * layers of one prefill sweep; paper Section 3.2: "a fresh ... matrix A for this batch (never
- * reused across batches)").  Sampling A needs only the seed, so up to `lanes` calls sample
+ * layers of one prefill sweep; paper Section 3.2 step 1.2 draws a new A for every batch and
+ * never uses one twice).  Sampling A needs only the seed, so up to `lanes` calls sample
  * their mixing pairs concurrently on streams owned by the context while `stream` runs the
  * shield rows and the three products of earlier calls; results are those of gelo_qkv_offload
  * with the same (kind, seed) per call.

@@ -62,6 +62,7 @@ EXPORTS = {
     "gelo_qkv_offload_batch_host_async": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_lanes": (_i, [_vp, _i]),
     "gelo_set_lane_share": (_i, [_vp, _i]),
+    "gelo_set_wait_limit_ns": (_i, [_vp, ctypes.c_ulonglong]),
     "gelo_batch_workspace_bytes": (_sz, [_i, _i, _i, _i, _i, _i]),
     "gelo_profile_start": (_i, [_vp]),
     "gelo_profile_stop": (_i, [_vp, _vp, _vp]),
@@ -182,6 +183,10 @@ class Context:
 
     def set_lane_share(self, share: int):
         self._check(self._lib.gelo_set_lane_share(self._h, share), "gelo_set_lane_share")
+
+    def set_wait_limit_ns(self, ns: int):
+        """Limit of the device-side barrier waits of the tensor-core kernels (0: give up at once)."""
+        self._check(self._lib.gelo_set_wait_limit_ns(self._h, int(ns)), "gelo_set_wait_limit_ns")
 
     def ensure_batch_workspace(self, n, k, d, p, dtype, lanes=None):
         """Workspace for the batched entry points with `lanes` concurrent sampling lanes."""

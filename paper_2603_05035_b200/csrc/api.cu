@@ -235,6 +235,15 @@ int unmix_impl(gelo_ctx* ctx, const void* Ainv, int lda, const void* Yp, int n, 
     return product(ctx, g, t3, st);
 }
 
+// The single-stage entry points have no scratch of their own; when the context holds a workspace with room for the
+// operand pairs, their large fp32 products run on the tensor cores exactly as inside the whole call (so that a plain
+// H W through gelo_project is timed on the same kernel as the obfuscated chain).  Without one they stay on the FMA kernel.
+const Tf32x3Scratch* stage_pairs(gelo_ctx* ctx, int rows, int k, int d, int p, int dtype, Layout* L)
+{
+    if (dtype != GELO_F32 || !ctx->ws) return nullptr;
+    return carve_ctx(ctx, rows, k, d, p, dtype, false, L) ? &L->t3 : nullptr;
+}
+
 int check_split(int p, const void* Q, const void* K, const void* V)
 {
     if (!Q) return GELO_ERR_INVALID;
@@ -334,11 +343,20 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     // Back-to-back batches of the same shape on the same stream keep the lanes running across the seam: each
     // lane only waits until the products that read its previous pair are done.  Otherwise the lanes start after
     // everything already enqueued on the caller's stream.
+    const int shape[6] = { n, k, d, p, dtype, host ? 1 : 0 };
+    bool same_shape = true;
+    for (int i = 0; i < 6; ++i) same_shape = same_shape && ctx->chain_shape[i] == shape[i];
     const bool chained = ctx->chain_valid && ctx->chain_stream == st && ctx->chain_key == L[D - 1].G &&
-                         ctx->chain_lanes == D;
+                         ctx->chain_lanes == D && same_shape;
     if (!chained) {
+        // a fresh start: the lanes AND the two copy streams begin after everything already on the caller's stream
+        // (an earlier call of another shape may still be using the regions that this batch stages into)
         GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
         for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaStreamWaitEvent(ctx->lane_stream[l], ctx->batch_start, 0));
+        if (host) {
+            GELO_CUDA_OK(cudaStreamWaitEvent(ctx->copy_in, ctx->batch_start, 0));
+            GELO_CUDA_OK(cudaStreamWaitEvent(ctx->copy_out, ctx->batch_start, 0));
+        }
     }
 
     auto enqueue_sample = [&](int i) -> int {
@@ -405,6 +423,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     ctx->chain_stream = st;
     ctx->chain_key = L[D - 1].G;
     ctx->chain_lanes = D;
+    for (int i = 0; i < 6; ++i) ctx->chain_shape[i] = shape[i];
     if (host && wait) GELO_CUDA_OK(cudaStreamSynchronize(st));
     return GELO_OK;
 }
@@ -816,7 +835,8 @@ int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int
         !W_dev || !Yp_dev || misaligned(U_dev) || misaligned(W_dev) || misaligned(Yp_dev))
         return GELO_ERR_INVALID;
     DeviceGuard guard(ctx->device);
-    return project_impl(ctx, U_dev, W_dev, m, d, p, dtype, Yp_dev, as_stream(stream));
+    Layout L;
+    return project_impl(ctx, U_dev, W_dev, m, d, p, dtype, Yp_dev, as_stream(stream), stage_pairs(ctx, m, 0, d, p, dtype, &L));
 }
 
 int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev, int n, int k, int p, int dtype,
@@ -828,7 +848,9 @@ int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev,
         return GELO_ERR_INVALID;
     GELO_TRY(check_split(p, Q_dev, K_dev, V_dev));
     DeviceGuard guard(ctx->device);
-    return unmix_impl(ctx, Ainv_dev, lda, Yp_dev, n, k, p, dtype, Q_dev, K_dev, V_dev, as_stream(stream));
+    Layout L;
+    return unmix_impl(ctx, Ainv_dev, lda, Yp_dev, n, k, p, dtype, Q_dev, K_dev, V_dev, as_stream(stream),
+                      stage_pairs(ctx, n, k, 8, p, dtype, &L));
 }
 
 int gelo_qkv_offload(gelo_ctx* ctx, const void* H_dev, const void* W_dev, int n, int k, int d, int p, int kind,
@@ -1005,6 +1027,14 @@ int gelo_set_level3(gelo_ctx* ctx, int mode)
 {
     if (!ctx || mode < 0 || mode > 3) return GELO_ERR_INVALID;
     ctx->level3 = mode;
+    return GELO_OK;
+}
+
+int gelo_set_wait_limit_ns(gelo_ctx* ctx, unsigned long long ns)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    drop_graphs(ctx);              // the limit is a launch parameter of the recorded kernels
+    ctx->wait_limit_ns = ns;
     return GELO_OK;
 }
 

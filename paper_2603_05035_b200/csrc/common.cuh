@@ -58,6 +58,7 @@ struct gelo_ctx {
     int level3 = 0;               // 0: tf32 tensor-core updates for bf16 calls with m >= 256; 1: always fp32 FMA;
                                   // 2: always tensor cores, three bf16 products of split operands; 3: always tensor cores, tf32
     long long launches = 0;
+    unsigned long long wait_limit_ns = 2000000000ull;   // limit of every device-side barrier wait (gelo_set_wait_limit_ns)
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
     bool tma_3d = true;           // N-major operand tiles as one three-dimensional TMA box where the layout allows
     // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
@@ -72,6 +73,7 @@ struct gelo_ctx {
     cudaStream_t chain_stream = nullptr;
     const void* chain_key = nullptr;
     int chain_lanes = 0;
+    int chain_shape[6] = {0, 0, 0, 0, 0, 0};   // n, k, d, p, dtype, host staging of the batch a later one may chain onto
     // replayable launch graphs of the sampling sequence, one per (lane scratch, kind, size, type)
     struct SampleGraph { const void* key_ptr; int m, kind, dtype, level3, tc_ctas; cudaGraphExec_t exec; long long launches; };
     std::vector<SampleGraph> graphs;
@@ -251,7 +253,7 @@ struct CondScratch {
     float* scal = nullptr;    // 16 floats
 };
 CondScratch carve_cond(Arena&, int m);
-// cond_out[0] = estimate; status_dev[1] = (estimate * 1.1 <= bound)
+// cond_out[0] = estimate; status_dev[1] = (estimate * 1.2 <= bound)
 // A, Ainv: m x m matrices of type `dtype` with row stride ld (a multiple of 8)
 int run_cond_estimate(gelo_ctx*, int m, const void* A, const void* Ainv, int ld, int dtype, float bound,
                       float* cond_out, const CondScratch&, cudaStream_t, bool deferred = false);

@@ -21,15 +21,19 @@
 //   the tensor-memory allocation, warps 2-9 drain the accumulator (two warps per TMEM lane
 //   quarter, half of the columns each).  Two accumulator stages let the epilogue of one tile
 //   overlap the main loop of the next.
-// * Every wait on an mbarrier is bounded; on expiry the CTA records GELO_ERR_TIMEOUT in the
+// * Every wait on an mbarrier is bounded in time (the context's wait limit, two seconds by default,
+//   measured on the GPU's global timer); on expiry the CTA records GELO_ERR_TIMEOUT in the
 //   context's status word, stops issuing work, releases tensor memory and returns.
 #include <cuda.h>
 
 #include "common.cuh"
+#include "tc_ptx.cuh"
 
 namespace gelo {
 
 namespace {
+
+using namespace tcx;
 
 constexpr int BM = 128;
 constexpr int BK = 64;
@@ -38,7 +42,6 @@ constexpr int kEpiWarps = 8;
 constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kABytes = BM * BK * 2;            // 16 KiB
 constexpr uint32_t kTmemCols = 512;
-constexpr unsigned long long kWaitLimit = 40ull * 1000 * 1000;   // try_wait rounds before giving up
 
 enum TcMode { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_SUB_F32 = 2, TC_EMIT_SPLIT = 3 };
 
@@ -60,123 +63,9 @@ struct TcParams {
     int a3d, b3d;                   // the MN-major A tile / the B tile arrives as ONE three-dimensional box (see make_map_nmajor)
     int out_f16;                    // TC_STORE_BF16: operands and output are IEEE half instead of bfloat16
     uint32_t idesc;                 // instruction descriptor (filled in by the launcher)
+    unsigned long long wait_ns;     // limit of every mbarrier wait, nanoseconds (filled in by the launcher from the context)
     int* status;
 };
-
-// ---- PTX wrappers -----------------------------------------------------------------------
-
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint32_t bar)
-{
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait: false when the limit ran out or another thread already gave up.
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag)
-{
-    for (unsigned long long spin = 0; spin < kWaitLimit; ++spin) {
-        if (mbar_try(bar, parity)) return true;
-        if ((spin & 1023) == 1023 && *abort_flag) return false;
-    }
-    return false;
-}
-
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z, uint32_t bar)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
-        ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                            uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ void tc_mma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc,
-                                            uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-
-__device__ __forceinline__ float round_tf32(float x)
-{
-    uint32_t r;
-    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
-    return __uint_as_float(r);
-}
-
-__device__ __forceinline__ void tc_ld_32cols(uint32_t taddr, uint32_t v[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tc_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor (sm_100 format): start address, leading and stride byte
-// offsets in 16-byte units, descriptor version 1, 128-byte swizzle.
-// Layout type 2: 128-byte swizzle of 16-byte chunks (8-row atoms).  Layout type 1: 128-byte swizzle of 32-byte
-// chunks (4-row atoms), the only layout that 32-bit operands may use when they are not K-major.
-__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes, uint32_t layout = 2)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((addr >> 4) & 0x3FFF);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
-    d |= (uint64_t)1 << 46;       // version
-    d |= (uint64_t)layout << 61;
-    return d;
-}
-
 
 // Epilogue staging for the in-place subtraction: every epilogue warp owns two 32 x 32 fp32 boxes (4 KiB each)
 // that TMA reduces into global memory.
@@ -210,16 +99,6 @@ struct TcCfg {
     static_assert(!kAMn || kTf32, "MN-major A is only wired up for the tf32 kind");
 };
 
-__device__ __forceinline__ uint32_t pack_bf16(uint32_t a, uint32_t b)
-{
-    __nv_bfloat162 h = __floats2bfloat162_rn(__uint_as_float(a), __uint_as_float(b));
-    return *reinterpret_cast<uint32_t*>(&h);
-}
-__device__ __forceinline__ uint32_t pack_f16(uint32_t a, uint32_t b)
-{
-    __half2 h = __floats2half2_rn(__uint_as_float(a), __uint_as_float(b));
-    return *reinterpret_cast<uint32_t*>(&h);
-}
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi)
 __device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t& lo)
 {
@@ -341,7 +220,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     for (int kb = kb_lo; kb < kb_hi; ++kb, ++it) {
                         const int s = it % kStages;
                         const uint32_t ph = (it / kStages) & 1u;
-                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag)) { ok = false; break; }
+                        if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, prm.wait_ns)) { ok = false; break; }
                         const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                         const uint32_t sb = sa + kABytes;
                         mbar_expect_tx(full_bar(s), Cfg::kStageBytes);
@@ -385,13 +264,13 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     }
                 const int a = acc_it % kAccStages;
                 const uint32_t aph = (acc_it / kAccStages) & 1u;
-                if (!mbar_wait(acc_empty_bar(a), aph ^ 1u, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(acc_empty_bar(a), aph ^ 1u, abort_flag, prm.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(a * BN);
                 for (int kb = 0; kb < kb_total; ++kb, ++it) {
                     const int s = it % kStages;
                     const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(full_bar(s), ph, abort_flag, prm.wait_ns)) { ok = false; break; }
                     tc_fence_after();
                     const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                     const uint32_t sb = sa + kABytes;
@@ -430,7 +309,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             if (kStaging && prm.mode == TC_SUB_F32) {
                 // C -= acc without reading C: the negated accumulator goes through a swizzled shared-memory box and
                 // a TMA reduce-add into global memory (the addition happens at the L2); TMA clips at the matrix edge
-                if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(acc_full_bar(a), aph, abort_flag, prm.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
                 const uint32_t my_staging = staging_base + (uint32_t)(warp - 2) * 2u * kStageBoxBytes;
@@ -459,7 +338,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     if (lane == 0) asm volatile("cp.async.bulk.commit_group;" ::: "memory");
                 }
             } else {
-                if (!mbar_wait(acc_full_bar(a), aph, abort_flag)) { ok = false; break; }
+                if (!mbar_wait(acc_full_bar(a), aph, abort_flag, prm.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(a * BN);
 #pragma unroll 1
@@ -572,6 +451,7 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
     if (p.mode != TC_STORE_BF16 && ctx->tc_update_ctas > 0 && grid > ctx->tc_update_ctas) grid = ctx->tc_update_ctas;
     TcParams q = p;
     // both operands of a kind::f16 instruction have the same 16-bit format: 1 = bfloat16, 0 = IEEE half
+    q.wait_ns = ctx->wait_limit_ns;
     q.idesc = (!kTf32 && p.out_f16) ? (Cfg::kInstrDesc & ~((7u << 7) | (7u << 10))) : Cfg::kInstrDesc;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);

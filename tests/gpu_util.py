@@ -23,14 +23,17 @@ def padded(m, ld, dtype):
     return torch.full((m, ld), float("nan"), device="cuda", dtype=dtype)
 
 
-def sample_rows(n, count, seed, extra=()):
-    """Row subset for sampled parity: first, last, tile edges, and random rows."""
+def sample_rows(n, count, seed, extra=(), tile=128):
+    """Row subset for sampled parity: first, last, both sides of every tile edge (so every `tile`-row tile of the
+    output contributes at least two rows), the rows named in `extra`, and random rows up to `count` (the edge rows are
+    kept even where they exceed it)."""
     rng = np.random.default_rng(seed)
     rows = {0, n - 1, *[r for r in extra if 0 <= r < n]}
-    for edge in range(128, n, 128):
+    for edge in range(tile, n, tile):
         rows.update((edge - 1, edge))
-        if len(rows) >= count // 2:
-            break
+    for t0 in range(0, n, tile):                       # a last, short tile still gets two rows
+        t1 = min(n, t0 + tile)
+        rows.update((t0, t1 - 1))
     while len(rows) < min(count, n):
         rows.add(int(rng.integers(0, n)))
     return np.array(sorted(rows), dtype=np.int64)

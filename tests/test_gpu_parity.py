@@ -260,6 +260,38 @@ def test_products_stage_parity(ctx, oracle, n, k, d, p, dt):
     assert oracle.rel_fro(y, oracle.direct(f64(H), f64(W))) <= TOL[dt]
 
 
+def test_mix_full_size_seam_inside_a_k_block(ctx, oracle):
+    """The mixing product alone at full size with the H / S seam in the middle of a 64-row k-block (n = 4000 is 32
+    past a multiple of 64), the operand pipeline at full depth: sampled rows of U against the oracle's product."""
+    n, k, d = 4000, 200, 4096
+    m = n + k
+    ld = ctx.mixing_ld(m)
+    g = torch.Generator(device="cuda"); g.manual_seed(77)
+    A = padded(m, ld, torch.bfloat16)
+    A[:, :m] = (torch.randn((m, m), device="cuda", generator=g) / np.sqrt(m)).to(torch.bfloat16)
+    H = inputs.make_hidden(n, d, "bf16", 78, True, "cuda")
+    S = (10.0 * torch.randn((k, d), device="cuda", generator=g)).to(torch.bfloat16)
+    U = torch.full((m, d), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ctx.mix(A, ld, H, S, n, k, d, "bf16", U)
+    torch.cuda.synchronize()
+    assert torch.isfinite(U).all()
+    rows = sample_rows(m, 64, seed=5, extra=(n - 1, n, n + 1))
+    ref = oracle.matmul(f64(A[rows][:, :m]), np.vstack([f64(H), f64(S)]))
+    u = f64(U[rows])
+    assert oracle.rel_fro(u, ref) <= 4e-3                  # one bf16 rounding of the output
+    assert np.max(np.abs(u - ref)) <= 8 * 4e-3 * np.sqrt(np.mean(ref * ref))
+    # a seam that is not even a multiple of 8 rows (the second segment then starts at the 16-byte boundary below it)
+    n2 = 3997
+    U2 = torch.full((n2 + k, d), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ld2 = ctx.mixing_ld(n2 + k)
+    A2 = padded(n2 + k, ld2, torch.bfloat16); A2[:, :n2 + k] = A[:n2 + k, :n2 + k]
+    ctx.mix(A2, ld2, H[:n2].contiguous(), S, n2, k, d, "bf16", U2)
+    torch.cuda.synchronize()
+    rows2 = np.array([0, 1, 127, 128, 2047, 2048, n2 - 1, n2, n2 + 1, n2 + k - 1], dtype=np.int64)
+    ref2 = oracle.matmul(f64(A2[rows2][:, :n2 + k]), np.vstack([f64(H[:n2]), f64(S)]))
+    assert oracle.rel_fro(f64(U2[rows2]), ref2) <= 4e-3
+
+
 # ------------------------------------------------------------------------- whole call
 
 def _run_offload(ctx, w, call, host=False):
@@ -296,9 +328,11 @@ def test_offload_full_size_sampled_rows(ctx, oracle, name, calls):
     for call in calls:
         H, W, y = _run_offload(ctx, w, call)
         assert np.isfinite(y).all()
-        rows = sample_rows(w.n, 96, seed=call)
+        rows = sample_rows(w.n, 96, seed=call, extra=(w.n - w.k - 1, w.n - w.k))
         ref = oracle.rows_times_w(f64(H), f64(W), rows)
         assert oracle.rel_fro(y[rows], ref) <= TOL[w.dtype]
+        # no single entry far off either: an error at the tolerance has an rms of TOL * rms(ref) per entry
+        assert np.max(np.abs(y[rows] - ref)) <= 8 * TOL[w.dtype] * np.sqrt(np.mean(ref * ref))
         # property that holds at any size: column sums of Y equal (1^T H) W
         colsum_ref = (f64(H).sum(axis=0)[None, :] @ f64(W)).ravel()
         scale = np.linalg.norm(y, axis=0).mean() * np.sqrt(w.n)
@@ -422,8 +456,10 @@ def test_batched_offload_full_size(oracle):
     assert c.last_status() == binding.OK
     for i in (0, 7, 19):
         y = np.hstack([f64(outs[0][i]), f64(outs[1][i]), f64(outs[2][i])])
-        rows = sample_rows(n, 48, seed=i)
-        assert oracle.rel_fro(y[rows], oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)) <= TOL["bf16"]
+        rows = sample_rows(n, 48, seed=i, extra=(n - k - 1, n - k))
+        ref = oracle.rows_times_w(f64(Hs[i]), f64(Ws[i]), rows)
+        assert oracle.rel_fro(y[rows], ref) <= TOL["bf16"]
+        assert np.max(np.abs(y[rows] - ref)) <= 8 * TOL["bf16"] * np.sqrt(np.mean(ref * ref))
     c.close()
 
 
@@ -587,6 +623,26 @@ def test_output_projection_unsplit(ctx, oracle, dt, kind):
     assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= TOL[dt]
 
 
+@pytest.mark.parametrize("p,kind", [(4096, ORTHOGONAL), (11008, NONORTHOGONAL)])
+def test_unsplit_projections_full_size(ctx, oracle, p, kind):
+    """The attention output projection (p = d) and an MLP up-projection (p = 11008, not a multiple of the 256-column
+    tiles) at n = 4096, d = 4096 with 204 shield rows: sampled rows against the oracle's H W."""
+    n, k, d = 4096, 204, 4096
+    ctx.ensure_workspace(n, k, d, p, "bf16")
+    H = inputs.make_hidden(n, d, "bf16", 51, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 51, "cuda")
+    Y = torch.full((n, p), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ctx.qkv_offload(H, W, n, k, d, p, kind, 5151, 10.0, "bf16", Y)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == binding.OK
+    assert torch.isfinite(Y).all()
+    rows = sample_rows(n, 64, seed=p)
+    ref = oracle.rows_times_w(f64(H), f64(W), rows)
+    y = f64(Y[rows])
+    assert oracle.rel_fro(y, ref) <= TOL["bf16"]
+    assert np.max(np.abs(y - ref)) <= 8 * TOL["bf16"] * np.sqrt(np.mean(ref * ref))
+
+
 # ------------------------------------------------------------------------- block-diagonal variant
 
 @pytest.mark.parametrize("dt,n,k,d,block,split", [("bf16", 1024, 52, 512, 256, True), ("f32", 300, 20, 256, 128, True),
@@ -730,3 +786,70 @@ def test_profile_counts_launches(ctx):
     assert prof["gemm_tc"]["launches"] == 3 and prof["gemm_tc"]["ms"] > 0          # mix, project, unmix
     assert prof["qr_panel"]["launches"] == 3                                        # m = 68: three 32-column panels
     assert prof["gemm_tc"]["work"] == pytest.approx(2.0 * (68 * 68 * 4096 + 68 * 4096 * 12288 + 64 * 68 * 12288))
+
+
+# ------------------------------------------------------------------------- bounded waits
+
+def test_zero_wait_limit_reports_timeout_and_context_stays_usable(oracle):
+    """With a wait limit of zero every tensor-core CTA gives up before it issues a copy or an MMA (nothing is in flight
+    when it returns); the status word then says TIMEOUT, and after the limit is restored the same call is correct."""
+    c = binding.Context(0)
+    n, d, p = 128, 256, 768
+    H = inputs.make_hidden(n, d, "bf16", 3, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 3, "cuda")
+    Y = torch.full((n, p), float("nan"), device="cuda", dtype=torch.bfloat16)
+    c.set_wait_limit_ns(0)
+    c.project(H, W, n, d, p, "bf16", Y)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.ERR_TIMEOUT
+    assert torch.isnan(Y).all()                            # nothing was computed, nothing was written
+    assert c.last_status() == binding.OK                   # reading the status cleared it
+    c.set_wait_limit_ns(2_000_000_000)
+    c.project(H, W, n, d, p, "bf16", Y)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    assert oracle.rel_fro(f64(Y), oracle.direct(f64(H), f64(W))) <= 4e-3
+    c.close()
+
+
+# ------------------------------------------------------------------------- ordering of the host variants
+
+def test_async_host_batches_of_different_shapes_back_to_back(oracle):
+    """Two enqueue-only host batches of different shapes on one lane (so that both stage into the same workspace
+    region), and a device call before a host batch, with no synchronisation in between: the copy streams of the
+    later call must wait for the earlier call's kernels.  Results against the device-resident variant, bytewise."""
+    c = binding.Context(0)
+    c.set_lanes(1)
+    shapes = [(192, 8, 256), (128, 4, 512)]
+    need = max(int(c._lib.gelo_batch_workspace_bytes(n, k, d, 3 * d, BF16, 1)) for n, k, d in shapes)
+    c.set_workspace(torch.empty(need, dtype=torch.uint8, device="cuda"))
+    calls = 3
+    data = []
+    for (n, k, d) in shapes:
+        p = 3 * d
+        Hs = [inputs.make_hidden(n, d, "bf16", 60 + i, True, "cuda") for i in range(calls)]
+        Ws = [inputs.make_weight(d, p, "bf16", 60 + i, "cuda") for i in range(calls)]
+        Hh = [h.cpu().pin_memory() for h in Hs]
+        out_h = [[torch.zeros((n, d), dtype=torch.bfloat16).pin_memory() for _ in range(calls)] for _ in range(3)]
+        out_d = [[torch.empty((n, d), device="cuda", dtype=torch.bfloat16) for _ in range(calls)] for _ in range(3)]
+        data.append((n, k, d, p, Hs, Ws, Hh, out_h, out_d))
+    kinds = [ORTHOGONAL, NONORTHOGONAL, ORTHOGONAL]
+    seeds = [900, 901, 902]
+    for rep in range(3):                                   # several rounds: the race, if any, is a matter of timing
+        # a single device call first (it uses the same workspace), then the two host batches, no sync in between
+        n0, k0, d0, p0, Hs0, Ws0, _, _, out_d0 = data[0]
+        c.qkv_offload(Hs0[0], Ws0[0], n0, k0, d0, p0, NONORTHOGONAL, 77, 10.0, "bf16", out_d0[0][0], out_d0[1][0], out_d0[2][0])
+        for (n, k, d, p, Hs, Ws, Hh, out_h, out_d) in data:
+            c.qkv_offload_batch_host_async(Hh, Ws, n, k, d, p, kinds, seeds, 10.0, "bf16", *out_h)
+        torch.cuda.synchronize()
+        assert c.last_status() == binding.OK
+        for (n, k, d, p, Hs, Ws, Hh, out_h, out_d) in data:
+            c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, 10.0, "bf16", *out_d)
+            torch.cuda.synchronize()
+            for j in range(3):
+                for i in range(calls):
+                    assert torch.equal(out_h[j][i], out_d[j][i].cpu()), (rep, n, j, i)
+                    out_h[j][i].zero_()
+    y = np.hstack([f64(data[1][8][j][1]) for j in range(3)])
+    assert oracle.rel_fro(y, oracle.direct(f64(data[1][4][1]), f64(data[1][5][1]))) <= TOL["bf16"]
+    c.close()
