@@ -560,6 +560,9 @@ def measure_workload(name, lanes, steps, warmup, calls=0, latency_steps=0):
     timed("mix", lambda r: ctx.mix(A, lda, Hs[r % calls], S if k else None, n, k, d, w.dtype, U), 16)
     timed("project", lambda r: ctx.project(U, Ws[r % calls], m, d, p, w.dtype, Yp), 32)
     timed("unmix", lambda r: ctx.unmix(X, lda, Yp, n, k, p, w.dtype, Q, K, V), 16)
+    if m <= 128 and w.dtype != "f32" and p % 32 == 0:
+        # small batches run Eq. 2 and Eq. 3 as one kernel inside the whole call
+        timed("project_unmix", lambda r: ctx.project_unmix(U, Ws[r % calls], X, lda, n, k, d, p, w.dtype, Q, K, V), 32)
     # the plain, unprotected projection through the same entry point, hence on the same kernel as the chain's products
     timed("plain_project", lambda r: ctx.project(Hs[r % calls], Ws[r % calls], n, d, p, w.dtype, Yp), 32)
     if w.dtype == "f32":

@@ -55,6 +55,8 @@ EXPORTS = {
     "gelo_project": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_unmix": (_i, [_vp, _vp, _i, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
+    "gelo_project_unmix": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "gelo_set_small_batch_fusion": (_i, [_vp, _i]),
     "gelo_qkv_offload_batch": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_qkv_offload_batch_host": (_i, [_vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_blockdiag_workspace_bytes": (ctypes.c_size_t, [_i, _i, _i, _i, _i, _i, _i]),
@@ -278,6 +280,14 @@ class Context:
     def unmix(self, Ainv, lda, Yp, n, k, p, dtype, Q, K=None, V=None, stream=None):
         self._check(self._lib.gelo_unmix(self._h, _ptr(Ainv), lda, _ptr(Yp), n, k, p, dtype_code(dtype),
                                          _ptr(Q), _ptr(K), _ptr(V), _stream(stream)), "gelo_unmix")
+
+    def project_unmix(self, U, W, Ainv, lda, n, k, d, p, dtype, Q, K=None, V=None, stream=None):
+        """Projection and unmixing of a small batch (n + k <= 128) in one kernel."""
+        self._check(self._lib.gelo_project_unmix(self._h, _ptr(U), _ptr(W), _ptr(Ainv), lda, n, k, d, p, dtype_code(dtype),
+                                                 _ptr(Q), _ptr(K), _ptr(V), _stream(stream)), "gelo_project_unmix")
+
+    def set_small_batch_fusion(self, on: bool):
+        self._check(self._lib.gelo_set_small_batch_fusion(self._h, 1 if on else 0), "gelo_set_small_batch_fusion")
 
     def qkv_offload(self, H, W, n, k, d, p, kind, seed, shield_scale, dtype, Q, K=None, V=None, stream=None):
         self._check(self._lib.gelo_qkv_offload(self._h, _ptr(H), _ptr(W), n, k, d, p, kind, seed, shield_scale,

@@ -204,6 +204,8 @@ int product(gelo_ctx* ctx, const GemmArgs& g, const Tf32x3Scratch* t3, cudaStrea
 int mix_impl(gelo_ctx* ctx, const void* A, int lda, const void* H, const void* S, int n, int k, int d,
              int dtype, void* U, cudaStream_t st, const Tf32x3Scratch* t3 = nullptr)
 {
+    if (ctx->fuse_small && mix_small_supports(n, k, d, dtype) && !misaligned(H) && !misaligned(S) && !misaligned(U))
+        return launch_mix_small(ctx, A, lda, H, S, n, k, d, dtype, U, st);
     GemmArgs g;
     g.M = n + k; g.N = d; g.K = n + k;
     g.A = A; g.lda = lda;
@@ -244,6 +246,17 @@ const Tf32x3Scratch* stage_pairs(gelo_ctx* ctx, int rows, int k, int d, int p, i
     return carve_ctx(ctx, rows, k, d, p, dtype, false, L) ? &L->t3 : nullptr;
 }
 
+// Eq. 2 and Eq. 3 of one call: one fused launch for a small batch (the weight is streamed once and Y' stays on chip),
+// otherwise the two products with Y' in workspace memory.
+int project_and_unmix(gelo_ctx* ctx, const void* U, const void* W, const void* Ainv, int lda, void* Yp, int n, int k, int d,
+                      int p, int dtype, void* Q, void* K, void* V, cudaStream_t st, const Tf32x3Scratch* t3)
+{
+    if (ctx->fuse_small && project_unmix_supports(ctx, n, k, d, p, dtype, lda, (K || V) ? 3 : 1))
+        return launch_project_unmix(ctx, U, W, Ainv, lda, n, k, d, p, dtype, Q, K, V, st);
+    GELO_TRY(project_impl(ctx, U, W, n + k, d, p, dtype, Yp, st, t3));
+    return unmix_impl(ctx, Ainv, lda, Yp, n, k, p, dtype, Q, K, V, st, t3);
+}
+
 int check_split(int p, const void* Q, const void* K, const void* V)
 {
     if (!Q) return GELO_ERR_INVALID;
@@ -260,8 +273,7 @@ int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, i
     GELO_TRY(sample_mixing_impl(ctx, L, m, kind, seed, dtype, L.A, L.Ainv, L.ldi, nullptr, st));
     GELO_TRY(run_shield_rows(ctx, H, n, d, k, shield_scale, seed, dtype, L.S, L.sh, st));
     GELO_TRY(mix_impl(ctx, L.A, L.ldi, H, k > 0 ? L.S : nullptr, n, k, d, dtype, L.U, st, &L.t3));
-    GELO_TRY(project_impl(ctx, L.U, W, m, d, p, dtype, L.Yp, st, &L.t3));
-    return unmix_impl(ctx, L.Ainv, L.ldi, L.Yp, n, k, p, dtype, Q, K, V, st, &L.t3);
+    return project_and_unmix(ctx, L.U, W, L.Ainv, L.ldi, L.Yp, n, k, d, p, dtype, Q, K, V, st, &L.t3);
 }
 
 
@@ -396,8 +408,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
         if (host) GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[b], 0));
         GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st, &L[0].t3));
-        GELO_TRY(project_impl(ctx, L[0].U, W[i], m, d, p, dtype, L[0].Yp, st, &L[0].t3));
-        GELO_TRY(unmix_impl(ctx, L[l].Ainv, L[l].ldi, L[0].Yp, n, k, p, dtype, Qi, Ki, Vi, st, &L[0].t3));
+        GELO_TRY(project_and_unmix(ctx, L[0].U, W[i], L[l].Ainv, L[l].ldi, L[0].Yp, n, k, d, p, dtype, Qi, Ki, Vi, st, &L[0].t3));
         GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
         if (host) {
             GELO_CUDA_OK(cudaEventRecord(ctx->h_free[b], st));
@@ -851,6 +862,25 @@ int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev,
     Layout L;
     return unmix_impl(ctx, Ainv_dev, lda, Yp_dev, n, k, p, dtype, Q_dev, K_dev, V_dev, as_stream(stream),
                       stage_pairs(ctx, n, k, 8, p, dtype, &L));
+}
+
+int gelo_project_unmix(gelo_ctx* ctx, const void* U_dev, const void* W_dev, const void* Ainv_dev, int lda, int n, int k,
+                       int d, int p, int dtype, void* Q_dev, void* K_dev, void* V_dev, void* stream)
+{
+    if (!ctx || n <= 0 || k < 0 || d <= 0 || p <= 0 || (d % 8) != 0 || (p % 8) != 0 || bad_dtype(dtype) || !U_dev || !W_dev ||
+        !Ainv_dev || bad_ld(lda, n + k) || misaligned(U_dev) || misaligned(W_dev) || misaligned(Ainv_dev) || misaligned(Q_dev) ||
+        misaligned(K_dev) || misaligned(V_dev))
+        return GELO_ERR_INVALID;
+    GELO_TRY(check_split(p, Q_dev, K_dev, V_dev));
+    DeviceGuard guard(ctx->device);
+    return launch_project_unmix(ctx, U_dev, W_dev, Ainv_dev, lda, n, k, d, p, dtype, Q_dev, K_dev, V_dev, as_stream(stream));
+}
+
+int gelo_set_small_batch_fusion(gelo_ctx* ctx, int on)
+{
+    if (!ctx) return GELO_ERR_INVALID;
+    ctx->fuse_small = on != 0;
+    return GELO_OK;
 }
 
 int gelo_qkv_offload(gelo_ctx* ctx, const void* H_dev, const void* W_dev, int n, int k, int d, int p, int kind,

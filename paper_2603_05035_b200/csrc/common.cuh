@@ -60,6 +60,8 @@ struct gelo_ctx {
     long long launches = 0;
     unsigned long long wait_limit_ns = 2000000000ull;   // limit of every device-side barrier wait (gelo_set_wait_limit_ns)
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
+    bool fuse_small = true;       // calls with m <= 128 run projection and unmixing as one kernel (gelo_set_small_batch_fusion)
+    int dec_group = 16;           // CTAs of the small-batch projection kernel that walk the k-blocks in step (0: all of them)
     bool tma_3d = true;           // N-major operand tiles as one three-dimensional TMA box where the layout allows
     // lanes of the batched entry points: each samples the mixing pair of one call on its own stream
     int lanes = 4;
@@ -168,6 +170,12 @@ int launch_gemm_tc_split_k(gelo_ctx*, int M, int N, int K, const void* Ahi, cons
 int launch_gemm_tf32(gelo_ctx*, int M, int N, int K, const float* A, int lda, bool a_mn, const float* B, int ldb,
                      bool subtract, float* C, int ldc, bool round_out, float out_scale, int ksplit, size_t plane, int* used,
                      cudaStream_t, float diag_sub = 0.0f, float post_scale = 1.0f);
+// D (m x m bf16) = post_scale * (out_scale * Q^T Q - diag_sub I): tf32 product over the tiles on and above the diagonal only
+int launch_gram_sym_bf16(gelo_ctx*, int m, const float* Q, int ld, void* D, int ldd, float out_scale, float diag_sub,
+                         float post_scale, cudaStream_t);
+// C (fp32) -= A (bf16) B (bf16), in place
+int launch_gemm_bf16_sub(gelo_ctx*, int M, int N, int K, const void* A, int lda, const void* B, int ldb, float* C, int ldc,
+                         cudaStream_t);
 // The tensor core drops the 13 low mantissa bits of an fp32 operand instead of rounding them.  For values whose
 // mantissas are spread log-uniformly that loses 2^-11 / (2 ln 2) of the magnitude on average, coherently over all
 // terms of a product; a result whose operand was truncated is scaled back by 1 + kTf32TruncLoss per such operand,
@@ -198,6 +206,20 @@ struct Tf32x3Scratch {
     float* planes = nullptr;              // kTf32x3Slices partial products of at most c_elems floats each
     size_t a_elems = 0, b_elems = 0, c_elems = 0;
 };
+
+// ---- projection and unmixing of a small batch in one kernel (decode.cu) ---------------------------------
+
+// true when launch_project_unmix can serve the call: 16-bit storage, m = n + k <= 128, p a multiple of 32 whose
+// 32-column boxes leave every CTA a slab of at most 128 columns
+bool project_unmix_supports(const gelo_ctx*, int n, int k, int d, int p, int dtype, int lda, int nsplit);
+// Q | K | V (or one n x p result in Q when K = V = nullptr) = (Ainv[0:n, 0:n+k] (U W)); U: (n+k) x d, W: d x p
+int launch_project_unmix(gelo_ctx*, const void* U, const void* W, const void* Ainv, int lda, int n, int k, int d, int p,
+                         int dtype, void* Q, void* K, void* V, cudaStream_t);
+
+// U = A [H; S] for n + k <= 128 rows of a 16-bit type on the FMA pipes (one light launch instead of a tensor-core one)
+bool mix_small_supports(int n, int k, int d, int dtype);
+int launch_mix_small(gelo_ctx*, const void* A, int lda, const void* H, const void* S, int n, int k, int d, int dtype, void* U,
+                     cudaStream_t);
 
 // ---- factorizations -------------------------------------------------------------------
 

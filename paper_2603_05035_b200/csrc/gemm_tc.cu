@@ -43,7 +43,7 @@ constexpr int kThreads = 64 + 32 * kEpiWarps;
 constexpr uint32_t kABytes = BM * BK * 2;            // 16 KiB
 constexpr uint32_t kTmemCols = 512;
 
-enum TcMode { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_SUB_F32 = 2, TC_EMIT_SPLIT = 3 };
+enum TcMode { TC_STORE_BF16 = 0, TC_STORE_F32 = 1, TC_SUB_F32 = 2, TC_EMIT_SPLIT = 3, TC_STORE_SYM16 = 4 };
 
 struct TcSegment { int a_sel, b_sel, a_k0, b_row0, kb; };
 
@@ -62,6 +62,8 @@ struct TcParams {
     float post_scale;               //   ... and the factor applied after that: out = post_scale * (out_scale * acc - diag_sub [row == col])
     int a3d, b3d;                   // the MN-major A tile / the B tile arrives as ONE three-dimensional box (see make_map_nmajor)
     int out_f16;                    // TC_STORE_BF16: operands and output are IEEE half instead of bfloat16
+    int tri, tri_tiles;             // TC_STORE_SYM16: the result is symmetric; only the tri_tiles tiles that reach the diagonal or lie
+                                    // above it are computed, and what lies below them is filled in by mirroring
     uint32_t idesc;                 // instruction descriptor (filled in by the launcher)
     unsigned long long wait_ns;     // limit of every mbarrier wait, nanoseconds (filled in by the launcher from the context)
     int* status;
@@ -109,6 +111,28 @@ __device__ __forceinline__ void split2(float a, float b, uint32_t& hi, uint32_t&
     lo = *reinterpret_cast<const uint32_t*>(&l);
 }
 
+// Row-tile and column-tile index of work item `tile`.  Ordinary products: row tiles fastest, then column tiles, then K
+// slices.  Symmetric products (prm.tri, 128 x 256 tiles): column tile nt owns the row tiles mt <= 2 nt + 1, i.e. those
+// whose first row is not below the tile's last column; they are enumerated column tile after column tile.
+__device__ __forceinline__ void tile_coords(const TcParams& prm, int tile, int m_tiles, int mn_tiles, int& mt, int& nt, int& slice)
+{
+    if (prm.tri) {
+        int t = tile;
+        nt = 0;
+        for (;;) {
+            const int cnt = min(m_tiles, 2 * nt + 2);
+            if (t < cnt) break;
+            t -= cnt; ++nt;
+        }
+        mt = t; slice = 0;
+        return;
+    }
+    const int mn = tile % mn_tiles;
+    slice = tile / mn_tiles;
+    mt = mn % m_tiles;
+    nt = mn / m_tiles;
+}
+
 // One 8-column group of the epilogue: w[G*8 .. G*8+7] are the fp32 accumulator values of row gm, columns
 // gn..gn+7 (G is a template parameter so that the register array is indexed by constants only).
 template <int G>
@@ -153,6 +177,29 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
     }
 }
 
+// Symmetric result (TC_STORE_SYM16): 32 consecutive entries of row gm from column gn on, as
+// post_scale * (out_scale * acc - diag_sub [on the diagonal]) in bf16.  Entries above the diagonal whose mirror image
+// lies in a tile that is not computed (see tile_coords) are also written there; consecutive lanes hold consecutive
+// rows, so those transposed stores are contiguous across the warp.
+__device__ __forceinline__ void store_symmetric(const TcParams& prm, int gm, int gn, const uint32_t (&v)[32])
+{
+    __nv_bfloat16* D = static_cast<__nv_bfloat16*>(prm.C0);
+    __align__(16) __nv_bfloat16 h[32];
+#pragma unroll
+    for (int j = 0; j < 32; ++j)
+        h[j] = __float2bfloat16_rn(prm.post_scale * (prm.out_scale * __uint_as_float(v[j]) - ((gm == gn + j) ? prm.diag_sub : 0.0f)));
+#pragma unroll
+    for (int g = 0; g < 4; ++g)
+        if (gn + 8 * g < prm.N)
+            *reinterpret_cast<uint4*>(D + (size_t)gm * prm.ldc + gn + 8 * g) = *reinterpret_cast<const uint4*>(&h[8 * g]);
+    const int my_pair = gm >> 8;                              // column tile of the mirrored entry
+#pragma unroll
+    for (int j = 0; j < 32; ++j) {
+        const int c = gn + j;
+        if (c > gm && c < prm.M && (c >> 7) > 2 * my_pair + 1) D[(size_t)c * prm.ldc + gm] = h[j];
+    }
+}
+
 template <int BN, int kStages, bool kStaging, bool kTf32, bool kAMn>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
@@ -181,7 +228,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     const int m_tiles = (prm.M + BM - 1) / BM;
     const int n_tiles = (prm.N + BN - 1) / BN;
     const int mn_tiles = m_tiles * n_tiles;
-    const int total_tiles = mn_tiles * prm.ksplit;
+    const int total_tiles = prm.tri ? prm.tri_tiles : mn_tiles * prm.ksplit;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < kStages; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
@@ -206,9 +253,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             uint32_t it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x) {
-                const int mn = tile % mn_tiles, slice = tile / mn_tiles;
-                const int m0 = (mn % m_tiles) * BM;
-                const int n0 = (mn / m_tiles) * BN;
+                int mt, nt, slice;
+                tile_coords(prm, tile, m_tiles, mn_tiles, mt, nt, slice);
+                const int m0 = mt * BM, n0 = nt * BN;
 #pragma unroll
                 for (int sg = 0; sg < 3; ++sg) {              // constant indices keep the parameters out of local memory
                     if (sg >= prm.nseg || !ok) break;
@@ -253,7 +300,7 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
             uint32_t it = 0, acc_it = 0;
             bool ok = true;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
-                const int slice = tile / mn_tiles;
+                const int slice = prm.tri ? 0 : tile / mn_tiles;
                 int kb_total = 0;
 #pragma unroll
                 for (int sg = 0; sg < 3; ++sg)
@@ -301,9 +348,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
         for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
             const int a = acc_it % kAccStages;
             const uint32_t aph = (acc_it / kAccStages) & 1u;
-            const int mn = tile % mn_tiles, slice = tile / mn_tiles;
-            const int m0 = (mn % m_tiles) * BM;
-            const int n0 = (mn / m_tiles) * BN;
+            int mt, nt, slice;
+            tile_coords(prm, tile, m_tiles, mn_tiles, mt, nt, slice);
+            const int m0 = mt * BM, n0 = nt * BN;
             const int gm = m0 + quarter * 32 + lane;
             const bool row_ok = gm < prm.M;
             if (kStaging && prm.mode == TC_SUB_F32) {
@@ -346,7 +393,9 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     uint32_t v[32];
                     tc_ld_32cols(taddr + c, v);
                     tc_ld_wait();
-                    if (row_ok) {
+                    if (prm.mode == TC_STORE_SYM16) {
+                        if (row_ok) store_symmetric(prm, gm, n0 + c, v);
+                    } else if (row_ok) {
                         const int gn = n0 + c;
                         if (gn < prm.N) epilogue_group<0>(prm, gm, gn, v, slice);
                         if (gn + 8 < prm.N) epilogue_group<1>(prm, gm, gn + 8, v, slice);
@@ -670,6 +719,66 @@ int launch_gemm_tf32(gelo_ctx* ctx, int M, int N, int K, const float* A, int lda
     if (used) *used = p.ksplit;
     return a_mn ? launch_tiles<256, 4, false, true, true>(ctx, ma, ma, mb, mb, mc, p, flops, st)
                 : launch_tiles<256, 4, false, true, false>(ctx, ma, ma, mb, mb, mc, p, flops, st);
+}
+
+// D (m x m bf16, stride ldd) = post_scale * (out_scale * Q^T Q - diag_sub I) for a row-major fp32 Q (stride ld): one
+// tf32 product in which only the tiles on and above the diagonal are computed (Q^T Q is symmetric) and the rest is
+// mirrored by the epilogue.  ldd >= m rounded up to 8.
+int launch_gram_sym_bf16(gelo_ctx* ctx, int m, const float* Q, int ld, void* D, int ldd, float out_scale, float diag_sub,
+                         float post_scale, cudaStream_t st)
+{
+    if (m <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    const int m8 = (m + 7) & ~7;
+    if ((ld % 4) || ld < m8 || (ldd % 8) || ldd < m8 || !aligned16(Q) || !aligned16(D)) return GELO_ERR_INVALID;
+    CUtensorMap ma, mb;
+    bool a3d = false, b3d = false;
+    if (!make_map_nmajor(ctx, &ma, Q, 4, true, (uint64_t)m, (uint64_t)m, (uint64_t)ld, 32, BM, &a3d) ||
+        !make_map_nmajor(ctx, &mb, Q, 4, true, (uint64_t)m8, (uint64_t)m, (uint64_t)ld, 32, 256, &b3d))
+        return GELO_ERR_CUDA;
+    TcParams p = {};
+    p.M = m; p.N = m8;
+    p.nseg = 1;
+    p.seg[0] = TcSegment{0, 0, 0, 0, ceil_div(m, 32)};
+    p.status = ctx->status_dev;
+    p.csplit = m8;
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
+    p.a3d = a3d ? 1 : 0; p.b3d = b3d ? 1 : 0;
+    p.out_scale = out_scale; p.diag_sub = diag_sub; p.post_scale = post_scale;
+    p.C0 = D; p.ldc = ldd;
+    p.mode = TC_STORE_SYM16;
+    p.tri = 1;
+    const int m_tiles = ceil_div(m, BM), n_tiles = ceil_div(m8, 256);
+    int tiles = 0;
+    for (int nt = 0; nt < n_tiles; ++nt) tiles += (m_tiles < 2 * nt + 2) ? m_tiles : 2 * nt + 2;
+    p.tri_tiles = tiles;
+    return launch_tiles<256, 4, false, true, true>(ctx, ma, ma, mb, mb, ma, p, 2.0 * m * (double)m * m, st);
+}
+
+// C (M x N fp32, stride ldc) -= A (M x K bf16, stride lda) * B (K x N bf16, stride ldb), in place by TMA reduce-add.
+int launch_gemm_bf16_sub(gelo_ctx* ctx, int M, int N, int K, const void* A, int lda, const void* B, int ldb, float* C, int ldc,
+                         cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if ((lda % 8) || (ldb % 8) || (ldc % 4) || !aligned16(A) || !aligned16(B) || !aligned16(C)) return GELO_ERR_INVALID;
+    CUtensorMap ma, mb, mc;
+    bool b3d = false;
+    if (!make_map(ctx, &ma, A, (uint64_t)K, (uint64_t)M, (uint64_t)lda, BK, BM) ||
+        !make_map_nmajor(ctx, &mb, B, 2, false, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, BK, 256, &b3d) ||
+        !make_map_f32_box(ctx, &mc, C, (uint64_t)N, (uint64_t)M, (uint64_t)ldc))
+        return GELO_ERR_CUDA;
+    TcParams p = {};
+    p.M = M; p.N = N;
+    p.nseg = 1;
+    p.seg[0] = TcSegment{0, 0, 0, 0, ceil_div(K, BK)};
+    p.status = ctx->status_dev;
+    p.csplit = N;
+    p.b3d = b3d ? 1 : 0;
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
+    p.mode = TC_SUB_F32;
+    p.C0 = C; p.ldc = ldc;
+    return launch_tiles<256, 3, true>(ctx, ma, ma, mb, mb, mc, p, 2.0 * M * (double)N * K, st);
 }
 
 int launch_gemm_tf32x3(gelo_ctx* ctx, int M, int N, int K, const float* Ahi, const float* Alo, int lda, const float* Bhi,

@@ -730,16 +730,21 @@ int run_householder_qr_tf32(gelo_ctx* ctx, int m, float* R, int ld, float* Q, co
 
 // The tf32 updates leave Q orthogonal to a few 1e-3 only (the tensor core truncates unrounded operands, which
 // shrinks every block reflector a little).  One Newton-Schulz step, Q <- Q - Q D with D = (Q^T Q - I) / 2, squares
-// that defect.  Both products are single large tf32 GEMMs.  Q is dense with log-uniformly spread mantissas, so the
-// truncation loss of Q^T Q is the known constant and is scaled back before the identity is subtracted; what is
-// left in D is zero-mean noise of a few 1e-4 (Frobenius norm over sqrt(m)), which bounds the polished defect.
-int polish_orthogonal_tf32(gelo_ctx* ctx, int m, float* Q, int ld, float* D, float* Qold, cudaStream_t st)
+// that defect.
+//   * D is symmetric: one tf32 product over the tiles on and above the diagonal (a little more than half of them),
+//     mirrored by the epilogue.  Q is dense with log-uniformly spread mantissas, so the truncation loss of Q^T Q is the
+//     known constant and is scaled back before the identity is subtracted; what is left in D is zero-mean noise of a
+//     few 1e-4 (Frobenius norm over sqrt(m)), which bounds the polished defect.
+//   * The correction Q D is small (D is a few 1e-3 per row), so 8 significant bits in each factor are plenty: D is
+//     stored in bf16, Q is copied to bf16 once, and the product runs at the bf16 rate, subtracted from the fp32 Q in
+//     place.  (Relative error of the correction 4e-3, i.e. about 1e-5 of Q.)
+// D16 and Q16 are scratch for m x ld 16-bit values each.
+int polish_orthogonal_tf32(gelo_ctx* ctx, int m, float* Q, int ld, float* D16, float* Q16, cudaStream_t st)
 {
     const float back2 = (1.0f + kTf32TruncLoss) * (1.0f + kTf32TruncLoss);
-    const int m8 = (m + 7) & ~7;
-    GELO_TRY(launch_gemm_tf32(ctx, m, m8, m, Q, ld, true, Q, ld, false, D, ld, true, back2, 1, 0, nullptr, st, 1.0f, 0.5f));
-    GELO_CUDA_OK(cudaMemcpyAsync(Qold, Q, (size_t)m * ld * sizeof(float), cudaMemcpyDeviceToDevice, st));
-    return launch_gemm_tf32(ctx, m, m, m, Qold, ld, false, D, ld, true, Q, ld, false, 1.0f, 1, 0, nullptr, st);
+    GELO_TRY(launch_gram_sym_bf16(ctx, m, Q, ld, D16, ld, back2, 1.0f, 0.5f, st));
+    GELO_TRY(launch_narrow(ctx, m, Q, ld, GELO_BF16, Q16, ld, st));
+    return launch_gemm_bf16_sub(ctx, m, m, m, Q16, ld, D16, ld, Q, ld, st);
 }
 
 }  // namespace gelo

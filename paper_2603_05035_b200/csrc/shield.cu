@@ -3,6 +3,8 @@
 //   1. row norms of H            -- one HBM pass, one warp per row, 16-byte loads
 //   2. median by rank counting   -- every element counts how many others precede it
 //   3. S = (scale * med / sqrt(d)) * N(0,1) from Philox stream 2
+#include <cooperative_groups.h>
+
 #include "common.cuh"
 #include "philox.cuh"
 
@@ -39,13 +41,11 @@ __device__ __forceinline__ float sumsq8h(const uint4& q)
 template <typename T> struct is_half_t { static constexpr bool value = false; };
 template <> struct is_half_t<__half> { static constexpr bool value = true; };
 
+// Euclidean norm of one row by one warp (16-byte loads, lanes strided over the row, butterfly sum): the same
+// summation order wherever it is used, so every route to the shield rows gives the same bytes.
 template <typename T>
-__global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, int n, int d, float* __restrict__ norms)
+__device__ __forceinline__ float warp_row_norm(const T* __restrict__ h, int d, int lane)
 {
-    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
-    const int lane = threadIdx.x & 31;
-    if (row >= n) return;
-    const T* h = H + (size_t)row * d;
     float s = 0.0f;
     if (sizeof(T) == 4) {
         const float4* h4 = reinterpret_cast<const float4*>(h);
@@ -54,12 +54,32 @@ __global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, 
             s = fmaf(v.x, v.x, s); s = fmaf(v.y, v.y, s); s = fmaf(v.z, v.z, s); s = fmaf(v.w, v.w, s);
         }
     } else {
+        // eight 16-byte loads in flight per lane; the partial sums are added in the order of the plain loop
         const uint4* h8 = reinterpret_cast<const uint4*>(h);
-        for (int j = lane; j < d / 8; j += 32) s += is_half_t<T>::value ? sumsq8h(__ldg(h8 + j)) : sumsq8(__ldg(h8 + j));
+        const int g = d / 8;
+        int j = lane;
+        for (; j + 7 * 32 < g; j += 8 * 32) {
+            uint4 v[8];
+#pragma unroll
+            for (int u = 0; u < 8; ++u) v[u] = __ldg(h8 + j + u * 32);
+#pragma unroll
+            for (int u = 0; u < 8; ++u) s += is_half_t<T>::value ? sumsq8h(v[u]) : sumsq8(v[u]);
+        }
+        for (; j < g; j += 32) s += is_half_t<T>::value ? sumsq8h(__ldg(h8 + j)) : sumsq8(__ldg(h8 + j));
     }
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) s += __shfl_xor_sync(0xffffffffu, s, off);
-    if (lane == 0) norms[row] = sqrtf(s);
+    return sqrtf(s);
+}
+
+template <typename T>
+__global__ void __launch_bounds__(256) row_norm_kernel(const T* __restrict__ H, int n, int d, float* __restrict__ norms)
+{
+    const int row = blockIdx.x * 8 + (threadIdx.x >> 5);
+    const int lane = threadIdx.x & 31;
+    if (row >= n) return;
+    const float v = warp_row_norm(H + (size_t)row * d, d, lane);
+    if (lane == 0) norms[row] = v;
 }
 
 // med[0], med[1] = the elements of rank (n-1)/2 and n/2 (ties broken by index).
@@ -87,6 +107,9 @@ __global__ void __launch_bounds__(256) median_rank_kernel(const float* __restric
 }
 
 template <typename T>
+__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q);
+
+template <typename T>
 __global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int k, int d, float scale,
                                                           const float* __restrict__ med, uint64_t seed)
 {
@@ -95,6 +118,13 @@ __global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int
     const uint64_t e0 = q << 2;
     if (e0 >= total) return;                      // d % 8 == 0, so blocks never straddle the end
     const float f = scale * (0.5f * (med[0] + med[1])) / sqrtf((float)d);
+    store_shield_block(S, e0, f, seed, q);
+}
+
+// S[e0 .. e0+3] = f * (the four normals of block q of the shield stream), in the storage type
+template <typename T>
+__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q)
+{
     float z[4];
     gaussian_block(seed, q, GELO_STREAM_SHIELD, 0u, z);
     if (sizeof(T) == 4) {
@@ -116,6 +146,66 @@ __global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int
     }
 }
 
+// All three steps in ONE launch for a batch of at most 256 rows (the decode-shaped call, where three dependent
+// launches cost more than their work): a thread-block cluster of up to 8 CTAs, one warp per row for the norms, every
+// norm stored into every CTA's shared memory (distributed shared memory), one cluster barrier, then each CTA ranks
+// the norms for itself and fills its share of S.  Same arithmetic in the same order as the three kernels above.
+constexpr int kShieldSmallRows = 256;
+
+template <typename T>
+__global__ void __launch_bounds__(1024, 1)
+shield_small_kernel(const T* __restrict__ H, int n, int d, int k, float scale, uint64_t seed, T* __restrict__ S)
+{
+    namespace cg = cooperative_groups;
+    cg::cluster_group cluster = cg::this_cluster();
+    const int CS = (int)cluster.num_blocks();
+    const int rank = (int)cluster.block_rank();
+    __shared__ float norms_s[kShieldSmallRows];
+    __shared__ float med_s[2];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int row = rank * 32 + warp;
+    if (row < n) {
+        const float v = warp_row_norm(H + (size_t)row * d, d, lane);
+        if (lane < CS) cluster.map_shared_rank(&norms_s[row], lane)[0] = v;
+    }
+    if (CS > 1) cluster.sync(); else __syncthreads();
+    const int i = threadIdx.x;
+    if (i < n) {
+        const float mine = norms_s[i];
+        int rk = 0;
+        for (int t = 0; t < n; ++t) {
+            const float o = norms_s[t];
+            rk += (o < mine || (o == mine && t < i)) ? 1 : 0;
+        }
+        if (rk == (n - 1) / 2) med_s[0] = mine;
+        if (rk == n / 2) med_s[1] = mine;
+    }
+    __syncthreads();
+    const float f = scale * (0.5f * (med_s[0] + med_s[1])) / sqrtf((float)d);
+    const uint64_t blocks = ((uint64_t)k * d) >> 2;           // d % 8 == 0
+    for (uint64_t q = (uint64_t)rank * 1024 + threadIdx.x; q < blocks; q += (uint64_t)CS * 1024)
+        store_shield_block(S, q << 2, f, seed, q);
+}
+
+template <typename T>
+int launch_shield_small(gelo_ctx* ctx, const void* H, int n, int d, int k, float scale, uint64_t seed, void* S, cudaStream_t st)
+{
+    const int cs = ceil_div(n, 32);                           // <= 8
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(cs, 1, 1);
+    cfg.blockDim = dim3(1024, 1, 1);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    if (cudaLaunchKernelEx(&cfg, shield_small_kernel<T>, static_cast<const T*>(H), n, d, k, scale, seed, static_cast<T*>(S)) != cudaSuccess)
+        return GELO_ERR_CUDA;
+    return after_launch(ctx);
+}
+
 }  // namespace
 
 ShieldScratch carve_shield(Arena& a, int n)
@@ -130,6 +220,11 @@ int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float sca
                     int dtype, void* S, const ShieldScratch& s, cudaStream_t st)
 {
     if (k <= 0) return GELO_OK;
+    if (n <= kShieldSmallRows) {
+        if (dtype == GELO_BF16) return launch_shield_small<__nv_bfloat16>(ctx, H, n, d, k, scale, seed, S, st);
+        if (dtype == GELO_F16) return launch_shield_small<__half>(ctx, H, n, d, k, scale, seed, S, st);
+        return launch_shield_small<float>(ctx, H, n, d, k, scale, seed, S, st);
+    }
     if (dtype == GELO_BF16)
         row_norm_kernel<__nv_bfloat16><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(H), n, d, s.norms);
     else if (dtype == GELO_F16)

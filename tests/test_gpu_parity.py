@@ -292,6 +292,53 @@ def test_mix_full_size_seam_inside_a_k_block(ctx, oracle):
     assert oracle.rel_fro(f64(U2[rows2]), ref2) <= 4e-3
 
 
+@pytest.mark.parametrize("dt", ["bf16", "f16"])
+@pytest.mark.parametrize("n,k,d,p,split", [(64, 4, 4096, 12288, True), (64, 0, 256, 768, True), (100, 28, 520, 1536, True),
+                                           (1, 0, 8, 96, False), (7, 3, 72, 11008, False), (33, 0, 64, 4736, False)])
+def test_project_unmix_one_kernel(ctx, oracle, n, k, d, p, split, dt):
+    """Eq. 2 and Eq. 3 in one kernel for a small batch: against the oracle's two products (with Y' rounded to the
+    storage type in between, as the stand-alone projection stores it) and against the two stand-alone launches."""
+    m = n + k
+    ld = ctx.mixing_ld(m)
+    ctx.ensure_workspace(n, k, d, p, dt)
+    X = padded(m, ld, TDT[dt])
+    _, x64 = oracle.sample_mixing(m, 1, seed=32)
+    X[:, :m] = dev(x64, TDT[dt])
+    g = torch.Generator(device="cuda"); g.manual_seed(91)
+    U = (3.0 * torch.randn((m, d), device="cuda", generator=g)).to(TDT[dt])
+    W = inputs.make_weight(d, p, dt, 7, "cuda")
+    outs = [torch.full((n, p // 3 if split else p), float("nan"), device="cuda", dtype=TDT[dt]) for _ in range(3 if split else 1)]
+    ctx.project_unmix(U, W, X, ld, n, k, d, p, dt, *outs)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == binding.OK
+    y = np.hstack([f64(o) for o in outs])
+    assert np.isfinite(y).all()
+    yp = torch.as_tensor(oracle.matmul(f64(U), f64(W))).to(TDT[dt])           # Y' as stored
+    ref = oracle.matmul(f64(X[:n, :m]), f64(yp))
+    assert oracle.rel_fro(y, ref) <= 4e-3 * (1.0 if dt == "bf16" else 0.25)      # one rounding of the output
+    # the two stand-alone launches give the same values up to the summation order inside the tensor core
+    Yp = torch.empty((m, p), device="cuda", dtype=TDT[dt])
+    outs2 = [torch.empty_like(o) for o in outs]
+    ctx.project(U, W, m, d, p, dt, Yp)
+    ctx.unmix(X, ld, Yp, n, k, p, dt, *outs2)
+    torch.cuda.synchronize()
+    y2 = np.hstack([f64(o) for o in outs2])
+    assert oracle.rel_fro(y, y2) <= 1e-3 * (1.0 if dt == "bf16" else 0.25)
+
+
+def test_project_unmix_rejects_what_it_cannot_serve(ctx):
+    L = binding.load_library()
+    st = torch.cuda.current_stream().cuda_stream
+    t = torch.zeros((256, 256), device="cuda", dtype=torch.bfloat16)
+    q = torch.zeros((256, 8192), device="cuda", dtype=torch.bfloat16)
+    a = (ctx._h, t.data_ptr(), t.data_ptr(), t.data_ptr())
+    assert L.gelo_project_unmix(*a, 256, 129, 0, 256, 96, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED   # m > 128
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 72, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED    # p % 32
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 96, F32, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED
+    assert L.gelo_project_unmix(*a, 64, 64, 4, 256, 96, BF16, q.data_ptr(), None, None, st) == binding.ERR_INVALID         # lda < m
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 96, BF16, None, None, None, st) == binding.ERR_INVALID
+
+
 # ------------------------------------------------------------------------- whole call
 
 def _run_offload(ctx, w, call, host=False):
@@ -783,9 +830,9 @@ def test_profile_counts_launches(ctx):
     ctx.profile_start()
     ctx.qkv_offload(H, W, w.n, w.k, w.d, w.p, ORTHOGONAL, seed, 10.0, w.dtype, Q, K, V)
     prof = ctx.profile_stop()
-    assert prof["gemm_tc"]["launches"] == 3 and prof["gemm_tc"]["ms"] > 0          # mix, project, unmix
+    assert prof["gemm_tc"]["launches"] == 1 and prof["gemm_tc"]["ms"] > 0          # project + unmix in one tensor-core kernel
     assert prof["qr_panel"]["launches"] == 3                                        # m = 68: three 32-column panels
-    assert prof["gemm_tc"]["work"] == pytest.approx(2.0 * (68 * 68 * 4096 + 68 * 4096 * 12288 + 64 * 68 * 12288))
+    assert prof["gemm_tc"]["work"] == pytest.approx(2.0 * (68 * 4096 * 12288 + 64 * 68 * 12288))     # (the mix runs on the FMA pipes)
 
 
 # ------------------------------------------------------------------------- bounded waits
