@@ -216,7 +216,7 @@ int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int
 int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev, int n, int k,
                int p, int dtype, void* Q_dev, void* K_dev, void* V_dev, void* stream);
 
-/* Eq. 2 and Eq. 3 in one kernel for a small batch (m = n + k <= 128, 16-bit element types, p a multiple of 32 and at
+/* Eq. 2 and Eq. 3 in one kernel for a small batch (m = n + k <= 128, 16-bit element types, p a multiple of 64 and at
  * most 128 columns per SM): every SM streams its own column slab of W_dev once, keeps its slab of Y' = U W on chip,
  * rounds it to the element type exactly as gelo_project would store it, multiplies by the first n rows of Ainv_dev and
  * writes Q | K | V as gelo_unmix does.  Results equal gelo_project followed by gelo_unmix up to the summation order

@@ -209,8 +209,8 @@ struct Tf32x3Scratch {
 
 // ---- projection and unmixing of a small batch in one kernel (decode.cu) ---------------------------------
 
-// true when launch_project_unmix can serve the call: 16-bit storage, m = n + k <= 128, p a multiple of 32 whose
-// 32-column boxes leave every CTA a slab of at most 128 columns
+// true when launch_project_unmix can serve the call: 16-bit storage, m = n + k <= 128, p a multiple of 64 whose
+// 64-column boxes leave every CTA a slab of at most 128 columns
 bool project_unmix_supports(const gelo_ctx*, int n, int k, int d, int p, int dtype, int lda, int nsplit);
 // Q | K | V (or one n x p result in Q when K = V = nullptr) = (Ainv[0:n, 0:n+k] (U W)); U: (n+k) x d, W: d x p
 int launch_project_unmix(gelo_ctx*, const void* U, const void* W, const void* Ainv, int lda, int n, int k, int d, int p,

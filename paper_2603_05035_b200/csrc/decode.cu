@@ -4,21 +4,21 @@
 //     Y' = U W            (m x d) (d x p)      -- the offloaded contraction, bound by streaming W once from HBM
 //     Y  = (A^-1 Y')[0:n] (n x m) (m x p)      -- tiny; applied to each column slab of Y' while it is still on chip
 //
-// A product with so few rows is a stream of W: what matters is that every SM pulls a disjoint share of it.  W is cut
-// into boxes of 32 columns and the boxes are dealt evenly over one CTA per SM (p = 12288: 384 boxes, 2 or 3 per
-// CTA), so that each CTA streams its own d x (64 or 96) slab through a TMA / mbarrier pipeline while re-reading the
-// small U from L2.  The accumulator Y'_slab (m rows, padded to the 128 lanes of tensor memory) never goes to HBM:
+// A product with so few rows is a stream of W: what matters is that many SMs pull disjoint shares of it with long
+// requests.  W is cut into boxes of 64 columns (128-byte rows; measured: 64-byte rows stream at 4.3 TB/s, 128-byte rows
+// faster) and the boxes are dealt evenly over the CTAs (p = 12288: 192 boxes, 2 per CTA on 96 SMs), so that each CTA
+// streams its own d x 128 slab through a TMA / mbarrier pipeline while re-reading the small U from L2.  The accumulator Y'_slab (m rows, padded to the 128 lanes of tensor memory) never goes to HBM:
 // the epilogue warps round it to the storage type, exactly as the stand-alone projection would store it, lay it out
 // in shared memory as the B operand of a second tcgen05 product with the first n rows of A^-1, and write the result
 // straight into Q | K | V.  Two launches (gelo_project, gelo_unmix) and the round trip of Y' become one launch.
 //
-// Layouts.  U tiles and the A^-1 rows: K-major, 128-byte swizzle (as in gemm_tc.cu).  W boxes: 64 k-rows x 32
-// columns, N-major with the 64-byte swizzle (atoms of 8 k-rows x 64 bytes; boxes 4096 bytes apart).  The Y' slab:
+// Layouts.  U tiles and the A^-1 rows: K-major, 128-byte swizzle (as in gemm_tc.cu).  W boxes: 64 k-rows x 64
+// columns, N-major with the 128-byte swizzle (atoms of 8 k-rows x 128 bytes; boxes 8192 bytes apart).  The Y' slab:
 // N-major without swizzle, i.e. core matrices of 8 k-rows x 8 columns (128 contiguous bytes), 8-row groups 128 bytes
 // apart, 8-column groups kpad * 16 bytes apart - which is what a thread holding one row of the accumulator can write
 // as 16-byte pieces without bank conflicts.
-// Warp roles: warp 0 issues TMA, warp 1 issues MMA and owns tensor memory, warps 2-5 are the epilogue (one per
-// tensor-memory lane quarter).  Every barrier wait is bounded in time as in gemm_tc.cu.
+// Warp roles: warp 0 issues TMA, warps 1-2 issue MMA for alternate k-blocks (warp 1 owns tensor memory), warps 3-6 are
+// the epilogue (one per tensor-memory lane quarter).  Every barrier wait is bounded in time as in gemm_tc.cu.
 #include <cuda.h>
 
 #include "common.cuh"
@@ -30,22 +30,25 @@ namespace {
 
 using namespace tcx;
 
-constexpr int kDecThreads = 64 + 4 * 32;
+constexpr int kDecIssuers = 2;                           // MMA-issuing warps, each with its own accumulator of Y'
+constexpr int kDecThreads = 32 * (1 + kDecIssuers + 4);
 constexpr int kDecBK = 64;                              // k elements per stage: 128 bytes of a K-major row
 // The MMA always multiplies 128 rows of A.  Only the first kpad rows of a U tile (m real ones, zero-filled up to a
 // multiple of 16) are ever loaded; the rows behind them are whatever the following shared memory holds, and they only
 // reach accumulator rows that nobody reads.  Every byte of shared memory not spent on those rows is a byte of W in flight.
 constexpr uint32_t kDecRowBytes = kDecBK * 2;           // one K-major row of a tile: 128 bytes
 constexpr uint32_t kDecAReach = 128 * kDecRowBytes;     // bytes the MMA reads from the start of an A tile
-constexpr uint32_t kDecBoxBytes = kDecBK * 64;          // one W box: 64 k-rows x 32 columns
-constexpr int kDecMaxBoxes = 4;                         // boxes per CTA: slab of at most 128 columns
-constexpr uint32_t kDecTmemCols = 256;                  // Y' slab in columns 0.., Y slab in columns 128..
+constexpr int kDecBoxCols = 64;                         // W arrives in boxes of 64 columns: 128-byte rows, the longest a swizzled box takes
+constexpr uint32_t kDecBoxBytes = kDecBK * 128;         // one W box: 64 k-rows x 64 columns
+constexpr int kDecMaxBoxes = 2;                         // boxes per CTA: slab of at most 128 columns
+constexpr uint32_t kDecAccCols = 128;                   // columns of one accumulator (a slab is at most 128 columns wide)
+constexpr uint32_t kDecTmemCols = 512;                  // two partial Y' slabs, then the Y slab (a power of two)
 
 struct DecParams {
     int m, n, d;
     int kpad;                   // m rounded up to 16: the K extent of the second product, and the rows of a U tile
     int npad;                   // n rounded up to 16: the rows of A^-1 that are loaded
-    int boxes, base, rem;       // p / 32 boxes; CTA i takes base + (i < rem) of them
+    int boxes, base, rem;       // p / 64 boxes; CTA i takes base + (i < rem) of them
     int stages;                 // operand stages that fit next to the fixed buffers
     int nbmax;                  // base + (rem > 0): boxes of the widest slab (stage stride)
     int group;                  // CTAs per group; group g walks the k-blocks starting from g * kstep (see the kernel)
@@ -79,7 +82,7 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
     const uint32_t ainv_tile = (uint32_t)prm.npad * kDecRowBytes;                         // one K-major tile of A^-1 rows
     const uint32_t ainv_base = tiles_base + (uint32_t)prm.stages * stage_bytes;           // 1024-byte aligned
     const uint32_t y_base = ainv_base + 2u * ainv_tile;
-    const uint32_t y_bytes = (uint32_t)prm.kpad * 16u * (uint32_t)(prm.nbmax * 4);       // kpad x (nbmax * 32 columns) x 2 bytes
+    const uint32_t y_bytes = (uint32_t)prm.kpad * 16u * (uint32_t)(prm.nbmax * 8);       // kpad x (nbmax * 64 columns) x 2 bytes
     const uint32_t bar_off = (uint32_t)prm.stages * stage_bytes + 2u * ainv_tile + ((y_bytes + 15u) & ~15u);
     const uint32_t bar_base = tiles_base + bar_off;
     uint8_t* bar_gen = gen_base + bar_off;
@@ -96,8 +99,8 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
     const int cta = blockIdx.x;
     const int nb = prm.base + (cta < prm.rem ? 1 : 0);                 // boxes of this CTA's slab
     const int box0 = cta * prm.base + min(cta, prm.rem);
-    const int ncols = nb * 32;
-    const int col0 = box0 * 32;
+    const int ncols = nb * kDecBoxCols;
+    const int col0 = box0 * kDecBoxCols;
     const int nkb = (prm.d + kDecBK - 1) / kDecBK;
     // Every CTA needs every tile of U.  If all CTAs walked the k-blocks in the same order they would all ask the L2 for
     // the same few lines at the same moment; instead groups of neighbouring CTAs (neighbours read adjacent columns of
@@ -106,7 +109,7 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) { mbar_init(full_bar(s), 1); mbar_init(empty_bar(s), 1); }
-        mbar_init(ainv_bar, 1); mbar_init(acc1_bar, 1); mbar_init(y_bar, 4); mbar_init(acc2_bar, 1);
+        mbar_init(ainv_bar, 1); mbar_init(acc1_bar, kDecIssuers); mbar_init(y_bar, 4); mbar_init(acc2_bar, 1);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -135,60 +138,67 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
                 tma_load_2d(ainv_base + ainv_tile, &map_ainv, kDecBK, 0, ainv_bar);
             }
             const CUtensorMap* mw = (nb == prm.nbmax) ? &map_w_wide : &map_w_narrow;
+            int s = 0, kq = kb_first;
+            uint32_t ph = 0;
             for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % S;
-                const uint32_t ph = (uint32_t)(kb / S) & 1u;
                 if (!mbar_wait(empty_bar(s), ph ^ 1u, abort_flag, prm.wait_ns)) { ok = false; break; }
                 const uint32_t sa = tiles_base + (uint32_t)s * stage_bytes;
                 mbar_expect_tx(full_bar(s), a_bytes + (uint32_t)nb * kDecBoxBytes);
-                int kq = kb + kb_first;
-                if (kq >= nkb) kq -= nkb;
                 tma_load_3d(sa + a_bytes, mw, 0, kq * kDecBK, box0, full_bar(s));        // the W slab first: it comes from HBM
                 tma_load_2d(sa, &map_u, kq * kDecBK, 0, full_bar(s));
+                if (++s == S) { s = 0; ph ^= 1u; }
+                if (++kq == nkb) kq = 0;
             }
             if (!ok) { *abort_flag = 1; atomicCAS(prm.status, 0, (int)GELO_ERR_TIMEOUT); }
         }
-    } else if (warp == 1) {
-        // ================= MMA issuer =================
+    } else if (warp <= kDecIssuers) {
+        // ================= MMA issuers =================
+        // A thread needs some 700 cycles to get through one k-block (barrier test, four instructions, commit), about
+        // three times what the tensor core then spends on it, and the weight stream waits for the slower of the two.
+        // Two threads therefore take alternate k-blocks, each into an accumulator of its own (the epilogue adds them).
         if (lane == 0 && nb > 0) {
+            const int me = warp - 1;
             bool ok = true;
-            for (int kb = 0; kb < nkb; ++kb) {
-                const int s = kb % S;
-                const uint32_t ph = (uint32_t)(kb / S) & 1u;
+            const uint32_t acc = tmem_base + (uint32_t)me * kDecAccCols;
+            int s = me % S;
+            uint32_t ph = (uint32_t)(me / S) & 1u;
+            for (int kb = me; kb < nkb; kb += kDecIssuers) {
                 if (!mbar_wait(full_bar(s), ph, abort_flag, prm.wait_ns)) { ok = false; break; }
-                tc_fence_after();
                 const uint32_t sa = tiles_base + (uint32_t)s * stage_bytes;
                 const uint32_t sb = sa + a_bytes;
+                const uint64_t da0 = smem_desc(sa, 16, 1024, 2);                          // K-major, 128-byte swizzle
+                const uint64_t db0 = smem_desc(sb, kDecBoxBytes, 1024, 2);                // N-major, 128-byte swizzle
 #pragma unroll
-                for (int ks = 0; ks < 4; ++ks) {
-                    const uint64_t da = smem_desc(sa + ks * 32, 16, 1024, 2);              // K-major, 128-byte swizzle
-                    const uint64_t db = smem_desc(sb + ks * 1024, kDecBoxBytes, 512, 4);   // N-major, 64-byte swizzle
-                    tc_mma_bf16(tmem_base, da, db, idesc, (kb | ks) != 0 ? 1u : 0u);
-                }
+                for (int ks = 0; ks < 4; ++ks)       // the start address field counts 16-byte units: 32 and 2048 bytes per step
+                    tc_mma_bf16(acc, da0 + (uint64_t)(ks * 2), db0 + (uint64_t)(ks * 128), idesc, (kb != me || ks != 0) ? 1u : 0u);
                 tc_commit(empty_bar(s));
+                s += kDecIssuers;
+                if (s >= S) { s -= S; ph ^= 1u; }
             }
             if (ok) {
-                tc_commit(acc1_bar);
+                if (me < nkb) tc_commit(acc1_bar); else mbar_arrive(acc1_bar);            // (no k-block, nothing to wait for)
                 // second product: Y_slab = A^-1[0:n, 0:kpad] * Y'_slab once the epilogue has laid Y'_slab out
-                if (mbar_wait(y_bar, 0, abort_flag, prm.wait_ns) && mbar_wait(ainv_bar, 0, abort_flag, prm.wait_ns)) {
-                    tc_fence_after();
-                    const int ksteps = prm.kpad >> 4;
-                    for (int ks = 0; ks < ksteps; ++ks) {
-                        const uint32_t at = ainv_base + (uint32_t)(ks >> 2) * ainv_tile + (uint32_t)(ks & 3) * 32u;
-                        const uint64_t da = smem_desc(at, 16, 1024, 2);
-                        // no swizzle: 8-row groups 128 bytes apart (leading offset), 8-column groups kpad * 16 apart (stride offset)
-                        const uint64_t db = smem_desc(y_base + (uint32_t)ks * 256u, 128, (uint32_t)prm.kpad * 16u, 0);
-                        tc_mma_bf16(tmem_base + 128u, da, db, idesc, ks != 0 ? 1u : 0u);
+                if (me == 0) {
+                    if (mbar_wait(y_bar, 0, abort_flag, prm.wait_ns) && mbar_wait(ainv_bar, 0, abort_flag, prm.wait_ns)) {
+                        tc_fence_after();
+                        const int ksteps = prm.kpad >> 4;
+                        for (int ks = 0; ks < ksteps; ++ks) {
+                            const uint32_t at = ainv_base + (uint32_t)(ks >> 2) * ainv_tile + (uint32_t)(ks & 3) * 32u;
+                            const uint64_t da = smem_desc(at, 16, 1024, 2);
+                            // no swizzle: 8-row groups 128 bytes apart (leading offset), 8-column groups kpad * 16 apart (stride offset)
+                            const uint64_t db = smem_desc(y_base + (uint32_t)ks * 256u, 128, (uint32_t)prm.kpad * 16u, 0);
+                            tc_mma_bf16(tmem_base + (uint32_t)(kDecIssuers * kDecAccCols), da, db, idesc, ks != 0 ? 1u : 0u);
+                        }
+                        tc_commit(acc2_bar);
+                    } else {
+                        ok = false;
                     }
-                    tc_commit(acc2_bar);
-                } else {
-                    ok = false;
                 }
             }
             if (!ok) { *abort_flag = 1; atomicCAS(prm.status, 0, (int)GELO_ERR_TIMEOUT); }
         }
     } else if (nb > 0) {
-        // ================= epilogue (warps 2..5) =================
+        // ================= epilogue (four warps, one per tensor-memory lane quarter) =================
         const int quarter = warp & 3;                    // the tensor-memory lane quarter this warp may read
         const int row = quarter * 32 + lane;
         bool ok = true;
@@ -202,7 +212,15 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
                 for (int c = 0; c < ncols; c += 32) {
                     uint32_t v[32];
                     tc_ld_32cols(taddr + c, v);
-                    tc_ld_wait();
+                    if (nkb > 1) {                            // the second issuer's share of the k-blocks
+                        uint32_t w[32];
+                        tc_ld_32cols(taddr + kDecAccCols + c, w);
+                        tc_ld_wait();
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(w[j]));
+                    } else {
+                        tc_ld_wait();
+                    }
                     if (row < prm.kpad) {
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
@@ -230,7 +248,7 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
         if (ok) {
             tc_fence_after();
             if (quarter * 32 < prm.n) {
-                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + 128u;
+                const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(kDecIssuers * kDecAccCols);
                 for (int c = 0; c < ncols; c += 32) {
                     uint32_t v[32];
                     tc_ld_32cols(taddr + c, v);
@@ -275,17 +293,17 @@ bool map_kmajor(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, uint64_t cols,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// W (d x p, row stride p) as {32 columns, d rows, p / 32 boxes}: one copy brings `nb` boxes of 64 rows, each box landing
-// as 64 rows of 64 bytes in the 64-byte swizzle
+// W (d x p, row stride p) as {64 columns, d rows, p / 64 boxes}: one copy brings `nb` boxes of 64 rows, each box landing
+// as 64 rows of 128 bytes in the 128-byte swizzle
 bool map_w_boxes(gelo_ctx* ctx, CUtensorMap* map, const void* W, uint64_t d, uint64_t p, uint32_t nb)
 {
     EncodeFn enc = reinterpret_cast<EncodeFn>(ctx->tmap_encode);
-    const cuuint64_t dims[3] = { 32, d, p / 32 };
-    const cuuint64_t strides[2] = { p * 2, 64 };
-    const cuuint32_t box[3] = { 32, (cuuint32_t)kDecBK, nb };
+    const cuuint64_t dims[3] = { (cuuint64_t)kDecBoxCols, d, p / kDecBoxCols };
+    const cuuint64_t strides[2] = { p * 2, (cuuint64_t)kDecBoxCols * 2 };
+    const cuuint32_t box[3] = { (cuuint32_t)kDecBoxCols, (cuuint32_t)kDecBK, nb };
     const cuuint32_t estr[3] = { 1, 1, 1 };
     return enc(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(W), dims, strides, box, estr,
-               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -429,10 +447,10 @@ bool project_unmix_supports(const gelo_ctx* ctx, int n, int k, int d, int p, int
 {
     const int m = n + k;
     if (dtype == GELO_F32 || m > 128 || n <= 0 || k < 0 || d <= 0 || p <= 0) return false;
-    if ((d % 8) || (p % 32) || (lda % 8) || lda < m) return false;
+    if ((d % 8) || (p % kDecBoxCols) || (lda % 8) || lda < m) return false;
     if (nsplit != 1 && nsplit != 3) return false;
     if (nsplit == 3 && ((p % 3) || ((p / 3) % 8))) return false;
-    const int boxes = p / 32;
+    const int boxes = p / kDecBoxCols;
     const int ncta = boxes < ctx->sm_count ? boxes : ctx->sm_count;
     return (boxes + ncta - 1) / ncta <= kDecMaxBoxes;
 }
@@ -449,7 +467,7 @@ int launch_project_unmix(gelo_ctx* ctx, const void* U, const void* W, const void
     prm.m = m; prm.n = n; prm.d = d;
     prm.kpad = (m + 15) & ~15;
     prm.npad = (n + 15) & ~15;
-    prm.boxes = p / 32;
+    prm.boxes = p / kDecBoxCols;
     // as few CTAs as keep the widest slab no wider than it must be (p = 12288 on 148 SMs: 128 CTAs of 3 boxes each), which
     // evens the slabs out and leaves the other SMs to kernels of other streams
     const int widest = (prm.boxes + ctx->sm_count - 1) / ctx->sm_count;
@@ -459,7 +477,7 @@ int launch_project_unmix(gelo_ctx* ctx, const void* U, const void* W, const void
     const uint32_t a_bytes = (uint32_t)prm.kpad * kDecRowBytes;
     const uint32_t stage_bytes = a_bytes + (uint32_t)prm.nbmax * kDecBoxBytes;
     const uint32_t ainv_tile = (uint32_t)prm.npad * kDecRowBytes;
-    const uint32_t y_bytes = (uint32_t)prm.kpad * 16u * (uint32_t)(prm.nbmax * 4);
+    const uint32_t y_bytes = (uint32_t)prm.kpad * 16u * (uint32_t)(prm.nbmax * 8);
     // behind the last A-type tile (the second tile of A^-1 rows) the MMA still reads up to 128 rows' worth of bytes:
     // the tail of the allocation (Y' slab, barriers, padding) is made long enough for that
     uint32_t tail = ((y_bytes + 15u) & ~15u) + 512u /*barriers*/;
@@ -467,7 +485,10 @@ int launch_project_unmix(gelo_ctx* ctx, const void* U, const void* W, const void
     const uint32_t fixed = 2u * ainv_tile + tail + 1024u /*alignment*/;
     int stages = (int)((kDecSmemBudget - fixed) / stage_bytes);
     if (stages > 12) stages = 12;
-    if (stages < 2) return GELO_ERR_UNSUPPORTED;
+    // A stage must always be consumed by the same issuer thread: a thread that saw only every other phase of a stage's
+    // barrier could take the completed phase before last for the one it waits for (parities repeat after two phases).
+    stages -= stages % kDecIssuers;
+    if (stages < kDecIssuers) return GELO_ERR_UNSUPPORTED;
     prm.stages = stages;
     const uint32_t smem = (uint32_t)stages * stage_bytes + fixed;
     prm.group = ctx->dec_group > 0 ? ctx->dec_group : ncta;

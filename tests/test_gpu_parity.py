@@ -294,7 +294,7 @@ def test_mix_full_size_seam_inside_a_k_block(ctx, oracle):
 
 @pytest.mark.parametrize("dt", ["bf16", "f16"])
 @pytest.mark.parametrize("n,k,d,p,split", [(64, 4, 4096, 12288, True), (64, 0, 256, 768, True), (100, 28, 520, 1536, True),
-                                           (1, 0, 8, 96, False), (7, 3, 72, 11008, False), (33, 0, 64, 4736, False)])
+                                           (1, 0, 8, 192, False), (7, 3, 72, 11008, False), (33, 0, 64, 4736, False)])
 def test_project_unmix_one_kernel(ctx, oracle, n, k, d, p, split, dt):
     """Eq. 2 and Eq. 3 in one kernel for a small batch: against the oracle's two products (with Y' rounded to the
     storage type in between, as the stand-alone projection stores it) and against the two stand-alone launches."""
@@ -332,11 +332,11 @@ def test_project_unmix_rejects_what_it_cannot_serve(ctx):
     t = torch.zeros((256, 256), device="cuda", dtype=torch.bfloat16)
     q = torch.zeros((256, 8192), device="cuda", dtype=torch.bfloat16)
     a = (ctx._h, t.data_ptr(), t.data_ptr(), t.data_ptr())
-    assert L.gelo_project_unmix(*a, 256, 129, 0, 256, 96, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED   # m > 128
-    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 72, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED    # p % 32
-    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 96, F32, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED
-    assert L.gelo_project_unmix(*a, 64, 64, 4, 256, 96, BF16, q.data_ptr(), None, None, st) == binding.ERR_INVALID         # lda < m
-    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 96, BF16, None, None, None, st) == binding.ERR_INVALID
+    assert L.gelo_project_unmix(*a, 256, 129, 0, 256, 192, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED  # m > 128
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 96, BF16, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED    # p % 64
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 192, F32, q.data_ptr(), None, None, st) == binding.ERR_UNSUPPORTED
+    assert L.gelo_project_unmix(*a, 64, 64, 4, 256, 192, BF16, q.data_ptr(), None, None, st) == binding.ERR_INVALID        # lda < m
+    assert L.gelo_project_unmix(*a, 128, 64, 0, 256, 192, BF16, None, None, None, st) == binding.ERR_INVALID
 
 
 # ------------------------------------------------------------------------- whole call
