@@ -218,6 +218,9 @@ int mix_impl(gelo_ctx* ctx, const void* A, int lda, const void* H, const void* S
 int project_impl(gelo_ctx* ctx, const void* U, const void* W, int m, int d, int p, int dtype, void* Yp,
                  cudaStream_t st, const Tf32x3Scratch* t3 = nullptr)
 {
+    // a product with few rows is a stream of W: the kernel of the small-batch path, without its unmixing half
+    if (ctx->fuse_small && project_unmix_supports(ctx, m, 0, d, p, dtype, (m + 7) & ~7, 1) && !misaligned(U) && !misaligned(Yp))
+        return launch_project_unmix(ctx, U, W, nullptr, 0, m, 0, d, p, dtype, Yp, nullptr, nullptr, st);
     GemmArgs g;
     g.M = m; g.N = p; g.K = d;
     g.A = U; g.lda = d; g.B = W; g.ldb = p;

@@ -56,6 +56,7 @@ struct DecParams {
     void* C0; void* C1; void* C2;
     int ldc, csplit;
     int out_f16;
+    int plain;                  // no second product: the rounded Y' slab itself is the result (m rows)
     unsigned long long wait_ns;
     int* status;
 };
@@ -131,7 +132,7 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
         // ================= TMA producer =================
         if (lane == 0 && nb > 0) {
             bool ok = true;
-            if (prm.wait_ns != 0) {
+            if (prm.wait_ns != 0 && !prm.plain) {
                 // the first n rows of A^-1 (columns past m and rows past n arrive as zeros)
                 mbar_expect_tx(ainv_bar, 2u * ainv_tile);
                 tma_load_2d(ainv_base, &map_ainv, 0, 0, ainv_bar);
@@ -178,7 +179,7 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
             if (ok) {
                 if (me < nkb) tc_commit(acc1_bar); else mbar_arrive(acc1_bar);            // (no k-block, nothing to wait for)
                 // second product: Y_slab = A^-1[0:n, 0:kpad] * Y'_slab once the epilogue has laid Y'_slab out
-                if (me == 0) {
+                if (me == 0 && !prm.plain) {
                     if (mbar_wait(y_bar, 0, abort_flag, prm.wait_ns) && mbar_wait(ainv_bar, 0, abort_flag, prm.wait_ns)) {
                         tc_fence_after();
                         const int ksteps = prm.kpad >> 4;
@@ -221,7 +222,17 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
                     } else {
                         tc_ld_wait();
                     }
-                    if (row < prm.kpad) {
+                    if (prm.plain) {
+                        if (row < prm.m) {
+#pragma unroll
+                            for (int g = 0; g < 4; ++g) {
+                                const int gc = col0 + c + 8 * g;
+                                const int chunk = gc / prm.csplit;
+                                void* base = chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2);
+                                store8(base, (size_t)row * prm.ldc + (gc - chunk * prm.csplit), v + 8 * g, prm.out_f16);
+                            }
+                        }
+                    } else if (row < prm.kpad) {
 #pragma unroll
                         for (int g = 0; g < 4; ++g) {
                             uint32_t q0, q1, q2, q3;
@@ -238,14 +249,16 @@ project_unmix_kernel(const __grid_constant__ CUtensorMap map_u, const __grid_con
                     }
                 }
             }
-            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads this through the async proxy
-            tc_fence_before();
-            __syncwarp();
-            if (lane == 0) mbar_arrive(y_bar);
-            // ---- Y slab: rows 0 .. n-1 to Q | K | V ----
-            if (!mbar_wait(acc2_bar, 0, abort_flag, prm.wait_ns)) ok = false;
+            if (!prm.plain) {
+                asm volatile("fence.proxy.async.shared::cta;" ::: "memory");   // the tensor core reads this through the async proxy
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(y_bar);
+                // ---- Y slab: rows 0 .. n-1 to Q | K | V ----
+                if (!mbar_wait(acc2_bar, 0, abort_flag, prm.wait_ns)) ok = false;
+            }
         }
-        if (ok) {
+        if (ok && !prm.plain) {
             tc_fence_after();
             if (quarter * 32 < prm.n) {
                 const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(kDecIssuers * kDecAccCols);
@@ -455,11 +468,13 @@ bool project_unmix_supports(const gelo_ctx* ctx, int n, int k, int d, int p, int
     return (boxes + ncta - 1) / ncta <= kDecMaxBoxes;
 }
 
-// Q | K | V (or one n x p result when K = V = nullptr) = (Ainv[0:n, 0:m] (U W)) for m = n + k <= 128.
+// Q | K | V (or one n x p result when K = V = nullptr) = (Ainv[0:n, 0:m] (U W)) for m = n + k <= 128.  With
+// Ainv == nullptr the kernel stops after the first product: the result is U W itself (n + k rows).
 int launch_project_unmix(gelo_ctx* ctx, const void* U, const void* W, const void* Ainv, int lda, int n, int k, int d, int p,
                          int dtype, void* Q, void* K, void* V, cudaStream_t st)
 {
     const int nsplit = (K || V) ? 3 : 1;
+    if (!Ainv) lda = (n + k + 7) & ~7;
     if (!project_unmix_supports(ctx, n, k, d, p, dtype, lda, nsplit)) return GELO_ERR_UNSUPPORTED;
     if (!ctx->tmap_encode) return GELO_ERR_CUDA;
     const int m = n + k;
@@ -500,11 +515,12 @@ int launch_project_unmix(gelo_ctx* ctx, const void* U, const void* W, const void
     prm.ldc = nsplit == 3 ? p / 3 : p;
     prm.csplit = nsplit == 3 ? p / 3 : p;
     prm.out_f16 = dtype == GELO_F16 ? 1 : 0;
+    prm.plain = Ainv ? 0 : 1;
     prm.wait_ns = ctx->wait_limit_ns;
     prm.status = ctx->status_dev;
     CUtensorMap mu, mww, mwn, ma;
     if (!map_kmajor(ctx, &mu, U, (uint64_t)d, (uint64_t)m, (uint64_t)d, (uint32_t)prm.kpad) ||
-        !map_kmajor(ctx, &ma, Ainv, (uint64_t)m, (uint64_t)n, (uint64_t)lda, (uint32_t)prm.npad) ||
+        !map_kmajor(ctx, &ma, Ainv ? Ainv : U, (uint64_t)m, (uint64_t)n, (uint64_t)(Ainv ? lda : d), (uint32_t)prm.npad) ||
         !map_w_boxes(ctx, &mww, W, (uint64_t)d, (uint64_t)p, (uint32_t)prm.nbmax) ||
         !map_w_boxes(ctx, &mwn, W, (uint64_t)d, (uint64_t)p, (uint32_t)(prm.base > 0 ? prm.base : 1)))
         return GELO_ERR_CUDA;

@@ -486,6 +486,124 @@ t_merge_kernel(const float* __restrict__ part, int slabs, int ldp, const float* 
     for (int idx = tid; idx < 128 * 128; idx += 1024) T128[idx] = Tm[idx >> 7][idx & 127];
 }
 
+// ---- the whole factorisation of a small matrix (m <= 128) in one launch ---------------------------------------
+//
+// A decode-shaped call mixes a few dozen rows, and for such a matrix the blocked path above is some thirty dependent
+// launches of a few microseconds each.  Here one CTA does everything with the matrix in registers: eight consecutive
+// lanes share COLUMN c (lane h of the group holds rows h, h + 8, ...), so applying a reflector to a column is a dozen
+// private FMAs plus a three-step shuffle inside the group, and the only block-wide communication is the reflector
+// itself, which the owners of column j write to shared memory once per column (one barrier per column).  The
+// reflectors stay in shared memory; afterwards each group builds its column of Q = H_0 ... H_(m-1) by applying them
+// backwards to e_c (only H_j with j <= c touch it), with no barrier at all.
+// Same conventions as the blocked path: R (upper triangle, diagonal of either sign) overwrites G, Q is unsigned.
+template <int RM>
+__global__ void __launch_bounds__(8 * RM, 1)
+qr_small_kernel(float* __restrict__ G, int ld, int m, float* __restrict__ Q)
+{
+    constexpr int RPT = RM / 8;
+    extern __shared__ float qs_smem[];
+    float* Vs = qs_smem;                      // RM x RM: row j = reflector j over the rows
+    float* tau_s = qs_smem + RM * RM;
+    const int c = threadIdx.x >> 3, h = threadIdx.x & 7;
+    const unsigned gmask = 0xFFu << (threadIdx.x & 24);        // the eight lanes of this column
+    auto group_sum = [&](float v) {
+        v += __shfl_xor_sync(gmask, v, 1);
+        v += __shfl_xor_sync(gmask, v, 2);
+        v += __shfl_xor_sync(gmask, v, 4);
+        return v;
+    };
+    float x[RPT];
+#pragma unroll
+    for (int i = 0; i < RPT; ++i) {
+        const int r = h + 8 * i;
+        x[i] = (r < m && c < m) ? G[(size_t)r * ld + c] : 0.0f;
+    }
+    for (int j = 0; j < m; ++j) {
+        if (c == j) {
+            float s = 0.0f, a = 0.0f;
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) {
+                const int r = h + 8 * i;
+                s = fmaf((r > j) ? x[i] : 0.0f, x[i], s);
+                a += (r == j) ? x[i] : 0.0f;
+            }
+            const float sigma = group_sum(s), alpha = group_sum(a);
+            float beta = alpha, tau = 0.0f, scale = 0.0f;
+            if (sigma > 0.0f) {
+                beta = -copysignf(sqrtf(fmaf(alpha, alpha, sigma)), alpha);
+                tau = (beta - alpha) / beta;
+                scale = 1.0f / (alpha - beta);
+            }
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) {
+                const int r = h + 8 * i;
+                Vs[j * RM + r] = (r < j) ? 0.0f : ((r == j) ? 1.0f : x[i] * scale);
+                x[i] = (r < j) ? x[i] : ((r == j) ? beta : 0.0f);
+            }
+            if (h == 0) tau_s[j] = tau;
+        }
+        __syncthreads();
+        if (c > j && c < m) {
+            const float* v = Vs + j * RM + h;
+            float w = 0.0f;
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) w = fmaf(v[8 * i], x[i], w);            // v is zero above row j
+            const float tw = tau_s[j] * group_sum(w);
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) x[i] = fmaf(-tw, v[8 * i], x[i]);
+        }
+    }
+    if (c < m) {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+            const int r = h + 8 * i;
+            if (r < m) G[(size_t)r * ld + c] = x[i];
+        }
+    }
+    // ---- column c of Q ----
+    if (c < m) {
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) x[i] = (h + 8 * i == c) ? 1.0f : 0.0f;
+        for (int j = c; j >= 0; --j) {
+            const float* v = Vs + j * RM + h;
+            float w = 0.0f;
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) w = fmaf(v[8 * i], x[i], w);
+            const float tw = tau_s[j] * group_sum(w);
+#pragma unroll
+            for (int i = 0; i < RPT; ++i) x[i] = fmaf(-tw, v[8 * i], x[i]);
+        }
+#pragma unroll
+        for (int i = 0; i < RPT; ++i) {
+            const int r = h + 8 * i;
+            if (r < m) Q[(size_t)r * ld + c] = x[i];
+        }
+    }
+}
+
+template <int RM>
+int launch_qr_small_rm(gelo_ctx* ctx, int m, float* G, int ld, float* Q, cudaStream_t st)
+{
+    const int smem = (RM * RM + RM) * (int)sizeof(float);
+    static bool attr_done[64] = {};
+    if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
+        GELO_CUDA_OK(cudaFuncSetAttribute(qr_small_kernel<RM>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_done[ctx->device] = true;
+    }
+    qr_small_kernel<RM><<<1, 8 * RM, smem, st>>>(G, ld, m, Q);
+    return after_launch(ctx);
+}
+
+constexpr int kSmallQrRows = 128;
+
+int launch_qr_small(gelo_ctx* ctx, int m, float* G, int ld, float* Q, cudaStream_t st)
+{
+    if (m <= 32) return launch_qr_small_rm<32>(ctx, m, G, ld, Q, st);
+    if (m <= 64) return launch_qr_small_rm<64>(ctx, m, G, ld, Q, st);
+    if (m <= 96) return launch_qr_small_rm<96>(ctx, m, G, ld, Q, st);
+    return launch_qr_small_rm<128>(ctx, m, G, ld, Q, st);
+}
+
 }  // namespace
 
 size_t qr_scratch_bytes(int m, int ld)
@@ -508,6 +626,7 @@ QrScratch carve_qr(Arena& a, int m, int ld)
 
 int run_householder_qr(gelo_ctx* ctx, int m, float* R, int ld, float* Q, const QrScratch& s, cudaStream_t st)
 {
+    if (m <= kSmallQrRows && ctx->fuse_small) return launch_qr_small(ctx, m, R, ld, Q, st);
     const int npanels = ceil_div(m, NB);
     // ---- factorisation ----
     for (int pnl = 0; pnl < npanels; ++pnl) {
