@@ -297,8 +297,12 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
     } else if (warp == 1) {
         // ================= MMA issuer =================
         if (lane == 0) {
-            uint32_t it = 0, acc_it = 0;
+            uint32_t acc_it = 0;
+            uint32_t s = 0, ph = 0;                   // operand stage and the parity of its "full" phase
+            bool ready = false;                       // stage s is already known to be full (tested ahead, see tc_mma4_*_try)
             bool ok = true;
+            // k advance per instruction in sixteen-byte units of the descriptors' start address
+            constexpr uint64_t kAStep = kAMn ? (Cfg::kMnStep >> 4) : 2, kBStep = Cfg::kMnStep >> 4;
             for (int tile = blockIdx.x; tile < total_tiles && ok; tile += gridDim.x, ++acc_it) {
                 const int slice = prm.tri ? 0 : tile / mn_tiles;
                 int kb_total = 0;
@@ -314,24 +318,21 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                 if (!mbar_wait(acc_empty_bar(a), aph ^ 1u, abort_flag, prm.wait_ns)) { ok = false; break; }
                 tc_fence_after();
                 const uint32_t tmem_d = tmem_base + (uint32_t)(a * BN);
-                for (int kb = 0; kb < kb_total; ++kb, ++it) {
-                    const int s = it % kStages;
-                    const uint32_t ph = (it / kStages) & 1u;
-                    if (!mbar_wait(full_bar(s), ph, abort_flag, prm.wait_ns)) { ok = false; break; }
-                    tc_fence_after();
+                for (int kb = 0; kb < kb_total; ++kb) {
+                    if (!ready && !mbar_wait(full_bar(s), ph, abort_flag, prm.wait_ns)) { ok = false; break; }
                     const uint32_t sa = tiles_base + s * Cfg::kStageBytes;
                     const uint32_t sb = sa + kABytes;
-#pragma unroll
-                    for (int ks = 0; ks < 4; ++ks) {          // four instructions of 32 bytes of k (16 bf16 / 8 tf32) per stage
-                        // A K-major: 8-row groups 1024 bytes apart, 32 bytes per k step.  A MN-major: like B below.
-                        const uint64_t da = kAMn ? smem_desc(sa + ks * Cfg::kMnStep, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout)
-                                                 : smem_desc(sa + ks * 32, 16, 1024);
-                        // B: N-major, 128-byte-wide boxes kBoxBytes apart, k-row atoms kMnSbo bytes apart
-                        const uint64_t db = smem_desc(sb + ks * Cfg::kMnStep, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout);
-                        if (kTf32) tc_mma_tf32(tmem_d, da, db, prm.idesc, (kb | ks) != 0 ? 1u : 0u);
-                        else tc_mma_bf16(tmem_d, da, db, prm.idesc, (kb | ks) != 0 ? 1u : 0u);
-                    }
+                    // A K-major: 8-row groups 1024 bytes apart, 32 bytes per k step.  A MN-major: like B.
+                    const uint64_t da = kAMn ? smem_desc(sa, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout) : smem_desc(sa, 16, 1024);
+                    // B: N-major, 128-byte-wide boxes kBoxBytes apart, k-row atoms kMnSbo bytes apart
+                    const uint64_t db = smem_desc(sb, Cfg::kBoxBytes, Cfg::kMnSbo, Cfg::kMnLayout);
+                    const uint32_t ns = (s + 1 == kStages) ? 0u : s + 1;
+                    const uint32_t nph = (ns == 0u) ? (ph ^ 1u) : ph;
+                    // four instructions of 32 bytes of k (16 bf16 / 8 tf32) per stage
+                    ready = kTf32 ? tc_mma4_tf32_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph)
+                                  : tc_mma4_bf16_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph);
                     tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
+                    s = ns; ph = nph;
                 }
                 if (!ok) break;
                 tc_commit(acc_full_bar(a));           // accumulator complete

@@ -265,8 +265,9 @@ int launch_lu_panel(gelo_ctx* ctx, float* M, int ld, int m, int j0, int jb, int*
     // alone on the GPU: as many SMs as give every thread at least two rows; in a batch with many sampling lanes: as
     // few SMs as hold the panel (every SM it occupies is one that the other lanes' kernels cannot use)
     const int rows_per_thread = ctx->tc_update_ctas > 0 ? kMaxRowsPerThread : 2;
-    int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * rows_per_thread < rows) cs *= 2;
+    // (a cluster may have any size up to eight: five CTAs where four are too few, not eight)
+    int cs = ceil_div(rows, kPanelWarps * rows_per_thread);
+    if (cs > kClusterMax) cs = kClusterMax;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
     int* sd = ctx->status_dev;
     ProfScope ps(ctx, PROF_LU_PANEL, 1.0 * rows * (double)jb * jb, st);   // flops of the eliminations

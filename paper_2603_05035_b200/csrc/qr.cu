@@ -335,8 +335,9 @@ int launch_qr_panel(gelo_ctx* ctx, float* R, int ld, int m, int j0, int jb, floa
     // step); in a batch with many sampling lanes it packs up to 28 rows per thread and occupies as few SMs as
     // possible, since every SM it holds is one that the other lanes' kernels cannot use.
     const int rows_per_thread = ctx->tc_update_ctas > 0 ? kMaxRowsPerThread : 2;
-    int cs = 1;
-    while (cs < kClusterMax && cs * kPanelWarps * rows_per_thread < rows) cs *= 2;
+    // (a cluster may have any size up to eight: five CTAs where four are too few, not eight)
+    int cs = ceil_div(rows, kPanelWarps * rows_per_thread);
+    if (cs > kClusterMax) cs = kClusterMax;
     const int rpt = ceil_div(rows, cs * kPanelWarps);
     ProfScope ps(ctx, PROF_QR_PANEL, 2.0 * rows * (double)jb * jb, st);   // flops of the column dots and updates
     cudaError_t e;

@@ -101,6 +101,39 @@ __device__ __forceinline__ void tc_mma_tf32(uint32_t tmem_d, uint64_t desc_a, ui
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
 
+// The four MMA instructions of one operand stage (k advances by `astep` / `bstep` sixteen-byte units of the descriptors'
+// start address), with a barrier test tucked in front of them: the test of the NEXT stage's "full" barrier takes about
+// a hundred cycles to answer, and asked here its answer arrives while the four instructions issue instead of holding
+// up the next stage.  Returns whether that barrier phase had completed.
+#define GELO_TC_MMA4_TRY(KIND)                                                                                          \
+    uint32_t ready;                                                                                                     \
+    asm volatile(                                                                                                       \
+        "{\n\t.reg .pred q, p;\n\t"                                                                                    \
+        "mbarrier.try_wait.parity.shared::cta.b64 q, [%8], %9;\n\t"                                                     \
+        "setp.ne.b32 p, %7, 0;\n\t"                                                                                     \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%1], %2, %3, %6, p;\n\t"                                              \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%1], %4, %5, %6, 1;\n\t"                                              \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%1], %10, %11, %6, 1;\n\t"                                            \
+        "tcgen05.mma.cta_group::1.kind::" KIND " [%1], %12, %13, %6, 1;\n\t"                                            \
+        "selp.u32 %0, 1, 0, q;\n\t}"                                                                                    \
+        : "=r"(ready)                                                                                                   \
+        : "r"(tmem_d), "l"(da), "l"(db), "l"(da + astep), "l"(db + bstep), "r"(idesc), "r"(accumulate), "r"(next_bar),  \
+          "r"(next_parity), "l"(da + 2 * astep), "l"(db + 2 * bstep), "l"(da + 3 * astep), "l"(db + 3 * bstep)          \
+        : "memory");                                                                                                    \
+    return ready != 0;
+
+__device__ __forceinline__ bool tc_mma4_bf16_try(uint32_t tmem_d, uint64_t da, uint64_t db, uint64_t astep, uint64_t bstep,
+                                                 uint32_t idesc, uint32_t accumulate, uint32_t next_bar, uint32_t next_parity)
+{
+    GELO_TC_MMA4_TRY("f16")
+}
+__device__ __forceinline__ bool tc_mma4_tf32_try(uint32_t tmem_d, uint64_t da, uint64_t db, uint64_t astep, uint64_t bstep,
+                                                 uint32_t idesc, uint32_t accumulate, uint32_t next_bar, uint32_t next_parity)
+{
+    GELO_TC_MMA4_TRY("tf32")
+}
+#undef GELO_TC_MMA4_TRY
+
 __device__ __forceinline__ float round_tf32(float x)
 {
     uint32_t r;
