@@ -378,6 +378,37 @@ void oracle_shield_rows(int64_t n, int64_t d, int64_t k, const double* H, double
     for (int64_t i = 0; i < k * d; ++i) S[i] *= f;
 }
 
+/*
+ * Student-t shield rows (Section 4.4.1, Table 9 lists "Student-t" beside Gaussian shields without
+ * degrees of freedom or scaling; reading: nu is a parameter, the draws are standardised to unit
+ * variance so that the same global factor gives the same expected row energy as Gaussian shields).
+ * Element e owns B = 4 * ceil((nu + 1) / 4) consecutive positions of the Gaussian stream
+ * (seed, stream 2, attempt word = nu), starting at e * B:
+ *     t = g_0 / sqrt((g_1^2 + ... + g_nu^2) / nu),   x = t * sqrt((nu - 2) / nu),   3 <= nu <= 63.
+ */
+void oracle_student_t(uint64_t seed, uint32_t nu, uint64_t first, uint64_t count, double* out)
+{
+    const uint64_t B = 4u * (((uint64_t)nu + 1u + 3u) / 4u);
+    double g[64];
+    for (uint64_t i = 0; i < count; ++i) {
+        const uint64_t e = first + i;
+        oracle_gaussian(seed, 2u, nu, e * B, (uint64_t)nu + 1u, g);
+        double chi = 0.0;
+        for (uint32_t j = 1; j <= nu; ++j) chi += g[j] * g[j];
+        out[i] = g[0] / sqrt(chi / (double)nu) * sqrt(((double)nu - 2.0) / (double)nu);
+    }
+}
+
+/* S (k x d) = (scale * median row norm of H / sqrt(d)) * X, X standardised Student-t draws. */
+void oracle_shield_rows_t(int64_t n, int64_t d, int64_t k, const double* H, double scale,
+                          uint64_t seed, uint32_t nu, double* S)
+{
+    if (k <= 0) return;
+    const double f = scale * oracle_median_row_norm(n, d, H) / sqrt((double)d);
+    oracle_student_t(seed, nu, 0, (uint64_t)k * (uint64_t)d, S);
+    for (int64_t i = 0; i < k * d; ++i) S[i] *= f;
+}
+
 /* ------------------------------------------------------------------ */
 /* The chain (Eq. 1-3 with H_full = [H; S])                            */
 /* ------------------------------------------------------------------ */

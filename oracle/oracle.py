@@ -32,7 +32,7 @@ __all__ = [
     "ORTHOGONAL", "NONORTHOGONAL", "DEFAULT_GAMMA", "COND_BOUND", "build", "philox4x32_10",
     "philox_words", "gaussian", "matmul", "rows_times_w", "householder_qr", "lu_inverse",
     "singular_extremes", "cond2", "sample_mixing", "sample_mixing_verified", "median_row_norm",
-    "shield_rows", "chain", "direct", "rel_fro", "num_threads",
+    "shield_rows", "student_t", "shield_rows_t", "chain", "direct", "rel_fro", "num_threads",
 ]
 
 
@@ -215,6 +215,24 @@ def shield_rows(H, k, scale, seed):
     n, d = H.shape
     S = np.empty((int(k), d), dtype=np.float64)
     _load().oracle_shield_rows(_i64(n), _i64(d), _i64(k), _p(H), _dbl(scale), _u64(seed), _p(S))
+    return S
+
+
+def student_t(seed, nu, count, first=0):
+    """Standardised (unit-variance) Student-t draws with nu degrees of freedom, elements first..first+count-1."""
+    assert 3 <= int(nu) <= 63
+    out = np.empty(int(count), dtype=np.float64)
+    _load().oracle_student_t(_u64(seed), _u32(nu), _u64(first), _u64(count), _p(out))
+    return out
+
+
+def shield_rows_t(H, k, scale, seed, nu):
+    """S (k x d) = (scale * median row norm of H / sqrt(d)) * standardised Student-t draws (Table 9's other kind)."""
+    assert 3 <= int(nu) <= 63
+    H = _f64(H)
+    n, d = H.shape
+    S = np.empty((int(k), d), dtype=np.float64)
+    _load().oracle_shield_rows_t(_i64(n), _i64(d), _i64(k), _p(H), _dbl(scale), _u64(seed), _u32(nu), _p(S))
     return S
 
 

@@ -222,6 +222,40 @@ def test_median_row_norm_and_shields(oracle):
     assert oracle.shield_rows(H, 0, 10.0, seed=77).shape == (0, 4096)
 
 
+def test_student_t_shields(oracle):
+    """Student-t shield rows (Section 4.4.1, Table 9 names the kind): the distribution against scipy's, the
+    standardisation, the way an element is assembled from the pinned Gaussian stream, and the scaling rule."""
+    from scipy import stats
+    for nu in (3, 5, 10):
+        x = oracle.student_t(99, nu, 400_000)
+        t = x / np.sqrt((nu - 2.0) / nu)                      # undo the standardisation: plain t_nu
+        assert stats.kstest(t, stats.t(df=nu).cdf).pvalue > 1e-3
+        assert stats.kstest(x, "norm").pvalue < 1e-6          # and visibly not Gaussian: heavier tails
+        assert abs(np.mean(x)) < 0.01
+        if nu >= 5:
+            assert abs(np.var(x) - 1.0) < (0.03 if nu > 5 else 0.08)      # unit variance (slow convergence near nu = 4)
+    x10 = oracle.student_t(7, 10, 1_000_000)
+    assert abs(np.mean(x10**4) / np.var(x10)**2 - (3.0 + 6.0 / (10 - 4))) < 0.15      # kurtosis 3 + 6 / (nu - 4) = 4
+    # element e is built from positions e * B .. e * B + nu of the Gaussian stream (seed, stream 2, attempt = nu)
+    nu, B = 5, 8
+    g = oracle.gaussian(7, 2, nu, 1, 6 * B).ravel()
+    x = oracle.student_t(7, nu, 6)
+    for e in range(6):
+        blk = g[e * B: e * B + nu + 1]
+        want = blk[0] / np.sqrt(np.sum(blk[1:] ** 2) / nu) * np.sqrt((nu - 2.0) / nu)
+        assert x[e] == pytest.approx(want, rel=1e-13)
+    assert np.array_equal(oracle.student_t(7, nu, 3, first=2), x[2:5])
+    # the shield rows: one global factor scale * median / sqrt(d) on those draws, expected row energy as for Gaussian rows
+    rng = np.random.default_rng(6)
+    H = rng.standard_normal((64, 4096))
+    H /= np.sqrt((H * H).mean(axis=1, keepdims=True))
+    S = oracle.shield_rows_t(H, 6, 10.0, seed=77, nu=8)
+    med = np.median(np.linalg.norm(H, axis=1))
+    assert np.allclose(S, (10.0 * med / 64.0) * oracle.student_t(77, 8, 6 * 4096).reshape(6, 4096), rtol=1e-14)
+    assert np.allclose(np.linalg.norm(S, axis=1), 10.0 * med, rtol=0.15)
+    assert oracle.shield_rows_t(H, 0, 10.0, seed=77, nu=8).shape == (0, 4096)
+
+
 # --------------------------------------------------------------------------
 # What the paper fixes (Section 3.2 and its Gram-leak discussion)
 # --------------------------------------------------------------------------
