@@ -409,6 +409,58 @@ void oracle_shield_rows_t(int64_t n, int64_t d, int64_t k, const double* H, doub
     for (int64_t i = 0; i < k * d; ++i) S[i] *= f;
 }
 
+/*
+ * FP8 operands for the offloaded product (the paper's Limitations / Future Work name FP8 beside FP16;
+ * reading: the product of Eq. 2, the one the untrusted accelerator runs, takes U and W in the OCP
+ * 8-bit format E4M3 -- sign, 4 exponent bits with bias 7, 3 mantissa bits, no infinities, largest
+ * finite value 448, subnormals down to 2^-9 -- with ONE fp32 scale per tensor, s = max|x| / 448,
+ * code = round-to-nearest-even(x / s) with the division in binary32, and Y' = (s_U s_W) (U8 W8)).
+ */
+double oracle_e4m3_decode(uint8_t code)
+{
+    const int sign = code >> 7, e = (code >> 3) & 15, f = code & 7;
+    double v;
+    if (e == 15 && f == 7) v = NAN;                               /* the one NaN pattern per sign */
+    else if (e == 0) v = ldexp((double)f, -9);                    /* subnormal: f * 2^-3 * 2^-6 */
+    else v = ldexp(1.0 + (double)f / 8.0, e - 7);
+    return sign ? -v : v;
+}
+
+/* Nearest E4M3 value to x (ties to the even mantissa), saturating at +-448. */
+uint8_t oracle_e4m3_encode(float x)
+{
+    const uint8_t sign = signbit(x) ? 0x80u : 0u;
+    double a = fabs((double)x);
+    if (isnan(a)) return (uint8_t)(sign | 0x7Fu);
+    if (a >= 448.0) return (uint8_t)(sign | 0x7Eu);               /* 448 = 1.75 * 2^8 */
+    /* spacing of the representable values around a: 2^(e-3) for normals (e >= -6), 2^-9 below 2^-6 */
+    int e;
+    frexp(a, &e);                                                  /* a = m * 2^e, 0.5 <= m < 1  ->  exponent e - 1 */
+    int ex = e - 1;
+    if (ex < -6) ex = -6;
+    const double q = ldexp(1.0, ex - 3);
+    double n = nearbyint(a / q);                                   /* default rounding mode: ties to even */
+    double r = n * q;
+    if (r >= 448.0) return (uint8_t)(sign | 0x7Eu);
+    if (r == 0.0) return sign;
+    int e2;
+    const double m2 = frexp(r, &e2);                               /* r = m2 * 2^e2 */
+    int ex2 = e2 - 1;
+    if (ex2 < -6) return (uint8_t)(sign | (uint8_t)nearbyint(r / ldexp(1.0, -9)));
+    const int f = (int)nearbyint((m2 * 2.0 - 1.0) * 8.0);
+    return (uint8_t)(sign | ((ex2 + 7) << 3) | f);
+}
+
+/* scale = max|x| / 448 in binary32 (1 if the tensor is all zero); codes[i] = encode(x[i] / scale), binary32 division */
+float oracle_quantize_e4m3(int64_t count, const float* x, uint8_t* codes)
+{
+    float amax = 0.0f;
+    for (int64_t i = 0; i < count; ++i) { const float a = fabsf(x[i]); if (a > amax) amax = a; }
+    const float scale = amax > 0.0f ? amax / 448.0f : 1.0f;
+    for (int64_t i = 0; i < count; ++i) codes[i] = oracle_e4m3_encode(x[i] / scale);
+    return scale;
+}
+
 /* ------------------------------------------------------------------ */
 /* The chain (Eq. 1-3 with H_full = [H; S])                            */
 /* ------------------------------------------------------------------ */

@@ -32,7 +32,7 @@ __all__ = [
     "ORTHOGONAL", "NONORTHOGONAL", "DEFAULT_GAMMA", "COND_BOUND", "build", "philox4x32_10",
     "philox_words", "gaussian", "matmul", "rows_times_w", "householder_qr", "lu_inverse",
     "singular_extremes", "cond2", "sample_mixing", "sample_mixing_verified", "median_row_norm",
-    "shield_rows", "student_t", "shield_rows_t", "chain", "direct", "rel_fro", "num_threads",
+    "shield_rows", "student_t", "shield_rows_t", "e4m3_decode", "e4m3_encode", "quantize_e4m3", "project_e4m3", "chain", "direct", "rel_fro", "num_threads",
 ]
 
 
@@ -54,6 +54,11 @@ def _load():
         build()
         lib = ctypes.CDLL(_LIB)
         lib.oracle_median_row_norm.restype = ctypes.c_double
+        lib.oracle_e4m3_decode.restype = ctypes.c_double
+        lib.oracle_e4m3_decode.argtypes = [ctypes.c_uint8]
+        lib.oracle_e4m3_encode.restype = ctypes.c_uint8
+        lib.oracle_e4m3_encode.argtypes = [ctypes.c_float]
+        lib.oracle_quantize_e4m3.restype = ctypes.c_float
         for name in ("oracle_householder_qr", "oracle_lu_inverse", "oracle_singular_extremes",
                      "oracle_sample_mixing", "oracle_chain"):
             getattr(lib, name).restype = ctypes.c_int
@@ -234,6 +239,33 @@ def shield_rows_t(H, k, scale, seed, nu):
     S = np.empty((int(k), d), dtype=np.float64)
     _load().oracle_shield_rows_t(_i64(n), _i64(d), _i64(k), _p(H), _dbl(scale), _u64(seed), _u32(nu), _p(S))
     return S
+
+
+def e4m3_decode(codes):
+    """Values (float64) of an array of E4M3 codes (uint8)."""
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    table = np.array([_load().oracle_e4m3_decode(c) for c in range(256)], dtype=np.float64)
+    return table[codes]
+
+
+def e4m3_encode(x):
+    """Nearest E4M3 code (ties to even, saturating at 448) of every element of a float32 array."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    L = _load()
+    return np.array([L.oracle_e4m3_encode(float(v)) for v in x.ravel()], dtype=np.uint8).reshape(x.shape)
+
+
+def quantize_e4m3(x):
+    """Per-tensor quantisation: (codes uint8, scale float32) with scale = max|x| / 448, codes = encode(x / scale)."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    codes = np.empty(x.shape, dtype=np.uint8)
+    scale = _load().oracle_quantize_e4m3(_i64(x.size), _p(x), _p(codes))
+    return codes, np.float32(scale)
+
+
+def project_e4m3(u_codes, u_scale, w_codes, w_scale):
+    """Y' = (s_U s_W) (U8 W8): the offloaded product of Eq. 2 on E4M3 operands, exact in fp64."""
+    return float(u_scale) * float(w_scale) * matmul(e4m3_decode(u_codes), e4m3_decode(w_codes))
 
 
 def chain(A, Ainv, H, S, W, want_intermediates=False):

@@ -256,6 +256,48 @@ def test_student_t_shields(oracle):
     assert oracle.shield_rows_t(H, 0, 10.0, seed=77, nu=8).shape == (0, 4096)
 
 
+def test_e4m3_format_and_quantiser(oracle):
+    """The 8-bit format of the FP8 projection: every code against torch's float8_e4m3fn (an independent implementation of
+    the OCP format), rounding against torch's cast, and the per-tensor scale rule."""
+    import torch
+    codes = np.arange(256, dtype=np.uint8)
+    ours = oracle.e4m3_decode(codes)
+    theirs = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    assert np.array_equal(np.isnan(ours), np.isnan(theirs)) and np.isnan(ours).sum() == 2
+    assert np.array_equal(ours[~np.isnan(ours)], theirs[~np.isnan(theirs)])
+    assert np.nanmax(ours) == 448.0 and np.min(ours[ours > 0]) == 2.0 ** -9
+    # encode: decode(encode(v)) == v for every finite code, and nearest-even rounding agrees with torch's cast
+    finite = ~np.isnan(ours)
+    back = oracle.e4m3_encode(ours[finite].astype(np.float32))
+    assert np.array_equal(oracle.e4m3_decode(back), ours[finite])
+    rng = np.random.default_rng(8)
+    x = np.concatenate([rng.standard_normal(20000) * 50, rng.standard_normal(20000) * 0.01, rng.uniform(-448, 448, 20000),
+                        (ours[finite][:-1] + ours[finite][1:]) / 2]).astype(np.float32)        # incl. exact midpoints
+    x = x[np.abs(x) <= 448.0]
+    want = torch.from_numpy(x.copy()).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = oracle.e4m3_encode(x)
+    same = oracle.e4m3_decode(got) == oracle.e4m3_decode(want)           # (+0 and -0 compare equal)
+    assert same.all()
+    assert oracle.e4m3_decode(oracle.e4m3_encode(np.float32([1e9, -1e9, 500.0]))).tolist() == [448.0, -448.0, 448.0]
+    # per-tensor scale: the largest magnitude lands on +-448, relative error of a normal value at most 2^-4
+    t = (rng.standard_normal((64, 96)) * 3).astype(np.float32)
+    c, s = oracle.quantize_e4m3(t)
+    assert s == np.float32(np.abs(t).max()) / np.float32(448.0)
+    deq = oracle.e4m3_decode(c) * float(s)
+    assert np.abs(deq).max() == pytest.approx(np.abs(t).max(), rel=1e-6)
+    big = np.abs(t) > np.abs(t).max() * 2.0 ** -8                          # values that stay normal after scaling
+    assert np.max(np.abs(deq[big] - t[big]) / np.abs(t[big])) <= 2.0 ** -4 + 1e-6
+    cz, sz = oracle.quantize_e4m3(np.zeros((3, 5), dtype=np.float32))
+    assert sz == 1.0 and not cz.any()
+    # the product on quantised operands against numpy on the decoded values
+    u, w = rng.standard_normal((7, 40)).astype(np.float32), rng.standard_normal((40, 9)).astype(np.float32)
+    (uc, us), (wc, ws) = oracle.quantize_e4m3(u), oracle.quantize_e4m3(w)
+    ref = (oracle.e4m3_decode(uc) * float(us)) @ (oracle.e4m3_decode(wc) * float(ws))
+    assert np.allclose(oracle.project_e4m3(uc, us, wc, ws), ref, rtol=1e-12, atol=1e-12)
+    # and it approximates the unquantised product to a few percent (3 mantissa bits per operand)
+    assert oracle.rel_fro(oracle.project_e4m3(uc, us, wc, ws), u.astype(np.float64) @ w.astype(np.float64)) < 0.08
+
+
 # --------------------------------------------------------------------------
 # What the paper fixes (Section 3.2 and its Gram-leak discussion)
 # --------------------------------------------------------------------------
