@@ -180,6 +180,16 @@ int gelo_sample_mixing(gelo_ctx* ctx, int m, int kind, uint64_t seed, int dtype,
 int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale,
                      uint64_t seed, int dtype, void* S_dev, void* stream);
 
+/* The other shield kind the paper's attack study lists (Section 4.4.1, Table 9: "Student-t"; it gives neither the
+ * degrees of freedom nor a scaling, so both are read as follows).  S_dev (k x d) = (scale * median_i ||H_i||_2 /
+ * sqrt(d)) * x, with x standardised Student-t draws of `nu` degrees of freedom (3 <= nu <= 63, unit variance, so the
+ * expected row energy is that of the Gaussian kind): element e owns B = 4 ceil((nu + 1) / 4) consecutive positions of
+ * the Gaussian stream (seed, stream 2, attempt word nu) from e * B on, t = g_0 / sqrt((g_1^2 + .. + g_nu^2) / nu),
+ * x = t sqrt((nu - 2) / nu).  gelo_set_shield_student_t makes the whole-call entry points draw this kind (0 = Gaussian). */
+int gelo_shield_rows_t(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale, uint64_t seed, int nu,
+                       int dtype, void* S_dev, void* stream);
+int gelo_set_shield_student_t(gelo_ctx* ctx, int nu);
+
 /* gelo_shield_rows for callers that cannot allocate device memory, and so cannot give the
  * context a workspace: a component loaded into a process whose memory pool belongs to someone
  * else (a serving engine's plugin, a confidential-computing runtime with a frozen allocator),
@@ -209,6 +219,23 @@ int gelo_mix(gelo_ctx* ctx, const void* A_dev, int lda, const void* H_dev, const
  * also the plain, unprotected projection. */
 int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int d, int p,
                  int dtype, void* Yp_dev, void* stream);
+
+/* FP8 operands for the offloaded product (the paper's Limitations and Future Work name FP8 beside FP16; reading: the
+ * product of Eq. 2, the one that runs on the untrusted accelerator, takes its operands in the OCP format E4M3 with one
+ * fp32 scale per tensor, while mixing and unmixing stay in the 16-bit type).
+ *   gelo_quantize_e4m3: codes_dev (rows x cols bytes, dense) = nearest-even E4M3 of X_dev / scale (binary32 division,
+ *       saturating at +-448), scale = max|X| / 448 (1 for an all-zero tensor) written to scale_dev[0]; scale_dev must hold
+ *       TWO floats (the second is scratch) and be 8-byte aligned.  X_dev: rows x cols of `dtype`, dense, cols a multiple
+ *       of 16.  Weights are quantised once and reused; U is quantised per call.
+ *   gelo_project_e4m3: Yp_dev (m x p bf16) = (u_scale * w_scale) * (U8 (m x d) * W8 (d x p)), fp32 accumulation on the
+ *       tensor cores (kind::f8f6f4).  d and p multiples of 16.
+ * With 3 mantissa bits per operand the product carries about 5% relative error (rms) against the unquantised one, and the
+ * 10x shield rows bring 6x the energy of the data into Y', so after unmixing the data rows see about 12%: this path is
+ * for callers that accept FP8-grade accuracy, and is checked against the fp64 product of the SAME stored codes. */
+int gelo_quantize_e4m3(gelo_ctx* ctx, const void* X_dev, int rows, int cols, int dtype, void* codes_dev, float* scale_dev,
+                       void* stream);
+int gelo_project_e4m3(gelo_ctx* ctx, const void* U8_dev, const float* u_scale_dev, const void* W8_dev, const float* w_scale_dev,
+                      int m, int d, int p, void* Yp_dev, void* stream);
 
 /* Rows 0..n-1 of Ainv * Yp (shield rows are dropped by never computing them), split by
  * column thirds into Q_dev, K_dev, V_dev (each n x p/3; p % 3 == 0 and p/3 % 8 == 0).  If

@@ -51,9 +51,13 @@ EXPORTS = {
     "gelo_sample_mixing": (_i, [_vp, _i, _i, _u64, _i, _vp, _vp, _i, _vp, _vp]),
     "gelo_shield_rows": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
     "gelo_shield_rows_static": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _vp, _vp]),
+    "gelo_shield_rows_t": (_i, [_vp, _vp, _i, _i, _i, _f, _u64, _i, _i, _vp, _vp]),
+    "gelo_set_shield_student_t": (_i, [_vp, _i]),
     "gelo_mix": (_i, [_vp, _vp, _i, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_project": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _vp, _vp]),
     "gelo_unmix": (_i, [_vp, _vp, _i, _vp, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
+    "gelo_quantize_e4m3": (_i, [_vp, _vp, _i, _i, _i, _vp, _vp, _vp]),
+    "gelo_project_e4m3": (_i, [_vp, _vp, _vp, _vp, _vp, _i, _i, _i, _vp, _vp]),
     "gelo_qkv_offload": (_i, [_vp, _vp, _vp, _i, _i, _i, _i, _i, _u64, _f, _i, _vp, _vp, _vp, _vp]),
     "gelo_project_unmix": (_i, [_vp, _vp, _vp, _vp, _i, _i, _i, _i, _i, _i, _vp, _vp, _vp, _vp]),
     "gelo_set_small_batch_fusion": (_i, [_vp, _i]),
@@ -264,6 +268,15 @@ class Context:
         self._check(self._lib.gelo_shield_rows(self._h, _ptr(H), n, d, k, scale, seed, dtype_code(dtype),
                                                _ptr(S), _stream(stream)), "gelo_shield_rows")
 
+    def shield_rows_t(self, H, n, d, k, scale, seed, nu, dtype, S, stream=None):
+        """Student-t shield rows with nu degrees of freedom (standardised to unit variance)."""
+        self._check(self._lib.gelo_shield_rows_t(self._h, _ptr(H), n, d, k, scale, seed, nu, dtype_code(dtype),
+                                                 _ptr(S), _stream(stream)), "gelo_shield_rows_t")
+
+    def set_shield_student_t(self, nu: int):
+        """Shield kind of the whole-call entry points: 0 Gaussian, else Student-t with nu degrees of freedom."""
+        self._check(self._lib.gelo_set_shield_student_t(self._h, nu), "gelo_set_shield_student_t")
+
     def shield_rows_static(self, H, n, d, k, scale, seed, dtype, S, stream=None):
         """Shield rows for callers that cannot allocate: scratch lives inside the library (n <= 65536)."""
         self._check(self._lib.gelo_shield_rows_static(self._h, _ptr(H), n, d, k, scale, seed, dtype_code(dtype),
@@ -276,6 +289,16 @@ class Context:
     def project(self, U, W, m, d, p, dtype, Yp, stream=None):
         self._check(self._lib.gelo_project(self._h, _ptr(U), _ptr(W), m, d, p, dtype_code(dtype), _ptr(Yp),
                                            _stream(stream)), "gelo_project")
+
+    def quantize_e4m3(self, X, rows, cols, dtype, codes, scale, stream=None):
+        """codes (uint8, rows x cols) and scale (two floats: the scale and a scratch slot) from X."""
+        self._check(self._lib.gelo_quantize_e4m3(self._h, _ptr(X), rows, cols, dtype_code(dtype), _ptr(codes), _ptr(scale),
+                                                 _stream(stream)), "gelo_quantize_e4m3")
+
+    def project_e4m3(self, U8, u_scale, W8, w_scale, m, d, p, Yp, stream=None):
+        """Yp (bf16) = u_scale * w_scale * (U8 @ W8) on E4M3 operands."""
+        self._check(self._lib.gelo_project_e4m3(self._h, _ptr(U8), _ptr(u_scale), _ptr(W8), _ptr(w_scale), m, d, p, _ptr(Yp),
+                                                _stream(stream)), "gelo_project_e4m3")
 
     def unmix(self, Ainv, lda, Yp, n, k, p, dtype, Q, K=None, V=None, stream=None):
         self._check(self._lib.gelo_unmix(self._h, _ptr(Ainv), lda, _ptr(Yp), n, k, p, dtype_code(dtype),

@@ -274,7 +274,7 @@ int offload_impl(gelo_ctx* ctx, const Layout& L, const void* H, const void* W, i
 {
     const int m = n + k;
     GELO_TRY(sample_mixing_impl(ctx, L, m, kind, seed, dtype, L.A, L.Ainv, L.ldi, nullptr, st));
-    GELO_TRY(run_shield_rows(ctx, H, n, d, k, shield_scale, seed, dtype, L.S, L.sh, st));
+    GELO_TRY(run_shield_rows(ctx, H, n, d, k, shield_scale, seed, dtype, L.S, L.sh, st, ctx->shield_nu));
     GELO_TRY(mix_impl(ctx, L.A, L.ldi, H, k > 0 ? L.S : nullptr, n, k, d, dtype, L.U, st, &L.t3));
     return project_and_unmix(ctx, L.U, W, L.Ainv, L.ldi, L.Yp, n, k, d, p, dtype, Q, K, V, st, &L.t3);
 }
@@ -407,7 +407,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
             Hi = hd;
             Qi = y; Ki = split ? y + third : nullptr; Vi = split ? y + 2 * third : nullptr;
         }
-        GELO_TRY(run_shield_rows(ctx, Hi, n, d, k, shield_scale, seeds[i], dtype, L[0].S, L[0].sh, st));
+        GELO_TRY(run_shield_rows(ctx, Hi, n, d, k, shield_scale, seeds[i], dtype, L[0].S, L[0].sh, st, ctx->shield_nu));
         GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
         if (host) GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->y_free[b], 0));
         GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, Hi, k > 0 ? L[0].S : nullptr, n, k, d, dtype, L[0].U, st, &L[0].t3));
@@ -530,7 +530,7 @@ int offload_blockdiag_impl(gelo_ctx* ctx, int calls, const void* const* H, const
     for (long long v = 0; v < total && v < D; ++v) GELO_TRY(enqueue_sample(v));
     for (int c = 0; c < calls; ++c) {
         const char* Hc = static_cast<const char*>(H[c]);
-        GELO_TRY(run_shield_rows(ctx, Hc, n, d, k, shield_scale, seeds[c], dtype, S, sh, st));
+        GELO_TRY(run_shield_rows(ctx, Hc, n, d, k, shield_scale, seeds[c], dtype, S, sh, st, ctx->shield_nu));
         for (int j = 0; j < P.nb; ++j) {
             const int l = (int)(((long long)c * P.nb + j) % D);
             const int u0 = P.d0[j] + P.s0[j];
@@ -831,6 +831,31 @@ int gelo_shield_rows(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, floa
     return run_shield_rows(ctx, H_dev, n, d, k, scale, seed, dtype, S_dev, sh, as_stream(stream));
 }
 
+int gelo_shield_rows_t(gelo_ctx* ctx, const void* H_dev, int n, int d, int k, float scale, uint64_t seed, int nu,
+                       int dtype, void* S_dev, void* stream)
+{
+    if (!ctx || n <= 0 || d <= 0 || k < 0 || bad_dtype(dtype) || (d % 8) != 0 || !H_dev || misaligned(H_dev) || nu < 3 || nu > 63)
+        return GELO_ERR_INVALID;
+    if (k == 0) return GELO_OK;
+    if (!S_dev || misaligned(S_dev)) return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    if (!ctx->ws) return GELO_ERR_WORKSPACE;
+    Arena a;
+    a.base = static_cast<char*>(ctx->ws);
+    a.cap = ctx->ws_bytes;
+    ShieldScratch sh = carve_shield(a, n);
+    if (!a.ok) return GELO_ERR_WORKSPACE;
+    ctx->chain_valid = false;
+    return run_shield_rows(ctx, H_dev, n, d, k, scale, seed, dtype, S_dev, sh, as_stream(stream), nu);
+}
+
+int gelo_set_shield_student_t(gelo_ctx* ctx, int nu)
+{
+    if (!ctx || (nu != 0 && (nu < 3 || nu > 63))) return GELO_ERR_INVALID;
+    ctx->shield_nu = nu;
+    return GELO_OK;
+}
+
 int gelo_mix(gelo_ctx* ctx, const void* A_dev, int lda, const void* H_dev, const void* S_dev, int n, int k,
              int d, int dtype, void* U_dev, void* stream)
 {
@@ -851,6 +876,26 @@ int gelo_project(gelo_ctx* ctx, const void* U_dev, const void* W_dev, int m, int
     DeviceGuard guard(ctx->device);
     Layout L;
     return project_impl(ctx, U_dev, W_dev, m, d, p, dtype, Yp_dev, as_stream(stream), stage_pairs(ctx, m, 0, d, p, dtype, &L));
+}
+
+int gelo_quantize_e4m3(gelo_ctx* ctx, const void* X_dev, int rows, int cols, int dtype, void* codes_dev, float* scale_dev,
+                       void* stream)
+{
+    if (!ctx || rows <= 0 || cols <= 0 || (cols % 16) != 0 || bad_dtype(dtype) || !X_dev || !codes_dev || !scale_dev ||
+        misaligned(X_dev) || misaligned(codes_dev) || (reinterpret_cast<uintptr_t>(scale_dev) & 7u))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return launch_quantize_e4m3(ctx, X_dev, rows, cols, cols, dtype, codes_dev, cols, scale_dev, as_stream(stream));
+}
+
+int gelo_project_e4m3(gelo_ctx* ctx, const void* U8_dev, const float* u_scale_dev, const void* W8_dev, const float* w_scale_dev,
+                      int m, int d, int p, void* Yp_dev, void* stream)
+{
+    if (!ctx || m <= 0 || d <= 0 || p <= 0 || (d % 16) != 0 || (p % 16) != 0 || !U8_dev || !W8_dev || !u_scale_dev ||
+        !w_scale_dev || !Yp_dev || misaligned(U8_dev) || misaligned(W8_dev) || misaligned(Yp_dev))
+        return GELO_ERR_INVALID;
+    DeviceGuard guard(ctx->device);
+    return launch_gemm_e4m3(ctx, m, p, d, U8_dev, d, W8_dev, p, u_scale_dev, w_scale_dev, Yp_dev, p, as_stream(stream));
 }
 
 int gelo_unmix(gelo_ctx* ctx, const void* Ainv_dev, int lda, const void* Yp_dev, int n, int k, int p, int dtype,

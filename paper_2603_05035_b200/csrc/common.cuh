@@ -60,6 +60,7 @@ struct gelo_ctx {
     long long launches = 0;
     unsigned long long wait_limit_ns = 2000000000ull;   // limit of every device-side barrier wait (gelo_set_wait_limit_ns)
     void* tmap_encode = nullptr;  // cuTensorMapEncodeTiled, resolved at creation
+    int shield_nu = 0;            // shield rows of the whole-call entry points: 0 Gaussian, else Student-t with this many degrees of freedom
     bool fuse_small = true;       // calls with m <= 128 run projection and unmixing as one kernel (gelo_set_small_batch_fusion)
     int dec_group = 16;           // CTAs of the small-batch projection kernel that walk the k-blocks in step (0: all of them)
     bool tma_3d = true;           // N-major operand tiles as one three-dimensional TMA box where the layout allows
@@ -176,6 +177,11 @@ int launch_gram_sym_bf16(gelo_ctx*, int m, const float* Q, int ld, void* D, int 
 // C (fp32) -= A (bf16) B (bf16), in place
 int launch_gemm_bf16_sub(gelo_ctx*, int M, int N, int K, const void* A, int lda, const void* B, int ldb, float* C, int ldc,
                          cudaStream_t);
+// ---- E4M3 operands for the offloaded product (fp8.cu, gemm_tc.cu) ----
+int launch_quantize_e4m3(gelo_ctx*, const void* x, int rows, int cols, int ld, int dtype, void* out, int ldo, float* scale,
+                         cudaStream_t);
+int launch_gemm_e4m3(gelo_ctx*, int M, int N, int K, const void* A8, int lda, const void* B8, int ldb, const float* sa,
+                     const float* sb, void* C, int ldc, cudaStream_t);
 // The tensor core drops the 13 low mantissa bits of an fp32 operand instead of rounding them.  For values whose
 // mantissas are spread log-uniformly that loses 2^-11 / (2 ln 2) of the magnitude on average, coherently over all
 // terms of a product; a result whose operand was truncated is scaled back by 1 + kTf32TruncLoss per such operand,
@@ -337,7 +343,8 @@ struct ShieldScratch {
     float* med = nullptr;     // 2
 };
 ShieldScratch carve_shield(Arena&, int n);
+// nu = 0: Gaussian rows; 3 <= nu <= 63: standardised Student-t rows with nu degrees of freedom
 int run_shield_rows(gelo_ctx*, const void* H, int n, int d, int k, float scale, uint64_t seed,
-                    int dtype, void* S, const ShieldScratch&, cudaStream_t);
+                    int dtype, void* S, const ShieldScratch&, cudaStream_t, int nu = 0);
 
 }  // namespace gelo

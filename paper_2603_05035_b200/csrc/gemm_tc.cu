@@ -62,6 +62,8 @@ struct TcParams {
     float post_scale;               //   ... and the factor applied after that: out = post_scale * (out_scale * acc - diag_sub [row == col])
     int a3d, b3d;                   // the MN-major A tile / the B tile arrives as ONE three-dimensional box (see make_map_nmajor)
     int out_f16;                    // TC_STORE_BF16: operands and output are IEEE half instead of bfloat16
+    const float* scale_a;           // TC_STORE_BF16 with 8-bit operands: the per-tensor scales (device scalars); the
+    const float* scale_b;           //   accumulator is multiplied by their product before it is rounded
     int tri, tri_tiles;             // TC_STORE_SYM16: the result is symmetric; only the tri_tiles tiles that reach the diagonal or lie
                                     // above it are computed, and what lies below them is filled in by mirroring
     uint32_t idesc;                 // instruction descriptor (filled in by the launcher)
@@ -78,27 +80,28 @@ constexpr uint32_t kStagingBytes = kEpiWarps * 2 * kStageBoxBytes;
 // the shared-memory geometry: kTf32 only changes the element count per k-block, the box width of the N-major B tile
 // (128 bytes = 64 bf16 or 32 fp32 columns) and the instruction.  kAMn (tf32 only): the A tile arrives as four
 // boxes of 32 m-columns x 32 k-rows, i.e. laid out exactly like a 128-column B tile.
-template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false>
+template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false, bool kF8 = false>
 struct TcCfg {
     static constexpr uint32_t kStagingUsed = kStaging ? kStagingBytes : 0u;
-    static constexpr int kBKE = kTf32 ? 32 : 64;                           // elements of k per stage
-    static constexpr int kBoxCols = kTf32 ? 32 : 64;                       // columns of one N-major box (128 bytes)
+    static constexpr int kBKE = kF8 ? 128 : (kTf32 ? 32 : 64);             // elements of k per stage
+    static constexpr int kBoxCols = kF8 ? 128 : (kTf32 ? 32 : 64);         // columns of one N-major box (128 bytes)
     static constexpr uint32_t kBoxBytes = (uint32_t)kBKE * 128u;           // one N-major box: kBKE rows of 128 bytes
     static constexpr uint32_t kBBytes = (BN / kBoxCols) * kBoxBytes;
     static constexpr uint32_t kStageBytes = kABytes + kBBytes;
     static constexpr uint32_t kSmemBytes = kStages * kStageBytes + kStagingUsed + 1024 /*alignment slack*/ + 256 /*barriers*/;
     // k advance per instruction inside an N-major (or MN-major A) tile: 16 bf16 rows or 8 tf32 rows of 128 bytes
-    static constexpr uint32_t kMnStep = kTf32 ? 1024u : 2048u;
+    static constexpr uint32_t kMnStep = kF8 ? 4096u : (kTf32 ? 1024u : 2048u);   // 32 e4m3 rows, 16 bf16 rows or 8 tf32 rows
     // N-major tiles: bf16 in the 16-byte-chunk swizzle (atoms of 8 k-rows, 1024 bytes), fp32 in the 32-byte-chunk
     // swizzle (atoms of 4 k-rows, 512 bytes)
     static constexpr uint32_t kMnLayout = kTf32 ? 1u : 2u;
     static constexpr uint32_t kMnSbo = kTf32 ? 512u : 1024u;
     // Instruction descriptor: fp32 accumulate, operand formats (1 = bf16, 2 = tf32), A K-major or MN-major,
     // B N-major, M = 128, N = BN.
-    static constexpr uint32_t kFmt = kTf32 ? 2u : 1u;
+    static constexpr uint32_t kFmt = kF8 ? 0u : (kTf32 ? 2u : 1u);         // kind::f8f6f4: 0 = E4M3
     static constexpr uint32_t kInstrDesc = (1u << 4) | (kFmt << 7) | (kFmt << 10) | ((kAMn ? 1u : 0u) << 15) | (1u << 16) |
                                            ((uint32_t)(BN >> 3) << 17) | ((uint32_t)(BM >> 4) << 24);
     static_assert(!kAMn || kTf32, "MN-major A is only wired up for the tf32 kind");
+    static_assert(!(kF8 && kTf32), "one operand kind per instance");
 };
 
 // x = hi + lo with hi = bf16(x), lo = bf16(x - hi)
@@ -141,9 +144,16 @@ __device__ __forceinline__ void epilogue_group(const TcParams& prm, int gm, int 
     const uint32_t v[8] = {w[G * 8 + 0], w[G * 8 + 1], w[G * 8 + 2], w[G * 8 + 3],
                            w[G * 8 + 4], w[G * 8 + 5], w[G * 8 + 6], w[G * 8 + 7]};
     if (prm.mode == TC_STORE_BF16) {
+        const uint32_t (&v0)[8] = v;
         const int chunk = gn / prm.csplit;
         void* base = chunk == 0 ? prm.C0 : (chunk == 1 ? prm.C1 : prm.C2);
         const size_t off = (size_t)gm * prm.ldc + (gn - chunk * prm.csplit);
+        uint32_t v[8] = {v0[0], v0[1], v0[2], v0[3], v0[4], v0[5], v0[6], v0[7]};
+        if (prm.scale_a) {
+            const float sc = prm.scale_a[0] * prm.scale_b[0];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = __float_as_uint(sc * __uint_as_float(v[j]));
+        }
         uint4 pk;
         if (prm.out_f16) {
             pk.x = pack_f16(v[0], v[1]); pk.y = pack_f16(v[2], v[3]);
@@ -200,13 +210,13 @@ __device__ __forceinline__ void store_symmetric(const TcParams& prm, int gm, int
     }
 }
 
-template <int BN, int kStages, bool kStaging, bool kTf32, bool kAMn>
+template <int BN, int kStages, bool kStaging, bool kTf32, bool kAMn, bool kF8>
 __global__ void __launch_bounds__(kThreads, 1)
 gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant__ CUtensorMap map_a1,
                const __grid_constant__ CUtensorMap map_b0, const __grid_constant__ CUtensorMap map_b1,
                const __grid_constant__ CUtensorMap map_c, const TcParams prm)
 {
-    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn>;
+    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn, kF8>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t tiles_base = (raw + 1023u) & ~1023u;                 // swizzle atoms need 1024-byte alignment
@@ -329,7 +339,8 @@ gemm_tc_kernel(const __grid_constant__ CUtensorMap map_a0, const __grid_constant
                     const uint32_t ns = (s + 1 == kStages) ? 0u : s + 1;
                     const uint32_t nph = (ns == 0u) ? (ph ^ 1u) : ph;
                     // four instructions of 32 bytes of k (16 bf16 / 8 tf32) per stage
-                    ready = kTf32 ? tc_mma4_tf32_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph)
+                    ready = kF8 ? tc_mma4_f8_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph)
+                          : kTf32 ? tc_mma4_tf32_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph)
                                   : tc_mma4_bf16_try(tmem_d, da, db, kAStep, kBStep, prm.idesc, kb != 0 ? 1u : 0u, full_bar(ns), nph);
                     tc_commit(empty_bar(s));          // frees the stage once these MMAs have read it
                     s = ns; ph = nph;
@@ -461,7 +472,8 @@ bool make_map_nmajor(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, int elem_
     EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
     if (!enc) return false;
     const uint32_t box_cols = 128u / (uint32_t)elem_bytes;
-    const CUtensorMapDataType dt = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
+    const CUtensorMapDataType dt = elem_bytes == 4 ? CU_TENSOR_MAP_DATA_TYPE_FLOAT32
+                                 : elem_bytes == 1 ? CU_TENSOR_MAP_DATA_TYPE_UINT8 : CU_TENSOR_MAP_DATA_TYPE_BFLOAT16;
     const CUtensorMapSwizzle sw = chunk32 ? CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B : CU_TENSOR_MAP_SWIZZLE_128B;
     const uint64_t chunks = (cols + box_cols - 1) / box_cols;
     if (ctx->tma_3d && ld >= chunks * box_cols && tile_cols / box_cols > 1) {
@@ -484,15 +496,15 @@ bool make_map_nmajor(gelo_ctx* ctx, CUtensorMap* map, const void* ptr, int elem_
                CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false>
+template <int BN, int kStages, bool kStaging, bool kTf32 = false, bool kAMn = false, bool kF8 = false>
 int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, const CUtensorMap& b0,
                  const CUtensorMap& b1, const CUtensorMap& c, const TcParams& p, double flops, cudaStream_t st)
 {
-    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn>;
+    using Cfg = TcCfg<BN, kStages, kStaging, kTf32, kAMn, kF8>;
     static_assert(Cfg::kSmemBytes <= 227 * 1024, "shared memory budget");
     static bool attr_done[64] = {};
     if (ctx->device >= 0 && ctx->device < 64 && !attr_done[ctx->device]) {
-        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        GELO_CUDA_OK(cudaFuncSetAttribute(gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn, kF8>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                           (int)Cfg::kSmemBytes));
         attr_done[ctx->device] = true;
     }
@@ -502,10 +514,10 @@ int launch_tiles(gelo_ctx* ctx, const CUtensorMap& a0, const CUtensorMap& a1, co
     TcParams q = p;
     // both operands of a kind::f16 instruction have the same 16-bit format: 1 = bfloat16, 0 = IEEE half
     q.wait_ns = ctx->wait_limit_ns;
-    q.idesc = (!kTf32 && p.out_f16) ? (Cfg::kInstrDesc & ~((7u << 7) | (7u << 10))) : Cfg::kInstrDesc;
+    q.idesc = (!kTf32 && !kF8 && p.out_f16) ? (Cfg::kInstrDesc & ~((7u << 7) | (7u << 10))) : Cfg::kInstrDesc;
     {
         ProfScope ps(ctx, PROF_GEMM_TC, flops, st);
-        gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, q);
+        gemm_tc_kernel<BN, kStages, kStaging, kTf32, kAMn, kF8><<<grid, kThreads, Cfg::kSmemBytes, st>>>(a0, a1, b0, b1, c, q);
     }
     return after_launch(ctx);
 }
@@ -780,6 +792,43 @@ int launch_gemm_bf16_sub(gelo_ctx* ctx, int M, int N, int K, const void* A, int 
     p.mode = TC_SUB_F32;
     p.C0 = C; p.ldc = ldc;
     return launch_tiles<256, 3, true>(ctx, ma, ma, mb, mb, mc, p, 2.0 * M * (double)N * K, st);
+}
+
+// Y (M x N, bf16) = (sa sb) A8 (M x K, E4M3, row stride lda bytes) * B8 (K x N, E4M3, row stride ldb bytes): the offloaded
+// product on 8-bit operands (kind::f8f6f4, fp32 accumulation), sa and sb device scalars.  A stage holds 128 bytes of
+// k per A row, i.e. 128 values, and the matching 128 rows of B in boxes of 128 columns.
+int launch_gemm_e4m3(gelo_ctx* ctx, int M, int N, int K, const void* A8, int lda, const void* B8, int ldb, const float* sa,
+                     const float* sb, void* C, int ldc, cudaStream_t st)
+{
+    if (M <= 0 || N <= 0 || K <= 0) return GELO_OK;
+    if (!ctx->tmap_encode) return GELO_ERR_CUDA;
+    if ((lda % 16) || (ldb % 16) || (ldc % 8) || (N % 8) || !aligned16(A8) || !aligned16(B8) || !aligned16(C) || !sa || !sb)
+        return GELO_ERR_INVALID;
+    EncodeTiledFn enc = reinterpret_cast<EncodeTiledFn>(ctx->tmap_encode);
+    CUtensorMap ma, mb;
+    {
+        const cuuint64_t dims[2] = { (cuuint64_t)K, (cuuint64_t)M };
+        const cuuint64_t strides[1] = { (cuuint64_t)lda };
+        const cuuint32_t box[2] = { 128, BM };
+        const cuuint32_t estr[2] = { 1, 1 };
+        if (enc(&ma, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(A8), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+                CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+            return GELO_ERR_CUDA;
+    }
+    bool b3d = false;
+    if (!make_map_nmajor(ctx, &mb, B8, 1, false, (uint64_t)N, (uint64_t)K, (uint64_t)ldb, 128, 256, &b3d)) return GELO_ERR_CUDA;
+    TcParams p = {};
+    p.M = M; p.N = N;
+    p.nseg = 1;
+    p.seg[0] = TcSegment{0, 0, 0, 0, ceil_div(K, 128)};
+    p.ksplit = 1; p.kb_per_split = 1 << 30; p.plane = 0;
+    p.mode = TC_STORE_BF16;
+    p.b3d = b3d ? 1 : 0;
+    p.C0 = C; p.C1 = C; p.C2 = C;
+    p.ldc = ldc; p.csplit = N;
+    p.scale_a = sa; p.scale_b = sb;
+    p.status = ctx->status_dev;
+    return launch_tiles<256, 4, false, false, false, true>(ctx, ma, ma, mb, mb, ma, p, 2.0 * M * (double)N * K, st);
 }
 
 int launch_gemm_tf32x3(gelo_ctx* ctx, int M, int N, int K, const float* Ahi, const float* Alo, int lda, const float* Bhi,

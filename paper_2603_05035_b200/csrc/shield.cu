@@ -107,26 +107,51 @@ __global__ void __launch_bounds__(256) median_rank_kernel(const float* __restric
 }
 
 template <typename T>
-__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q);
+__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q, int nu);
+
+// Standardised Student-t draw of element e (Section 4.4.1, Table 9 names Student-t shields): the element owns
+// B = 4 ceil((nu + 1) / 4) positions of the Gaussian stream (seed, shield stream, attempt word = nu) from e * B on,
+//     t = g_0 / sqrt((g_1^2 + ... + g_nu^2) / nu),   x = t sqrt((nu - 2) / nu)     (unit variance for nu > 2).
+__device__ __forceinline__ float student_t_draw(uint64_t seed, uint64_t e, int nu)
+{
+    const uint64_t blocks = (uint64_t)((nu + 1 + 3) >> 2);
+    float g0 = 0.0f, chi = 0.0f;
+    for (uint64_t b = 0; b < blocks; ++b) {
+        float z[4];
+        gaussian_block(seed, e * blocks + b, GELO_STREAM_SHIELD, (uint32_t)nu, z);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int idx = (int)b * 4 + j;
+            if (idx == 0) g0 = z[j];
+            else if (idx <= nu) chi = fmaf(z[j], z[j], chi);
+        }
+    }
+    return g0 / sqrtf(chi / (float)nu) * sqrtf(((float)nu - 2.0f) / (float)nu);
+}
 
 template <typename T>
 __global__ void __launch_bounds__(256) shield_fill_kernel(T* __restrict__ S, int k, int d, float scale,
-                                                          const float* __restrict__ med, uint64_t seed)
+                                                          const float* __restrict__ med, uint64_t seed, int nu)
 {
     const uint64_t total = (uint64_t)k * d;
     const uint64_t q = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     const uint64_t e0 = q << 2;
     if (e0 >= total) return;                      // d % 8 == 0, so blocks never straddle the end
     const float f = scale * (0.5f * (med[0] + med[1])) / sqrtf((float)d);
-    store_shield_block(S, e0, f, seed, q);
+    store_shield_block(S, e0, f, seed, q, nu);
 }
 
 // S[e0 .. e0+3] = f * (the four normals of block q of the shield stream), in the storage type
 template <typename T>
-__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q)
+__device__ __forceinline__ void store_shield_block(T* __restrict__ S, uint64_t e0, float f, uint64_t seed, uint64_t q, int nu)
 {
     float z[4];
-    gaussian_block(seed, q, GELO_STREAM_SHIELD, 0u, z);
+    if (nu > 0) {
+#pragma unroll
+        for (int j = 0; j < 4; ++j) z[j] = student_t_draw(seed, e0 + j, nu);
+    } else {
+        gaussian_block(seed, q, GELO_STREAM_SHIELD, 0u, z);
+    }
     if (sizeof(T) == 4) {
         *reinterpret_cast<float4*>(reinterpret_cast<float*>(S) + e0) = make_float4(f * z[0], f * z[1], f * z[2], f * z[3]);
     } else if (is_half_t<T>::value) {
@@ -154,7 +179,7 @@ constexpr int kShieldSmallRows = 256;
 
 template <typename T>
 __global__ void __launch_bounds__(1024, 1)
-shield_small_kernel(const T* __restrict__ H, int n, int d, int k, float scale, uint64_t seed, T* __restrict__ S)
+shield_small_kernel(const T* __restrict__ H, int n, int d, int k, float scale, uint64_t seed, T* __restrict__ S, int nu)
 {
     namespace cg = cooperative_groups;
     cg::cluster_group cluster = cg::this_cluster();
@@ -184,11 +209,11 @@ shield_small_kernel(const T* __restrict__ H, int n, int d, int k, float scale, u
     const float f = scale * (0.5f * (med_s[0] + med_s[1])) / sqrtf((float)d);
     const uint64_t blocks = ((uint64_t)k * d) >> 2;           // d % 8 == 0
     for (uint64_t q = (uint64_t)rank * 1024 + threadIdx.x; q < blocks; q += (uint64_t)CS * 1024)
-        store_shield_block(S, q << 2, f, seed, q);
+        store_shield_block(S, q << 2, f, seed, q, nu);
 }
 
 template <typename T>
-int launch_shield_small(gelo_ctx* ctx, const void* H, int n, int d, int k, float scale, uint64_t seed, void* S, cudaStream_t st)
+int launch_shield_small(gelo_ctx* ctx, const void* H, int n, int d, int k, float scale, uint64_t seed, void* S, int nu, cudaStream_t st)
 {
     const int cs = ceil_div(n, 32);                           // <= 8
     cudaLaunchConfig_t cfg = {};
@@ -201,7 +226,7 @@ int launch_shield_small(gelo_ctx* ctx, const void* H, int n, int d, int k, float
     attr[0].val.clusterDim.x = cs; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    if (cudaLaunchKernelEx(&cfg, shield_small_kernel<T>, static_cast<const T*>(H), n, d, k, scale, seed, static_cast<T*>(S)) != cudaSuccess)
+    if (cudaLaunchKernelEx(&cfg, shield_small_kernel<T>, static_cast<const T*>(H), n, d, k, scale, seed, static_cast<T*>(S), nu) != cudaSuccess)
         return GELO_ERR_CUDA;
     return after_launch(ctx);
 }
@@ -217,13 +242,14 @@ ShieldScratch carve_shield(Arena& a, int n)
 }
 
 int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float scale, uint64_t seed,
-                    int dtype, void* S, const ShieldScratch& s, cudaStream_t st)
+                    int dtype, void* S, const ShieldScratch& s, cudaStream_t st, int nu)
 {
     if (k <= 0) return GELO_OK;
+    if (nu != 0 && (nu < 3 || nu > 63)) return GELO_ERR_INVALID;
     if (n <= kShieldSmallRows) {
-        if (dtype == GELO_BF16) return launch_shield_small<__nv_bfloat16>(ctx, H, n, d, k, scale, seed, S, st);
-        if (dtype == GELO_F16) return launch_shield_small<__half>(ctx, H, n, d, k, scale, seed, S, st);
-        return launch_shield_small<float>(ctx, H, n, d, k, scale, seed, S, st);
+        if (dtype == GELO_BF16) return launch_shield_small<__nv_bfloat16>(ctx, H, n, d, k, scale, seed, S, nu, st);
+        if (dtype == GELO_F16) return launch_shield_small<__half>(ctx, H, n, d, k, scale, seed, S, nu, st);
+        return launch_shield_small<float>(ctx, H, n, d, k, scale, seed, S, nu, st);
     }
     if (dtype == GELO_BF16)
         row_norm_kernel<__nv_bfloat16><<<ceil_div(n, 8), 256, 0, st>>>(static_cast<const __nv_bfloat16*>(H), n, d, s.norms);
@@ -237,11 +263,11 @@ int run_shield_rows(gelo_ctx* ctx, const void* H, int n, int d, int k, float sca
     const uint64_t blocks = ((uint64_t)k * d + 3) / 4;
     const unsigned grid = (unsigned)((blocks + 255) / 256);
     if (dtype == GELO_BF16)
-        shield_fill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<__nv_bfloat16*>(S), k, d, scale, s.med, seed);
+        shield_fill_kernel<__nv_bfloat16><<<grid, 256, 0, st>>>(static_cast<__nv_bfloat16*>(S), k, d, scale, s.med, seed, nu);
     else if (dtype == GELO_F16)
-        shield_fill_kernel<__half><<<grid, 256, 0, st>>>(static_cast<__half*>(S), k, d, scale, s.med, seed);
+        shield_fill_kernel<__half><<<grid, 256, 0, st>>>(static_cast<__half*>(S), k, d, scale, s.med, seed, nu);
     else
-        shield_fill_kernel<float><<<grid, 256, 0, st>>>(static_cast<float*>(S), k, d, scale, s.med, seed);
+        shield_fill_kernel<float><<<grid, 256, 0, st>>>(static_cast<float*>(S), k, d, scale, s.med, seed, nu);
     return after_launch(ctx);
 }
 

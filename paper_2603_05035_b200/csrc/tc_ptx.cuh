@@ -132,6 +132,11 @@ __device__ __forceinline__ bool tc_mma4_tf32_try(uint32_t tmem_d, uint64_t da, u
 {
     GELO_TC_MMA4_TRY("tf32")
 }
+__device__ __forceinline__ bool tc_mma4_f8_try(uint32_t tmem_d, uint64_t da, uint64_t db, uint64_t astep, uint64_t bstep,
+                                               uint32_t idesc, uint32_t accumulate, uint32_t next_bar, uint32_t next_parity)
+{
+    GELO_TC_MMA4_TRY("f8f6f4")
+}
 #undef GELO_TC_MMA4_TRY
 
 __device__ __forceinline__ float round_tf32(float x)

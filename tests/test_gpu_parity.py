@@ -229,6 +229,41 @@ def _random_mixing(oracle, m, kind, seed, dt):
 
 
 @pytest.mark.parametrize("dt", ["f32", "bf16"])
+@pytest.mark.parametrize("n,d,k,nu", [(64, 4096, 4, 5), (2048, 1024, 102, 3), (300, 256, 7, 10), (7, 64, 3, 63)])
+def test_student_t_shield_rows(ctx, oracle, n, d, k, nu, dt):
+    """Student-t shield rows (both the one-launch and the three-kernel route) against the oracle."""
+    ctx.ensure_workspace(n, k, d, 3 * d, dt)
+    H = inputs.make_hidden(n, d, dt, 11, False, "cuda")
+    S = torch.full((k, d), float("nan"), device="cuda", dtype=TDT[dt])
+    ctx.shield_rows_t(H, n, d, k, 10.0, 321, nu, dt, S)
+    torch.cuda.synchronize()
+    ref = oracle.shield_rows_t(f64(H), k, 10.0, 321, nu)
+    # fp32 normals agree with the oracle's to 2e-6 absolute; the ratio g_0 / sqrt(mean g^2) keeps that as a relative error
+    # of about 1e-5 of the largest entries; bf16 adds its rounding
+    tol = 2e-5 if dt == "f32" else 4e-3
+    assert oracle.rel_fro(f64(S), ref) <= tol
+    assert np.max(np.abs(f64(S) - ref)) <= 10 * tol * np.sqrt(np.mean(ref * ref)) * (1 + np.max(np.abs(ref)) / np.sqrt(np.mean(ref * ref)))
+
+
+def test_whole_call_with_student_t_shields(oracle):
+    """The result is H W whatever the shield rows are (Eq. 4); the call must stay inside the tolerance with the
+    heavier-tailed kind too."""
+    c = make_ctx(600, 30, 512, 1536, "bf16")
+    c.set_shield_student_t(5)
+    n, k, d, p = 600, 30, 512, 1536
+    H = inputs.make_hidden(n, d, "bf16", 12, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 12, "cuda")
+    Q = torch.empty((n, d), device="cuda", dtype=torch.bfloat16); K = torch.empty_like(Q); V = torch.empty_like(Q)
+    c.qkv_offload(H, W, n, k, d, p, ORTHOGONAL, 5, 10.0, "bf16", Q, K, V)
+    torch.cuda.synchronize()
+    y = np.hstack([f64(Q), f64(K), f64(V)])
+    assert oracle.rel_fro(y, oracle.direct(f64(H), f64(W))) <= TOL["bf16"]
+    with pytest.raises(binding.GeloError):
+        c.set_shield_student_t(2)
+    c.close()
+
+
+@pytest.mark.parametrize("dt", ["f32", "bf16"])
 @pytest.mark.parametrize("n,k,d,p", [(64, 0, 256, 768), (64, 4, 256, 768), (130, 7, 264, 264 * 3),
                                       (1, 0, 8, 24), (200, 10, 512, 1536), (256, 0, 128, 384)])
 def test_products_stage_parity(ctx, oracle, n, k, d, p, dt):
@@ -900,3 +935,84 @@ def test_async_host_batches_of_different_shapes_back_to_back(oracle):
     y = np.hstack([f64(data[1][8][j][1]) for j in range(3)])
     assert oracle.rel_fro(y, oracle.direct(f64(data[1][4][1]), f64(data[1][5][1]))) <= TOL["bf16"]
     c.close()
+
+
+# ------------------------------------------------------------------------- E4M3 operands for the offloaded product
+
+@pytest.mark.parametrize("dt", ["bf16", "f32"])
+@pytest.mark.parametrize("rows,cols", [(68, 4096), (300, 528), (1, 16), (4300, 1024)])
+def test_e4m3_quantiser_is_bit_exact(ctx, oracle, rows, cols, dt):
+    """Per-tensor E4M3 quantiser: scale and every code against the oracle's (same binary32 division, same rounding)."""
+    g = torch.Generator(device="cuda"); g.manual_seed(rows + cols)
+    X = (torch.randn((rows, cols), device="cuda", generator=g) * torch.rand((rows, 1), device="cuda", generator=g) * 7).to(TDT[dt])
+    codes = torch.full((rows, cols), 0xAA, device="cuda", dtype=torch.uint8)
+    scale = torch.zeros(2, device="cuda", dtype=torch.float32)
+    ctx.quantize_e4m3(X, rows, cols, dt, codes, scale)
+    torch.cuda.synchronize()
+    ref_codes, ref_scale = oracle.quantize_e4m3(f64(X).astype(np.float32))
+    assert np.float32(scale[0].item()) == ref_scale
+    got = oracle.e4m3_decode(codes.cpu().numpy())
+    assert np.array_equal(got, oracle.e4m3_decode(ref_codes))          # (compares values: +0 and -0 are the same number)
+    Z = torch.zeros((8, 32), device="cuda", dtype=TDT[dt])
+    zc = torch.full((8, 32), 0xAA, device="cuda", dtype=torch.uint8)
+    ctx.quantize_e4m3(Z, 8, 32, dt, zc, scale)
+    torch.cuda.synchronize()
+    assert scale[0].item() == 1.0 and not zc.any()
+
+
+@pytest.mark.parametrize("m,d,p", [(200, 1024, 768), (130, 208, 272), (68, 4096, 12288), (1, 16, 16)])
+def test_e4m3_projection_stage(ctx, oracle, m, d, p):
+    """Eq. 2 on E4M3 operands: the device product against the oracle's product of the SAME stored codes (what is left
+    is the bf16 rounding of the output), and against the unquantised product (FP8-grade: a few percent)."""
+    U = (3.0 * torch.randn((m, d), device="cuda")).to(torch.bfloat16)
+    W = inputs.make_weight(d, p, "bf16", 21, "cuda")
+    U8 = torch.empty((m, d), device="cuda", dtype=torch.uint8); W8 = torch.empty((d, p), device="cuda", dtype=torch.uint8)
+    su = torch.zeros(2, device="cuda"); sw = torch.zeros(2, device="cuda")
+    ctx.quantize_e4m3(U, m, d, "bf16", U8, su)
+    ctx.quantize_e4m3(W, d, p, "bf16", W8, sw)
+    Y = torch.full((m, p), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ctx.project_e4m3(U8, su, W8, sw, m, d, p, Y)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == binding.OK
+    ref = oracle.project_e4m3(U8.cpu().numpy(), su[0].item(), W8.cpu().numpy(), sw[0].item())
+    assert oracle.rel_fro(f64(Y), ref) <= 4e-3
+    if d >= 208:
+        assert oracle.rel_fro(f64(Y), oracle.matmul(f64(U), f64(W))) <= 0.08
+
+
+def test_e4m3_projection_full_size_and_chain(ctx, oracle):
+    """The benchmark shape (m = 4300 mixed rows with 10x shield rows, d = 4096, p = 12288) on sampled rows, and what the
+    FP8 product does to the whole call: bf16 mix, E4M3 projection, bf16 unmix."""
+    n, k, d, p = 4096, 204, 4096, 12288
+    m = n + k
+    ld = ctx.mixing_ld(m)
+    ctx.ensure_workspace(n, k, d, p, "bf16")
+    H = inputs.make_hidden(n, d, "bf16", 61, True, "cuda")
+    W = inputs.make_weight(d, p, "bf16", 61, "cuda")
+    A = padded(m, ld, torch.bfloat16); X = padded(m, ld, torch.bfloat16)
+    S = torch.empty((k, d), device="cuda", dtype=torch.bfloat16)
+    U = torch.empty((m, d), device="cuda", dtype=torch.bfloat16)
+    ctx.sample_mixing(m, ORTHOGONAL, 6161, "bf16", A, X, ld)
+    ctx.shield_rows(H, n, d, k, 10.0, 6161, "bf16", S)
+    ctx.mix(A, ld, H, S, n, k, d, "bf16", U)
+    U8 = torch.empty((m, d), device="cuda", dtype=torch.uint8); W8 = torch.empty((d, p), device="cuda", dtype=torch.uint8)
+    su = torch.zeros(2, device="cuda"); sw = torch.zeros(2, device="cuda")
+    ctx.quantize_e4m3(U, m, d, "bf16", U8, su)
+    ctx.quantize_e4m3(W, d, p, "bf16", W8, sw)
+    Yp = torch.full((m, p), float("nan"), device="cuda", dtype=torch.bfloat16)
+    ctx.project_e4m3(U8, su, W8, sw, m, d, p, Yp)
+    Q = torch.empty((n, d), device="cuda", dtype=torch.bfloat16); K = torch.empty_like(Q); V = torch.empty_like(Q)
+    ctx.unmix(X, ld, Yp, n, k, p, "bf16", Q, K, V)
+    torch.cuda.synchronize()
+    assert ctx.last_status() == binding.OK and torch.isfinite(Yp).all()
+    rows = sample_rows(m, 48, seed=3, extra=(n - 1, n))
+    u_dec = oracle.e4m3_decode(U8[rows].cpu().numpy()) * su[0].item()
+    w_dec = oracle.e4m3_decode(W8.cpu().numpy()) * sw[0].item()
+    ref = oracle.matmul(u_dec, w_dec)
+    assert oracle.rel_fro(f64(Yp[rows]), ref) <= 4e-3
+    # the whole call: 3 mantissa bits per operand give about 5% on Y', and the shield rows' 6x energy brings the data
+    # rows to about 12% after unmixing (the bound derived for this path: 0.2)
+    y = np.hstack([f64(Q), f64(K), f64(V)])
+    drows = sample_rows(n, 32, seed=4)
+    err = oracle.rel_fro(y[drows], oracle.rows_times_w(f64(H), f64(W), drows))
+    assert 0.02 < err <= 0.2
