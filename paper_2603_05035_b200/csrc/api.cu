@@ -64,10 +64,21 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     L.Qraw = static_cast<float*>(a.take(mat * 4));
     L.A32 = static_cast<float*>(a.take(mat * 4));
     L.X32 = static_cast<float*>(a.take(mat * 4));
-    L.qr = carve_qr(a, L.m, L.ldi);
+    // Buffers that are never alive together share memory:
+    //   * while a QR runs, A32 and X32 are idle (they receive the signed Q0 / serve the polish and the LU afterwards):
+    //     the QR's split-K planes, its W blocks and the rank-32 partial sums live in A32 (as far as they fit: they need
+    //     4096 rows' worth, so this applies from m = 4096 up), the (high, low) pair of the trailing matrix in X32;
+    //   * the reflectors V die with the QR and the LU's working copy M is born after it: one matrix.
+    char* idle = reinterpret_cast<char*>(L.A32);          // (null in a size query: only the byte count matters then)
+    size_t idle_bytes = mat * 4;
+    L.qr = carve_qr(a, L.m, L.ldi, &idle, &idle_bytes);
     L.lu = carve_lu(a, L.m, L.ldi);
+    L.lu.M = L.qr.V;
     L.cond = carve_cond(a, L.m);
-    L.tc = carve_tc(a, L.m, L.ldi);
+    L.tc = carve_tc(a, L.m, L.ldi, &idle, &idle_bytes);
+    for (int h = 0; h < 2; ++h)                            // 2 x (m x ld) 16-bit values: exactly the fp32 matrix X32
+        L.tc.big[h] = L.X32 ? reinterpret_cast<char*>(L.X32) + (size_t)h * mat * 2 : nullptr;
+    if (!a.base) { L.qr.Wp = nullptr; L.tc.wf32 = nullptr; L.tc.w32[0] = L.tc.w32[1] = nullptr; }
     L.sh = carve_shield(a, n);
     L.cond_val = static_cast<float*>(a.take(16));
     L.A = a.take(mat * es);

@@ -247,8 +247,10 @@ struct QrScratch {       // all fp32
     float* W2 = nullptr; // kPanel x ld
     float* T128 = nullptr; // ceil(m / 128) blocks of 128 x 128: triangular factors of the outer blocks
 };
-size_t qr_scratch_bytes(int m, int ld);
-QrScratch carve_qr(Arena&, int m, int ld);
+void* take_idle(Arena&, char** idle, size_t* idle_bytes, size_t bytes);
+// `idle`, if given, is memory that nothing else uses while a factorisation runs (idle_bytes of it): scratch that lives
+// only then is placed there instead of in the arena (see carve() in api.cu for who is idle when)
+QrScratch carve_qr(Arena&, int m, int ld, char** idle = nullptr, size_t* idle_bytes = nullptr);
 // Factorises R (m x m, stride ld, overwritten; its diagonal holds diag(R) afterwards) and
 // writes the orthogonal factor Q with G = Q R.  The caller flips column j of Q where
 // R_jj < 0 (launch_finish_mixing with sign_diag = R) to reach the unique factor.
@@ -270,7 +272,7 @@ struct LuScratch {
     int* perm = nullptr;  // m
     int* swap_table = nullptr;  // composed interchanges of one panel / block: count, then (target, source) pairs
 };
-LuScratch carve_lu(Arena&, int m, int ld);
+LuScratch carve_lu(Arena&, int m, int ld);   // everything but the working copy M, which the caller points at memory of its choice
 int run_lu_inverse(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, cudaStream_t);
 struct TcScratch;
 int run_lu_inverse_tc(gelo_ctx*, int m, const float* A, int ld, float* Ainv, const LuScratch&, const TcScratch&,
@@ -330,7 +332,7 @@ struct TcScratch {
     float* sx = nullptr;                   // kOuter x (kSuper + kOuter)   V_i^T [V_(<i) | V_i] of the block being merged
     float* xb = nullptr;                   // kSuper x kOuter     its product with T_i
 };
-TcScratch carve_tc(Arena&, int m, int ld);
+TcScratch carve_tc(Arena&, int m, int ld, char** idle = nullptr, size_t* idle_bytes = nullptr);   // all but big[], set by the caller
 // C (M x N fp32) -= A (M x K fp32) * B (K x N fp32), K <= kSuper, on the tensor cores: three bf16 products of
 // (high, low) operand pairs, or (tf32) one tf32 product straight from the fp32 operands
 int tc_update_f32(gelo_ctx*, const TcScratch&, bool tf32, int M, int N, int K, const float* A, int lda, const float* B,

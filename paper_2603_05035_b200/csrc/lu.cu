@@ -526,8 +526,8 @@ int set_permutation(gelo_ctx* ctx, float* X, int ld, int m, const int* perm, cud
 
 LuScratch carve_lu(Arena& a, int m, int ld)
 {
+    (void)ld;
     LuScratch s;
-    s.M = static_cast<float*>(a.take((size_t)m * ld * sizeof(float)));
     s.ipiv = static_cast<int*>(a.take((size_t)m * sizeof(int)));
     s.perm = static_cast<int*>(a.take((size_t)m * sizeof(int)));
     s.swap_table = static_cast<int*>(a.take((size_t)(2 * 256 + 4) * sizeof(int)));

@@ -607,19 +607,26 @@ int launch_qr_small(gelo_ctx* ctx, int m, float* G, int ld, float* Q, cudaStream
 
 }  // namespace
 
-size_t qr_scratch_bytes(int m, int ld)
+
+// Takes `bytes` from the idle region if it has that much left, else from the arena.
+void* take_idle(Arena& a, char** idle, size_t* idle_bytes, size_t bytes)
 {
-    Arena a; a.cap = ~size_t(0) >> 1;
-    carve_qr(a, m, ld);
-    return a.off + 256;
+    const size_t need = (bytes + 255) & ~size_t(255);
+    if (idle && idle_bytes && *idle_bytes >= need) {
+        void* p = *idle;
+        *idle += need;
+        *idle_bytes -= need;
+        return p;
+    }
+    return a.take(bytes);
 }
 
-QrScratch carve_qr(Arena& a, int m, int ld)
+QrScratch carve_qr(Arena& a, int m, int ld, char** idle, size_t* idle_bytes)
 {
     QrScratch s;
     s.V = static_cast<float*>(a.take((size_t)m * ld * sizeof(float)));
     s.T = static_cast<float*>(a.take((size_t)ceil_div(m, NB) * NB * NB * sizeof(float)));
-    s.Wp = static_cast<float*>(a.take((size_t)kMaxSlabs * NB * ld * sizeof(float)));
+    s.Wp = static_cast<float*>(take_idle(a, idle, idle_bytes, (size_t)kMaxSlabs * NB * ld * sizeof(float)));
     s.W2 = static_cast<float*>(a.take((size_t)NB * ld * sizeof(float)));
     s.T128 = static_cast<float*>(a.take((size_t)ceil_div(m, 128) * 128 * 128 * sizeof(float)));
     return s;

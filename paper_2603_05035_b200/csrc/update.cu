@@ -258,7 +258,7 @@ rank_update_kernel(const float* __restrict__ A, int lda, const float* __restrict
 
 }  // namespace
 
-TcScratch carve_tc(Arena& a, int m, int ld)
+TcScratch carve_tc(Arena& a, int m, int ld, char** idle, size_t* idle_bytes)
 {
     TcScratch t;
     for (int h = 0; h < 2; ++h) {
@@ -267,12 +267,11 @@ TcScratch carve_tc(Arena& a, int m, int ld)
         t.rowB[h] = a.take((size_t)kSuper * ld * 2);
         t.rowB2[h] = a.take((size_t)kOuter * ld * 2);
         t.tt[h] = a.take((size_t)kOuter * kOuter * 2);
-        t.big[h] = a.take((size_t)m * ld * 2);
     }
     t.t128 = static_cast<float*>(a.take((size_t)kOuter * kOuter * 4));
     t.gram = static_cast<float*>(a.take((size_t)(m / 256 + 2) * kOuter * kOuter * 4));   // one partial Gram per 256-row slab
-    t.wf32 = static_cast<float*>(a.take((size_t)kMaxKSplit * kOuter * ld * 4));
-    for (int h = 0; h < 2; ++h) t.w32[h] = static_cast<float*>(a.take((size_t)kSuper * ld * 4));
+    t.wf32 = static_cast<float*>(take_idle(a, idle, idle_bytes, (size_t)kMaxKSplit * kOuter * ld * 4));
+    for (int h = 0; h < 2; ++h) t.w32[h] = static_cast<float*>(take_idle(a, idle, idle_bytes, (size_t)kSuper * ld * 4));
     t.tsuper = static_cast<float*>(a.take((size_t)ceil_div(m, kSuper) * kSuper * kSuper * 4));
     t.sx = static_cast<float*>(a.take((size_t)kOuter * (kSuper + kOuter) * 4));
     t.xb = static_cast<float*>(a.take((size_t)kSuper * kOuter * 4));
