@@ -34,8 +34,8 @@ METRIC = "obfuscated-QKV tokens/s at Llama-2-7B shapes"
 UNIT = "tokens/s"
 WORKLOAD = "prefill_bf16"
 # DRAM bytes over algorithmic bytes of the panel kernels, from one ncu capture of a panel of 3300 rows; traffic
-# scales with the rows, so other panel heights use the same ratio.
-PANEL_TRAFFIC_RATIO = 0.49
+# scales with the rows, so other panel heights use the same ratio (0.58 MB against 8 B x 4300 rows x 32 columns).
+PANEL_TRAFFIC_RATIO = 0.53
 
 
 def _peaks():
@@ -407,7 +407,7 @@ def run_ours(args):
                              "sms_used": 8, "frac_of_sms_used": dk["achieved"] / (alu_peak * 8 / 148),
                              "note": "latency-bound by design: 33 dependent column steps per launch on one cluster; "
                                      "other lanes' kernels use the remaining SMs concurrently",
-                             # ncu: 0.41 MB DRAM per launch against 0.85 MB algorithmic (8 B x rows x 32) at rows = 3300
+                             # ncu: 0.58 MB DRAM per launch against 1.10 MB algorithmic (8 B x rows x 32) at rows = 4300
                              "traffic": PANEL_TRAFFIC_RATIO * 8.0 * avg_rows * 32})
         elif dk["unit"] == "TFLOP/s":
             roofline.update({"bound": "tensor", "peak": peaks["bf16_tflops"], "frac": dk["achieved"] / peaks["bf16_tflops"],
@@ -419,8 +419,8 @@ def run_ours(args):
         proj_tflops = 2.0 * m * d * p / (stage_ms["project"] * 1e-3) / 1e12
         projection = {"kernel": "gemm_tc_kernel, Y' = U W", "bound": "tensor", "achieved": proj_tflops,
                       "peak": peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": proj_tflops / peaks["bf16_tflops"],
-                      # ncu: dram read 152.5 MB + write 85.0 MB per launch (algorithmic 241.6 MB)
-                      "traffic": 237.5e6}
+                      # ncu: dram read 162.6 MB + write 85.5 MB per launch (algorithmic 241.6 MB)
+                      "traffic": 248.0e6}
         f8_tflops = 2.0 * m * d * p / (stage_ms["project_e4m3"] * 1e-3) / 1e12
         projection_e4m3 = {"kernel": "gemm_tc_kernel (kind::f8f6f4), Y' = (s_U s_W) U8 W8", "bound": "tensor", "achieved": f8_tflops,
                            "peak": 2.0 * peaks["bf16_tflops"], "unit": "TFLOP/s", "frac": f8_tflops / (2.0 * peaks["bf16_tflops"]),
@@ -432,11 +432,11 @@ def run_ours(args):
                        "bound": "tensor", "achieved": upd_tflops, "peak": tf32_peak, "unit": "TFLOP/s",
                        "frac": upd_tflops / tf32_peak,
                        "peak_source": peaks["source"] + " bf16 GEMM x nominal tf32/bf16 ratio 0.5",
-                       # ncu: dram read 82.1 MB + write 8.9 MB per launch (algorithmic 147 MB, half of C stays in L2)
-                       "traffic": 91.0e6,
+                       # ncu: dram read 82.1 MB + write 9.0 MB per launch (algorithmic 147 MB, half of C stays in L2)
+                       "traffic": 91.1e6,
                        "note": "largest share of SM time among the sampling kernels; "
-                               "510 tiles of 16 k-blocks on 148 CTAs: bound by the tf32 main-loop rate (571 TFLOP/s sustained at large K) "
-                               "and the 3.45-wave quantisation"}
+                               "510 tiles of 16 k-blocks on 148 CTAs: fp32 operands re-read from L2 for every 128 x 256 tile (8.8 TB/s L2 -> SM) "
+                               "and the 3.45-wave quantisation; 630 TFLOP/s sustained at large K"}
         per_call_ms = ms_max / args.steps / calls
         chain_tflops = chain_flops / (chain_ms * 1e-3) / 1e12
         # all arithmetic of a sweep against the time the sweep takes with every lane busy: the Householder QR of every
