@@ -529,9 +529,16 @@ def measure_workload(name, lanes, steps, warmup, calls=0, latency_steps=0):
     Q = torch.empty((n, p // 3), device=dev, dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
     kinds = [w.kind(c) for c in range(calls)]
 
+    if m <= 128:
+        # small batches run whole calls on concurrent lanes: every call gets its own outputs
+        Qs = [torch.empty_like(Q) for _ in range(calls)]; Ks = [torch.empty_like(Q) for _ in range(calls)]
+        Vs = [torch.empty_like(Q) for _ in range(calls)]
+    else:
+        Qs, Ks, Vs = [Q] * calls, [K] * calls, [V] * calls
+
     def sweep(step):
         ctx.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, [w.seed + 100000 * (step + 7) + c for c in range(calls)],
-                              w.shield_scale, w.dtype, [Q] * calls, [K] * calls, [V] * calls)
+                              w.shield_scale, w.dtype, Qs, Ks, Vs)
 
     for i in range(max(3, warmup)):
         sweep(-1 - i)

@@ -106,6 +106,10 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     return L;
 }
 
+// Lanes other than the first hold only what sampling needs, except for small batches (m <= 128), whose lanes also
+// form their own shield rows and mixed matrix: those get an S and a U of their own (d columns wide).
+inline int lane_width(int n, int k, int d) { return (n + k <= 128) ? d : 0; }
+
 bool carve_ctx(gelo_ctx* ctx, int n, int k, int d, int p, int dtype, bool host_staging, Layout* out)
 {
     if (!ctx->ws) return false;
@@ -358,18 +362,25 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     a.cap = ctx->ws_bytes;
     Layout L[kMaxLanes];
     L[0] = carve(a, n, k, d, p, dtype, host);
-    for (int i = 1; i < D; ++i) L[i] = carve(a, n, k, 0, 0, dtype, false);
+    for (int i = 1; i < D; ++i) L[i] = carve(a, n, k, lane_width(n, k, d), 0, dtype, false);
     if (!a.ok) return GELO_ERR_WORKSPACE;
     const size_t es = elem_size(dtype);
     const bool split = K[0] != nullptr;
     const size_t third = (size_t)n * (p / 3) * es;
+    // A small batch (the decode shape) is a stream of W per call and little else; its other launches are short and
+    // latency-bound.  There the WHOLE call runs on its lane (sampling, shield rows, mixing, fused projection + unmixing,
+    // on the lane's own S and U): the weight streams of different calls overlap at their seams and the caller's stream
+    // only joins the lanes at the end of the batch.
+    bool small = !host && D > 1 && ctx->fuse_small && lane_width(n, k, d) > 0 && mix_small_supports(n, k, d, dtype) &&
+                 project_unmix_supports(ctx, n, k, d, p, dtype, L[0].ldi, split ? 3 : 1);
+    for (int i = 0; i < calls && small; ++i) small = !misaligned(H[i]);
     // with several lanes in flight each level-3 update takes a share of the SMs (ctx->lane_tc_share-th of them)
     ctx->tc_update_ctas = (D >= ctx->lane_tc_share && ctx->lane_tc_share > 1) ? ctx->sm_count / ctx->lane_tc_share : 0;
 
     // Back-to-back batches of the same shape on the same stream keep the lanes running across the seam: each
     // lane only waits until the products that read its previous pair are done.  Otherwise the lanes start after
     // everything already enqueued on the caller's stream.
-    const int shape[6] = { n, k, d, p, dtype, host ? 1 : 0 };
+    const int shape[6] = { n, k, d, p, dtype, (host ? 1 : 0) | (small ? 2 : 0) };
     bool same_shape = true;
     for (int i = 0; i < 6; ++i) same_shape = same_shape && ctx->chain_shape[i] == shape[i];
     const bool chained = ctx->chain_valid && ctx->chain_stream == st && ctx->chain_key == L[D - 1].G &&
@@ -385,6 +396,27 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         }
     }
 
+    if (small) {
+        // the lanes read H_i and write Q_i, K_i, V_i: not before this point of the caller's stream (a lane that runs on
+        // from the previous batch may sample ahead of it)
+        if (chained) GELO_CUDA_OK(cudaEventRecord(ctx->batch_start, st));
+        for (int i = 0; i < calls; ++i) {
+            const int l = i % D;
+            cudaStream_t ls = ctx->lane_stream[l];
+            GELO_TRY(sample_on_lane(ctx, L[l], l, m, kinds[i], seeds[i], dtype, ls));
+            if (chained && i < D) GELO_CUDA_OK(cudaStreamWaitEvent(ls, ctx->batch_start, 0));
+            GELO_TRY(run_shield_rows(ctx, H[i], n, d, k, shield_scale, seeds[i], dtype, L[l].S, L[l].sh, ls, ctx->shield_nu));
+            GELO_TRY(mix_impl(ctx, L[l].A, L[l].ldi, H[i], k > 0 ? L[l].S : nullptr, n, k, d, dtype, L[l].U, ls, nullptr));
+            GELO_TRY(project_and_unmix(ctx, L[l].U, W[i], L[l].Ainv, L[l].ldi, nullptr, n, k, d, p, dtype, Q[i],
+                                       split ? K[i] : nullptr, split ? V[i] : nullptr, ls, nullptr));
+        }
+        for (int l = 0; l < D; ++l) {
+            GELO_CUDA_OK(cudaEventRecord(ctx->lane_ready[l], ctx->lane_stream[l]));
+            GELO_CUDA_OK(cudaStreamWaitEvent(st, ctx->lane_ready[l], 0));
+        }
+        for (int l = 0; l < D; ++l) GELO_CUDA_OK(cudaEventRecord(ctx->lane_free[l], st));
+    }
+
     auto enqueue_sample = [&](int i) -> int {
         const int l = i % D;
         cudaStream_t ls = ctx->lane_stream[l];
@@ -394,7 +426,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
         return GELO_OK;
     };
 
-    for (int i = 0; i < D; ++i) GELO_TRY(enqueue_sample(i));
+    for (int i = 0; i < D && !small; ++i) GELO_TRY(enqueue_sample(i));
     // Host variant: activations come in on the context's copy-in stream and results leave on its copy-out stream,
     // through two staging pairs used alternately, so that the copies of call i overlap the products of calls i-1 and
     // i+1 (the two directions use different copy engines):
@@ -403,7 +435,7 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     //                                                                  -> record h_free_b, y_ready_b, lane_free
     //   copy-out:  [wait y_ready_b] Yd_b -> Q_i, K_i, V_i              -> record y_free_b
     // and at the end the caller's stream waits for the last copies out.
-    for (int i = 0; i < calls; ++i) {
+    for (int i = 0; i < calls && !small; ++i) {
         const int l = i % D;
         const int b = i & 1;
         const void* Hi = H[i];
@@ -593,7 +625,7 @@ size_t batch_workspace(int n, int k, int d, int p, int dtype, int lanes)
     Arena a;
     a.cap = ~size_t(0) >> 1;
     carve(a, n, k, d, p, dtype, true);
-    for (int i = 1; i < lanes; ++i) carve(a, n, k, 0, 0, dtype, false);
+    for (int i = 1; i < lanes; ++i) carve(a, n, k, lane_width(n, k, d), 0, dtype, false);
     return a.off + 256;
 }
 

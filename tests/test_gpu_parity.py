@@ -520,6 +520,51 @@ def test_batched_offload_matches_single_calls(oracle, name, calls, lanes):
     c.close()
 
 
+def test_small_batches_back_to_back_follow_the_callers_stream(oracle):
+    """Small batches run whole calls on the lanes.  A second batch whose inputs are produced on the caller's stream
+    AFTER the first batch (from the first batch's outputs) must see them, and the lanes that run on across the seam
+    must not overwrite outputs that the caller's stream still reads."""
+    w = inputs.WORKLOADS["decode_bf16"]
+    n, k, d, p = w.n, w.k, w.d, w.p
+    calls, lanes = 12, 4
+    c = binding.Context(0)
+    c.set_lanes(lanes)
+    c.ensure_batch_workspace(n, k, d, p, w.dtype, lanes)
+    kinds = [ORTHOGONAL if i % 3 else NONORTHOGONAL for i in range(calls)]
+    Hs, Ws, seeds = [], [], []
+    for i in range(calls):
+        H, W, seed = inputs.make_call_inputs(w, i, "cuda")
+        Hs.append(H); Ws.append(W); seeds.append(seed)
+    mk = lambda: [torch.full((n, p // 3), float("nan"), device="cuda", dtype=torch.bfloat16) for _ in range(calls)]
+    Q1, K1, V1 = mk(), mk(), mk()
+    Q2, K2, V2 = mk(), mk(), mk()
+    torch.cuda.synchronize()
+    c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, Q1, K1, V1)
+    # next layer's activations from this layer's outputs, on the caller's stream (d = p / 3 here)
+    H2 = [(0.5 * (Q1[i] + V1[i]) + Hs[i]).contiguous() for i in range(calls)]
+    seeds2 = [s_ + 999 for s_ in seeds]
+    c.qkv_offload_batch(H2, Ws, n, k, d, p, kinds, seeds2, w.shield_scale, w.dtype, Q2, K2, V2)
+    # the first batch's outputs are consumed after the second batch was enqueued
+    sums = [Q1[i].float().sum() + K1[i].float().sum() for i in range(calls)]
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    for i in range(calls):
+        Q = torch.empty((n, p // 3), device="cuda", dtype=torch.bfloat16); K = torch.empty_like(Q); V = torch.empty_like(Q)
+        c.qkv_offload(Hs[i], Ws[i], n, k, d, p, kinds[i], seeds[i], w.shield_scale, w.dtype, Q, K, V)
+        torch.cuda.synchronize()
+        assert torch.equal(Q, Q1[i]) and torch.equal(K, K1[i]) and torch.equal(V, V1[i])
+        assert float(sums[i]) == float(Q.float().sum() + K.float().sum())
+        h2 = (0.5 * (Q + V) + Hs[i]).contiguous()
+        assert torch.equal(h2, H2[i])
+        c.qkv_offload(h2, Ws[i], n, k, d, p, kinds[i], seeds2[i], w.shield_scale, w.dtype, Q, K, V)
+        torch.cuda.synchronize()
+        assert torch.equal(Q, Q2[i]) and torch.equal(K, K2[i]) and torch.equal(V, V2[i])
+        if i in (0, 5, 11):
+            y = np.hstack([f64(Q2[i]), f64(K2[i]), f64(V2[i])])
+            assert oracle.rel_fro(y, oracle.direct(f64(h2), f64(Ws[i]))) <= TOL["bf16"]
+    c.close()
+
+
 def test_batched_offload_full_size(oracle):
     w = inputs.WORKLOADS["prefill_bf16"]
     n, k, d, p = w.n, w.k, w.d, w.p
