@@ -142,8 +142,8 @@ int gelo_qr_orthogonal(gelo_ctx* ctx, int m, float* G_dev, int ld, float* Q_dev,
  * A_dev is preserved.  Needs workspace for (m, 0). */
 int gelo_lu_inverse(gelo_ctx* ctx, int m, const float* A_dev, int ld, float* Ainv_dev, void* stream);
 
-/* cond_dev[0] = estimate of kappa_2(A) = sigma_max(A) * sigma_max(A^-1) by power
- * iteration on A^T A and A^-T A^-1 (a lower estimate, within a few percent).  ld must be a multiple of 8
+/* cond_dev[0] = estimate of kappa_2(A) = sigma_max(A) * sigma_max(A^-1): square roots of the largest
+ * Ritz values of A^T A and A^-T A^-1 after six Lanczos steps (a lower estimate, within a few percent).  ld must be a multiple of 8
  * and both matrices 16-byte aligned. */
 int gelo_cond_estimate(gelo_ctx* ctx, int m, const float* A_dev, const float* Ainv_dev, int ld,
                        float* cond_dev, void* stream);

@@ -1,10 +1,13 @@
 // 2-norm condition number estimate of the non-orthogonal mixing matrix (paper
 // Mitigation 1: "generate and verify well-conditioned A (e.g., enforce kappa(A) < 100)").
-// kappa_2(A) = sigma_max(A) * sigma_max(A^-1); each factor by power iteration on
-// Op^T Op with Op = A (z = 0) and Op = A^-1 (z = 1), both run in the same launches.
+// kappa_2(A) = sigma_max(A) * sigma_max(A^-1); each factor is the square root of the largest Ritz value of
+// Op^T Op after a few Lanczos steps from a Gaussian start vector, with Op = A (z = 0) and Op = A^-1 (z = 1), both
+// run in the same launches.  (Six Lanczos steps are as close as twelve steps of the power iteration: the Ritz value
+// is the best estimate the Krylov space holds, the power iterate only its last vector.  A Ritz value never exceeds
+// lambda_max, so the estimate is a lower one.)
 // The operators are the matrices as stored (bf16 or fp32), i.e. exactly what the mixing and unmixing products
-// read.  All sums have a fixed order, so the estimate is bit-reproducible.  HBM-bound: every iteration streams
-// both matrices once from DRAM (the second touch of a row slab hits L2).
+// read.  All sums have a fixed order, so the estimate is bit-reproducible.  Every step streams both matrices once
+// from DRAM (the second touch of a row slab hits L2).
 #include "common.cuh"
 #include "philox.cuh"
 
@@ -13,14 +16,17 @@ namespace gelo {
 namespace {
 
 constexpr int kCondSlabsMax = 160;   // row slabs of one operator pass (one CTA each)
-constexpr int kPowerIters = 12;      // the estimate is within about 4% of kappa_2 after 12 steps (measured at m = 512 .. 4300)
+constexpr int kCondChunkCols = 256;  // entries per CTA of the reduction over slabs
+constexpr int kLanczosSteps = 6;     // the estimate is within about 6% of kappa_2 (measured at m = 64 .. 4300, gamma 0.5 .. 3)
 
 struct CondViews {
     const void* op[2];
     int ld, m, mpad, slabs, rows_per;
-    float* xhat;      // [2][mpad]
+    float* v;         // [2][mpad]  current Lanczos vector (unit length)
+    float* vprev;     // [2][mpad]  the one before
+    float* w;         // [2][mpad]  Op^T Op v
     float* partial;   // [2][slabs][mpad]
-    float* scal;      // [0..1] sigma estimates
+    float* tri;       // [2][2][kLanczosSteps]  diagonal and off-diagonal of the Lanczos tridiagonal matrices
 };
 
 __global__ void cond_init_kernel(CondViews v, uint64_t seed, uint32_t attempt)
@@ -38,39 +44,101 @@ __global__ void cond_init_kernel(CondViews v, uint64_t seed, uint32_t attempt)
     }
 }
 
-// xhat = (sum of slab partials) / its norm;  scal[z] = sqrt(norm)
-__global__ void __launch_bounds__(1024) cond_normalise_kernel(CondViews v)
+// w = sum of slab partials (slabs ascend: fixed order), one thread per entry.
+__global__ void __launch_bounds__(kCondChunkCols) cond_reduce_kernel(CondViews v)
 {
-    __shared__ float red[32];
-    __shared__ float total;
-    const int z = blockIdx.x;
-    float local = 0.0f;
-    for (int i = threadIdx.x; i < v.m; i += blockDim.x) {
-        float s = 0.0f;
-        for (int k = 0; k < v.slabs; ++k) s += v.partial[((size_t)z * v.slabs + k) * v.mpad + i];
-        v.xhat[(size_t)z * v.mpad + i] = s;
-        local = fmaf(s, s, local);
-    }
+    const int z = blockIdx.y;
+    const int i = blockIdx.x * kCondChunkCols + threadIdx.x;
+    if (i >= v.m) return;
+    const float* p = v.partial + (size_t)z * v.slabs * v.mpad + i;
+    float s = 0.0f;
+    for (int k = 0; k < v.slabs; ++k) s += p[(size_t)k * v.mpad];
+    v.w[(size_t)z * v.mpad + i] = s;
+}
+
+// Sum over the CTA's threads in a fixed order; every thread receives it.
+__device__ __forceinline__ float cond_block_sum(float local, float* red)
+{
 #pragma unroll
     for (int off = 16; off > 0; off >>= 1) local += __shfl_xor_sync(0xffffffffu, local, off);
+    __syncthreads();                                         // red may still be read from the previous sum
     if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = local;
     __syncthreads();
-    if (threadIdx.x < 32) {
-        float t = red[threadIdx.x];
+    float t = red[threadIdx.x & 31];
 #pragma unroll
-        for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
-        if (threadIdx.x == 0) total = t;
+    for (int off = 16; off > 0; off >>= 1) t += __shfl_xor_sync(0xffffffffu, t, off);
+    return t;
+}
+
+// One CTA per operator.  step < 0: v = w / |w| (the start vector), vprev = 0.  Otherwise the Lanczos recurrence
+//   alpha = v . w,  r = w - alpha v - beta_prev vprev,  beta = |r|,  vprev <- v,  v <- r / beta.
+__global__ void __launch_bounds__(1024) cond_lanczos_kernel(CondViews v, int step)
+{
+    __shared__ float red[32];
+    const int z = blockIdx.x;
+    float* vc = v.v + (size_t)z * v.mpad;
+    float* vp = v.vprev + (size_t)z * v.mpad;
+    float* w = v.w + (size_t)z * v.mpad;
+    float* alpha = v.tri + (size_t)z * 2 * kLanczosSteps;
+    float* beta = alpha + kLanczosSteps;
+    if (step < 0) {
+        float local = 0.0f;
+        for (int i = threadIdx.x; i < v.m; i += 1024) local = fmaf(w[i], w[i], local);
+        const float nrm = sqrtf(cond_block_sum(local, red));
+        const float inv = nrm > 0.0f ? 1.0f / nrm : 0.0f;
+        for (int i = threadIdx.x; i < v.m; i += 1024) { vc[i] = w[i] * inv; vp[i] = 0.0f; }
+        return;
     }
-    __syncthreads();
-    const float nrm = sqrtf(total);
-    const float inv = nrm > 0.0f ? 1.0f / nrm : 0.0f;
-    for (int i = threadIdx.x; i < v.m; i += blockDim.x) v.xhat[(size_t)z * v.mpad + i] *= inv;
-    if (threadIdx.x == 0) v.scal[z] = sqrtf(nrm);   // nrm -> lambda_max(Op^T Op) = sigma_max^2
+    float local = 0.0f;
+    for (int i = threadIdx.x; i < v.m; i += 1024) local = fmaf(vc[i], w[i], local);
+    const float a = cond_block_sum(local, red);
+    const float bprev = step > 0 ? beta[step - 1] : 0.0f;
+    local = 0.0f;
+    for (int i = threadIdx.x; i < v.m; i += 1024) {
+        const float r = w[i] - a * vc[i] - bprev * vp[i];
+        w[i] = r;
+        local = fmaf(r, r, local);
+    }
+    const float b = sqrtf(cond_block_sum(local, red));
+    const float inv = b > 0.0f ? 1.0f / b : 0.0f;
+    for (int i = threadIdx.x; i < v.m; i += 1024) {          // (each thread touches only the entries it wrote)
+        vp[i] = vc[i];
+        vc[i] = w[i] * inv;
+    }
+    if (threadIdx.x == 0) { alpha[step] = a; beta[step] = b; }
+}
+
+// Largest eigenvalue of the symmetric tridiagonal matrix (alpha[0..k-1]; beta[0..k-2]) by bisection on the number of
+// eigenvalues below x (Sturm sequence), between 0 and the Gershgorin bound.  A breakdown (beta = 0) only decouples
+// the matrix: the count stays valid.
+__device__ double tridiagonal_lambda_max(const float* alpha, const float* beta, int k)
+{
+    double hi = 0.0;
+    for (int i = 0; i < k; ++i) {
+        const double r = fabs((double)alpha[i]) + (i > 0 ? fabs((double)beta[i - 1]) : 0.0) + (i + 1 < k ? fabs((double)beta[i]) : 0.0);
+        if (r > hi) hi = r;
+    }
+    double lo = 0.0;
+    for (int it = 0; it < 60; ++it) {
+        const double x = 0.5 * (lo + hi);
+        int below = 0;
+        double q = 1.0;
+        for (int i = 0; i < k; ++i) {
+            const double b2 = i > 0 ? (double)beta[i - 1] * (double)beta[i - 1] : 0.0;
+            q = (double)alpha[i] - x - (i > 0 ? b2 / q : 0.0);
+            if (q == 0.0) q = -1e-300;
+            if (q < 0.0) ++below;
+        }
+        if (below == k) hi = x; else lo = x;
+    }
+    return 0.5 * (lo + hi);
 }
 
 __global__ void cond_verdict_kernel(CondViews v, float bound, float* cond_out, int* status, int deferred)
 {
-    const float c = v.scal[0] * v.scal[1];
+    // lambda_max(Op^T Op) = sigma_max^2
+    const float c = (float)(sqrt(tridiagonal_lambda_max(v.tri, v.tri + kLanczosSteps, kLanczosSteps)) *
+                            sqrt(tridiagonal_lambda_max(v.tri + 2 * kLanczosSteps, v.tri + 3 * kLanczosSteps, kLanczosSteps)));
     if (cond_out) cond_out[0] = c;
     const int ok = (c * 1.2f <= bound && c == c) ? 1 : 0;   // the estimate is a lower one (tests: >= 0.85 of the true value)
     status[1] = ok;
@@ -106,7 +174,7 @@ __device__ __forceinline__ void load8(const __half* p, float (&a)[8])
     }
 }
 
-// One power-iteration step Op^T (Op xhat) in a single pass over the operator: CTA (slab, z) first forms y_r =
+// One application Op^T (Op v) in a single pass over the operator: CTA (slab, z) first forms y_r =
 // Op[r, :] . xhat for its rows (one warp per row), then accumulates sum_r y_r Op[r, :] for every column; the
 // second read of the slab comes from L2.  partial[z][slab][:] receives the slab's contribution.
 template <typename T>
@@ -118,7 +186,7 @@ __global__ void __launch_bounds__(256) cond_step_kernel(CondViews v)
     const int r1 = min(v.m, r0 + v.rows_per);
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const T* op = static_cast<const T*>(v.op[z]);
-    const float* x = v.xhat + (size_t)z * v.mpad;
+    const float* x = v.v + (size_t)z * v.mpad;
     const int groups = (v.m + 7) >> 3;
     // loads are issued four at a time before anything is consumed: with one CTA's few warps per SM the kernel lives
     // on memory-level parallelism
@@ -176,8 +244,8 @@ CondScratch carve_cond(Arena& a, int m)
 {
     CondScratch s;
     const size_t mpad = (size_t)((m + 63) / 64) * 64;
-    s.vec = static_cast<float*>(a.take((2 + 2 * kCondSlabsMax) * mpad * sizeof(float)));
-    s.scal = static_cast<float*>(a.take(16 * sizeof(float)));
+    s.vec = static_cast<float*>(a.take((6 + 2 * kCondSlabsMax) * mpad * sizeof(float)));
+    s.scal = static_cast<float*>(a.take((16 + 4 * kLanczosSteps) * sizeof(float)));
     return s;
 }
 
@@ -189,23 +257,28 @@ int run_cond_estimate(gelo_ctx* ctx, int m, const void* A, const void* Ainv, int
     v.op[0] = A; v.op[1] = Ainv; v.ld = ld; v.m = m; v.mpad = ((m + 63) / 64) * 64;
     v.slabs = ceil_div(m, 32) < kCondSlabsMax ? ceil_div(m, 32) : kCondSlabsMax;
     v.rows_per = ceil_div(m, v.slabs);
-    v.xhat = s.vec;
-    v.partial = s.vec + 2 * (size_t)v.mpad;
-    v.scal = s.scal;
+    v.v = s.vec;
+    v.vprev = s.vec + 2 * (size_t)v.mpad;
+    v.w = s.vec + 4 * (size_t)v.mpad;
+    v.partial = s.vec + 6 * (size_t)v.mpad;
+    v.tri = s.scal + 16;
     const size_t ys_bytes = (size_t)v.rows_per * sizeof(float);
     if (ys_bytes > 48 * 1024) return GELO_ERR_UNSUPPORTED;
     dim3 gi(ceil_div(v.mpad, 4 * 256), 2);
     cond_init_kernel<<<gi, 256, 0, st>>>(v, 0x5eedull, 0u);
     GELO_TRY(after_launch(ctx));
-    cond_normalise_kernel<<<2, 1024, 0, st>>>(v);
-    GELO_TRY(after_launch(ctx));
-    for (int it = 0; it < kPowerIters; ++it) {
-        dim3 g(v.slabs, 2);
-        if (dtype == GELO_BF16) cond_step_kernel<__nv_bfloat16><<<g, 256, ys_bytes, st>>>(v);
-        else if (dtype == GELO_F16) cond_step_kernel<__half><<<g, 256, ys_bytes, st>>>(v);
-        else cond_step_kernel<float><<<g, 256, ys_bytes, st>>>(v);
+    const dim3 gr(ceil_div(m, kCondChunkCols), 2);
+    for (int step = -1; step < kLanczosSteps; ++step) {
+        if (step >= 0) {
+            dim3 g(v.slabs, 2);
+            if (dtype == GELO_BF16) cond_step_kernel<__nv_bfloat16><<<g, 256, ys_bytes, st>>>(v);
+            else if (dtype == GELO_F16) cond_step_kernel<__half><<<g, 256, ys_bytes, st>>>(v);
+            else cond_step_kernel<float><<<g, 256, ys_bytes, st>>>(v);
+            GELO_TRY(after_launch(ctx));
+        }
+        cond_reduce_kernel<<<gr, kCondChunkCols, 0, st>>>(v);
         GELO_TRY(after_launch(ctx));
-        cond_normalise_kernel<<<2, 1024, 0, st>>>(v);
+        cond_lanczos_kernel<<<2, 1024, 0, st>>>(v, step);
         GELO_TRY(after_launch(ctx));
     }
     cond_verdict_kernel<<<1, 1, 0, st>>>(v, bound, cond_out, ctx->status_dev, deferred ? 1 : 0);

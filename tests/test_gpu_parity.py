@@ -125,7 +125,7 @@ def test_cond_estimate(ctx, oracle, m, gamma):
     ctx.cond_estimate(m, A, X, ld, c)
     ref = oracle.cond2(A64)
     est = c.item()
-    assert 0.88 * ref <= est <= 1.001 * ref               # power iteration: a lower estimate within ~10%
+    assert 0.88 * ref <= est <= 1.001 * ref               # a Ritz value of a few Lanczos steps: a lower estimate within ~10%
 
 
 # ------------------------------------------------------------------------- sample_mixing
