@@ -74,6 +74,7 @@ Layout carve(Arena& a, int n, int k, int d, int p, int dtype, bool host_staging)
     L.qr = carve_qr(a, L.m, L.ldi, &idle, &idle_bytes);
     L.lu = carve_lu(a, L.m, L.ldi);
     L.lu.M = L.qr.V;
+    L.lu.Z = L.G;                                          // the Gaussian / R is dead once A32 is formed
     L.cond = carve_cond(a, L.m);
     L.tc = carve_tc(a, L.m, L.ldi, &idle, &idle_bytes);
     for (int h = 0; h < 2; ++h)                            // 2 x (m x ld) 16-bit values: exactly the fp32 matrix X32

@@ -268,6 +268,7 @@ int polish_orthogonal_tf32(gelo_ctx*, int m, float* Q, int ld, float* D, float* 
 
 struct LuScratch {
     float* M = nullptr;   // m x ld working copy
+    float* Z = nullptr;   // m x ld, optional: room for L^-1 (lets the forward solve skip the zero blocks); may not alias M, A or the result
     int* ipiv = nullptr;  // m
     int* perm = nullptr;  // m
     int* swap_table = nullptr;  // composed interchanges of one panel / block: count, then (target, source) pairs

@@ -514,6 +514,24 @@ __global__ void permuted_ones_kernel(float* __restrict__ X, int ld, int m, const
     if (r < m) X[(size_t)r * ld + perm[r]] = 1.0f;
 }
 
+// X[:, perm[k]] = Z[:, k] for every column k (Z P for the permutation matrix P with P[k, perm[k]] = 1); the padding
+// columns of X are cleared.  One CTA per row: the row is read in order and scattered inside its own 4 ld bytes.
+__global__ void __launch_bounds__(256)
+permute_columns_kernel(const float* __restrict__ Z, float* __restrict__ X, int ld, int m, const int* __restrict__ perm)
+{
+    const size_t row = (size_t)blockIdx.x * ld;
+    for (int k = threadIdx.x; k < ld; k += 256) {
+        if (k < m) X[row + perm[k]] = Z[row + k];
+        else X[row + k] = 0.0f;
+    }
+}
+
+__global__ void unit_diagonal_kernel(float* __restrict__ Z, int ld, int m)
+{
+    const int r = blockIdx.x * blockDim.x + threadIdx.x;
+    if (r < m) Z[(size_t)r * ld + r] = 1.0f;
+}
+
 // X = P (X[i, perm[i]] = 1): a memset at copy speed, then the ones.
 int set_permutation(gelo_ctx* ctx, float* X, int ld, int m, const int* perm, cudaStream_t st)
 {
@@ -598,6 +616,32 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         GELO_CUDA_OK(cudaFuncSetAttribute(build_perm_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)perm_smem));
     build_perm_kernel<<<1, 256, perm_smem, st>>>(s.ipiv, s.perm, m);
     GELO_TRY(after_launch(ctx));
+    if (s.Z) {
+        // L Y = P: Y = L^-1 P, and L^-1 is unit lower triangular.  Z = L^-1 is built in place from the identity, every
+        // block row touching only the columns left of its own end (the rest are zeros that stay zeros), which is a
+        // third of the arithmetic of solving against the dense P; Y is Z with its columns permuted.
+        float* Z = s.Z;
+        GELO_CUDA_OK(cudaMemsetAsync(Z, 0, (size_t)m * ld * sizeof(float), st));
+        unit_diagonal_kernel<<<ceil_div(m, 256), 256, 0, st>>>(Z, ld, m);
+        GELO_TRY(after_launch(ctx));
+        for (int s0 = 0; s0 < m; s0 += kSuper) {
+            const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
+            const int send = s0 + sw;
+            for (int b0 = s0; b0 < send; b0 += kOuter) {
+                const int ob = (send - b0 < kOuter) ? (send - b0) : kOuter;
+                const int bend = b0 + ob;
+                GELO_TRY(launch_tri_solve128<false>(ctx, M, ld, Z, ld, b0, ob, 0, bend, st));
+                if (send > bend)
+                    GELO_TRY(tc_update_f32(ctx, tc, tf32, send - bend, bend, ob, at(M, bend, b0), ld, at(Z, b0, 0), ld,
+                                           at(Z, bend, 0), ld, st));
+            }
+            if (m > send)
+                GELO_TRY(tc_update_f32(ctx, tc, tf32, m - send, send, sw, at(M, send, s0), ld, at(Z, s0, 0), ld, at(Z, send, 0), ld,
+                                       st));
+        }
+        permute_columns_kernel<<<m, 256, 0, st>>>(Z, X, ld, m, s.perm);
+        GELO_TRY(after_launch(ctx));
+    } else {
     GELO_TRY(set_permutation(ctx, X, ld, m, s.perm, st));
     for (int s0 = 0; s0 < m; s0 += kSuper) {
         const int sw = (m - s0 < kSuper) ? (m - s0) : kSuper;
@@ -612,6 +656,7 @@ int run_lu_inverse_tc(gelo_ctx* ctx, int m, const float* A, int ld, float* X, co
         }
         if (m > send)
             GELO_TRY(tc_update_f32(ctx, tc, tf32, m - send, m, sw, at(M, send, s0), ld, at(X, s0, 0), ld, at(X, send, 0), ld, st));
+    }
     }
     const int nsuper = ceil_div(m, kSuper);
     for (int sb = nsuper - 1; sb >= 0; --sb) {
