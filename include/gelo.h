@@ -283,6 +283,11 @@ int gelo_qkv_offload_host(gelo_ctx* ctx, const void* H_host, const void* W_dev, 
  *   Q_dev[i], K_dev[i], V_dev[i]: outputs of call i, as in gelo_unmix (K_dev[i] == V_dev[i] ==
  *   NULL for all i selects unsplit output).  Calls may share output buffers; they are written
  *   in call order.
+ * A small batch (n + k <= 128 on a 16-bit type, at least two lanes, outputs of different calls
+ * disjoint) runs each WHOLE call on its lane, shield rows, mixing and the fused projection +
+ * unmixing included, so that the weight streams of neighbouring calls overlap; `stream` then only
+ * waits for the lanes at the end.  The lanes read H_dev[i] and write the outputs after the point
+ * of `stream` at which the batch was enqueued.
  * Non-orthogonal calls use their first attempt only and never wait for the device: a missed
  * condition bound is reported by gelo_last_status as GELO_ERR_COND.  Needs a workspace of
  * gelo_batch_workspace_bytes(..., lanes) bytes.  Work on the lane streams is ordered after

@@ -4,6 +4,9 @@
 #include <new>
 
 #include "common.cuh"
+#include <algorithm>
+#include <utility>
+#include <vector>
 
 using namespace gelo;
 
@@ -375,6 +378,21 @@ int offload_batch_impl(gelo_ctx* ctx, int calls, const void* const* H, const voi
     bool small = !host && D > 1 && ctx->fuse_small && lane_width(n, k, d) > 0 && mix_small_supports(n, k, d, dtype) &&
                  project_unmix_supports(ctx, n, k, d, p, dtype, L[0].ldi, split ? 3 : 1);
     for (int i = 0; i < calls && small; ++i) small = !misaligned(H[i]);
+    if (small) {
+        // calls that share an output buffer are promised call order: keep those on the caller's stream
+        std::vector<std::pair<uintptr_t, uintptr_t>> out;
+        out.reserve((size_t)calls * 3);
+        const size_t bytes = split ? third : (size_t)n * p * es;
+        for (int i = 0; i < calls; ++i) {
+            out.emplace_back(reinterpret_cast<uintptr_t>(Q[i]), reinterpret_cast<uintptr_t>(Q[i]) + bytes);
+            if (split) {
+                out.emplace_back(reinterpret_cast<uintptr_t>(K[i]), reinterpret_cast<uintptr_t>(K[i]) + bytes);
+                out.emplace_back(reinterpret_cast<uintptr_t>(V[i]), reinterpret_cast<uintptr_t>(V[i]) + bytes);
+            }
+        }
+        std::sort(out.begin(), out.end());
+        for (size_t i = 1; i < out.size() && small; ++i) small = out[i].first >= out[i - 1].second;
+    }
     // with several lanes in flight each level-3 update takes a share of the SMs (ctx->lane_tc_share-th of them)
     ctx->tc_update_ctas = (D >= ctx->lane_tc_share && ctx->lane_tc_share > 1) ? ctx->sm_count / ctx->lane_tc_share : 0;
 

@@ -565,6 +565,42 @@ def test_small_batches_back_to_back_follow_the_callers_stream(oracle):
     c.close()
 
 
+def test_small_batch_with_shared_outputs_keeps_call_order():
+    """Calls of a batch may share their output buffers and are then written in call order, also for the small
+    batches whose calls would otherwise run concurrently on the lanes."""
+    w = inputs.WORKLOADS["decode_bf16"]
+    n, k, d, p = w.n, w.k, w.d, w.p
+    calls, lanes = 9, 4
+    c = binding.Context(0)
+    c.set_lanes(lanes)
+    c.ensure_batch_workspace(n, k, d, p, w.dtype, lanes)
+    Hs, Ws, seeds = [], [], []
+    for i in range(calls):
+        H, W, seed = inputs.make_call_inputs(w, i, "cuda")
+        Hs.append(H); Ws.append(W); seeds.append(seed)
+    kinds = [ORTHOGONAL] * calls
+    Q = torch.full((n, p // 3), float("nan"), device="cuda", dtype=torch.bfloat16); K = Q.clone(); V = Q.clone()
+    for rep in range(3):
+        c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, w.dtype, [Q] * calls, [K] * calls, [V] * calls)
+    torch.cuda.synchronize()
+    Ql = torch.empty_like(Q); Kl = torch.empty_like(Q); Vl = torch.empty_like(Q)
+    c.qkv_offload(Hs[-1], Ws[-1], n, k, d, p, kinds[-1], seeds[-1], w.shield_scale, w.dtype, Ql, Kl, Vl)
+    torch.cuda.synchronize()
+    assert torch.equal(Q, Ql) and torch.equal(K, Kl) and torch.equal(V, Vl)
+    # partially overlapping outputs count as shared too
+    big = torch.full((2 * n, p // 3), float("nan"), device="cuda", dtype=torch.bfloat16)
+    Qo = [big[: n], big[n // 2: n // 2 + n]]
+    Ko = [torch.empty_like(Q) for _ in range(2)]; Vo = [torch.empty_like(Q) for _ in range(2)]
+    c.qkv_offload_batch(Hs[:2], Ws[:2], n, k, d, p, kinds[:2], seeds[:2], w.shield_scale, w.dtype, Qo, Ko, Vo)
+    torch.cuda.synchronize()
+    c.qkv_offload(Hs[1], Ws[1], n, k, d, p, kinds[1], seeds[1], w.shield_scale, w.dtype, Ql, Kl, Vl)
+    c.qkv_offload(Hs[0], Ws[0], n, k, d, p, kinds[0], seeds[0], w.shield_scale, w.dtype, Q, K, V)
+    torch.cuda.synchronize()
+    assert torch.equal(Qo[1], Ql) and torch.equal(big[: n // 2], Q[: n // 2])
+    assert c.last_status() == binding.OK
+    c.close()
+
+
 def test_batched_offload_full_size(oracle):
     w = inputs.WORKLOADS["prefill_bf16"]
     n, k, d, p = w.n, w.k, w.d, w.p
