@@ -328,7 +328,7 @@ size_t gelo_batch_workspace_bytes(int n, int k, int d, int p, int dtype, int lan
 
 /* ---- structured variant: block-diagonal orthogonal mixing -------------------------------------- */
 
-/* The same offload with a block-diagonal orthogonal A (the paper lists "structured orthogonal transforms" as
+/* The same offload with a block-diagonal orthogonal A (the paper names structured orthogonal transforms as
  * future work for cheaper A-generation; this is one such structure, NOT the dense mixing of its Section 3.2).
  * The m = n + k rows are dealt into nb = ceil(m / block) groups (block a multiple of 64, nb <= lanes, n >= nb);
  * group j holds data rows [n j / nb, n (j+1) / nb) and shield rows [k j / nb, k (j+1) / nb), i.e. every group

@@ -252,7 +252,7 @@ int oracle_lu_inverse(int64_t m, const double* A, double* Ainv)
 }
 
 /* ------------------------------------------------------------------ */
-/* 2-norm condition number (Mitigation 1: "enforce kappa(A) < 100")    */
+/* 2-norm condition number (Mitigation 1: kappa(A) below a bound, 100)   */
 /* ------------------------------------------------------------------ */
 
 /*

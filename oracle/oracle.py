@@ -197,7 +197,7 @@ def sample_mixing(m, kind, seed, attempt=0, gamma=DEFAULT_GAMMA):
 
 def sample_mixing_verified(m, kind, seed, gamma=DEFAULT_GAMMA, bound=COND_BOUND, max_attempts=8):
     """Sample, verify kappa_2(A) <= bound for non-orthogonal A, resample with the next attempt
-    number otherwise ("generate and verify well-conditioned A").  Returns (A, Ainv, cond, attempt)."""
+    number otherwise (Mitigation 1 asks for a conditioning check on every drawn A).  Returns (A, Ainv, cond, attempt)."""
     for attempt in range(max_attempts):
         A, X = sample_mixing(m, kind, seed, attempt, gamma)
         if kind == ORTHOGONAL:

@@ -1,5 +1,5 @@
-// 2-norm condition number estimate of the non-orthogonal mixing matrix (paper
-// Mitigation 1: "generate and verify well-conditioned A (e.g., enforce kappa(A) < 100)").
+// 2-norm condition number estimate of the non-orthogonal mixing matrix (paper, Mitigation 1: a
+// non-orthogonal A is to be checked for good conditioning after it is drawn, a bound of 100 being the example).
 // kappa_2(A) = sigma_max(A) * sigma_max(A^-1); each factor is the square root of the largest Ritz value of
 // Op^T Op after a few Lanczos steps from a Gaussian start vector, with Op = A (z = 0) and Op = A^-1 (z = 1), both
 // run in the same launches.  (Six Lanczos steps are as close as twelve steps of the power iteration: the Ritz value
