@@ -720,9 +720,10 @@ def test_tensor_core_update_tf32(ctx, oracle, M, N, K):
     assert torch.isnan(C[:, N:]).all()                     # padding columns are never written
 
 
-@pytest.mark.parametrize("m", [100, 130, 257, 512, 1000])
+@pytest.mark.parametrize("m", [100, 130, 257, 512, 1000, 2300, 2700])
 def test_householder_qr_tf32_blocks(oracle, m):
-    """QR with tf32 level-3 updates and the Newton-Schulz polish, as the bf16 path runs it."""
+    """QR with tf32 level-3 updates and the Newton-Schulz polish, as the bf16 path runs it (2300 and 2700 rows: five and six
+    superblocks, the last one partial)."""
     c = make_ctx(m, 0, 8, 24, "f32")
     c.set_level3(3)
     ld = c.mixing_ld(m)
