@@ -565,6 +565,37 @@ def test_small_batches_back_to_back_follow_the_callers_stream(oracle):
     c.close()
 
 
+@pytest.mark.parametrize("dtype,n,k,d,p", [("f16", 48, 5, 1024, 3072), ("bf16", 100, 0, 2048, 1536), ("bf16", 17, 3, 512, 768)])
+def test_small_batches_other_shapes_and_types(oracle, dtype, n, k, d, p):
+    """Whole calls on the lanes for IEEE-half storage, for a call without shield rows and for a ragged row count:
+    same bytes as single calls, and H W within the 16-bit tolerance."""
+    w = inputs.Workload("small", n, k, d, p, dtype, (ORTHOGONAL, NONORTHOGONAL), 10.0, True, 77, 1)
+    calls, lanes = 7, 3
+    c = binding.Context(0)
+    c.set_lanes(lanes)
+    c.ensure_batch_workspace(n, k, d, p, dtype, lanes)
+    kinds = [w.kind(i) for i in range(calls)]
+    Hs, Ws, seeds = [], [], []
+    for i in range(calls):
+        H, W, seed = inputs.make_call_inputs(w, i, "cuda")
+        Hs.append(H); Ws.append(W); seeds.append(seed)
+    td = TDT[dtype]
+    mk = lambda: [torch.full((n, p // 3), float("nan"), device="cuda", dtype=td) for _ in range(calls)]
+    Qb, Kb, Vb = mk(), mk(), mk()
+    for rep in range(2):                                   # the second batch chains onto the first
+        c.qkv_offload_batch(Hs, Ws, n, k, d, p, kinds, seeds, w.shield_scale, dtype, Qb, Kb, Vb)
+    torch.cuda.synchronize()
+    assert c.last_status() == binding.OK
+    for i in range(calls):
+        Q = torch.empty((n, p // 3), device="cuda", dtype=td); K = torch.empty_like(Q); V = torch.empty_like(Q)
+        c.qkv_offload(Hs[i], Ws[i], n, k, d, p, kinds[i], seeds[i], w.shield_scale, dtype, Q, K, V)
+        torch.cuda.synchronize()
+        assert torch.equal(Q, Qb[i]) and torch.equal(K, Kb[i]) and torch.equal(V, Vb[i])
+        y = np.hstack([f64(Qb[i]), f64(Kb[i]), f64(Vb[i])])
+        assert oracle.rel_fro(y, oracle.direct(f64(Hs[i]), f64(Ws[i]))) <= TOL[dtype]
+    c.close()
+
+
 def test_small_batch_with_shared_outputs_keeps_call_order():
     """Calls of a batch may share their output buffers and are then written in call order, also for the small
     batches whose calls would otherwise run concurrently on the lanes."""
