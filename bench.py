@@ -26,6 +26,11 @@ import sys
 import threading
 import time
 
+# The batched entry points keep up to 32 lane streams busy; with the default of eight hardware work queues, streams
+# that share a queue wait for each other's launches (measured: 121.3 -> 118.7 ms per sweep).  The variable is read when
+# the CUDA context is created, i.e. it has to be set before torch touches the GPU; a caller's own setting wins.
+os.environ.setdefault("CUDA_DEVICE_MAX_CONNECTIONS", "32")
+
 ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
